@@ -1,0 +1,234 @@
+/*
+ * libstr -- token-reduced prefill of a hybrid Mamba-2 / attention layer stack, B200 (sm_100a).
+ *
+ * C ABI.  Conventions shared by every call:
+ *   - returns int: STR_OK (0) or a negative STR_ERR_* code; str_strerror() gives text.
+ *   - pointers named *_dev / documented "device" are DEVICE pointers owned by the caller; all
+ *     tensors are row-major and contiguous in the layout stated.  "host" pointers are host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work: they never allocate, free or synchronise, unless stated otherwise.
+ *   - scratch memory comes from a caller-provided device workspace whose size the matching
+ *     *_workspace_size() query returns (bytes; 256-byte aligned base expected).
+ *   - outputs are fully overwritten; inputs are never modified; in and out must not alias.
+ *   - dtype is STR_F32 (everything fp32) or STR_BF16 (bf16 storage, fp32 accumulation).
+ *   - bounded device-side waits: a kernel that gives up waiting records STR_ERR_TIMEOUT in the
+ *     context's device status word and returns; str_check_status() reads it back.
+ * Token order inside a sequence follows the paper's setting (Section 3.1): the n_vis visual
+ * tokens come first, the n_text text (query) tokens last; text tokens are never dropped.
+ */
+#ifndef STR_H_
+#define STR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    STR_OK = 0,
+    STR_ERR_INVALID_ARG = -1,
+    STR_ERR_UNSUPPORTED_SHAPE = -2,
+    STR_ERR_WORKSPACE_TOO_SMALL = -3,
+    STR_ERR_CUDA = -4,
+    STR_ERR_TIMEOUT = -5
+};
+
+enum { STR_F32 = 0, STR_BF16 = 1 };
+
+typedef struct str_ctx str_ctx;
+
+/* Context: device id, SM count, tensor-map encoder, device status word.  str_create allocates
+ * a few bytes of device memory and may synchronise; str_destroy frees them. */
+int str_create(int device, str_ctx **out);
+int str_destroy(str_ctx *ctx);
+const char *str_strerror(int code);
+/* Synchronises `stream`, returns the device status word (STR_OK or the first recorded error)
+ * and clears it.  The only hot-path call that synchronises. */
+int str_check_status(str_ctx *ctx, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * (1) Mamba-2 selective state-space scan.  Section 3.1 "State-Space (Mamba) Layers" and the
+ * appendix "State-Space Recurrence":  S_t = Abar_t S_{t-1} + x_t (Delta_t b_t)^T,  y_t = S_t c_t,
+ * Abar_t = exp(Delta_t * A_h) with the stored A_h < 0 (the paper writes exp(-Delta A), A > 0).
+ * Evaluated in chunked form (in-chunk cumulative log-decay, intra-chunk (C B^T o decay) X,
+ * chunk states, inter-chunk carry); the result equals the sequential recurrence up to fp32
+ * rounding and does not depend on the chunk length.
+ *   x   device [Bz,T,H,p] dtype        dt  device [Bz,T,H] fp32 (> 0, after softplus)
+ *   A   device [H] fp32 (< 0)          B,C device [Bz,T,G,n] dtype (head h uses group h/(H/G))
+ *   D   device [H] fp32 or NULL (y_t += D_h x_t)     init_state device [Bz,H,p,n] fp32 or NULL
+ *   y   device [Bz,T,H,p] dtype        final_state device [Bz,H,p,n] fp32 or NULL
+ * Q is a chunk-length hint (0 = library default); T need not be a multiple of it.
+ * Errors: INVALID_ARG (null pointer, non-positive size, H % G != 0), UNSUPPORTED_SHAPE
+ * (p or n beyond what the kernels tile), WORKSPACE_TOO_SMALL. */
+typedef struct {
+    int Bz, T, H, p, n, G, Q, dtype;
+} str_ssd_shape;
+size_t str_mamba2_prefill_workspace_size(const str_ssd_shape *s);
+int str_mamba2_prefill(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float *dt,
+                       const float *A, const void *B, const void *C, const float *D,
+                       const float *init_state, void *y, float *final_state, void *workspace,
+                       size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * (2a) Mamba importance, Eq. 2 (Decoupled Content Alignment, decay excluded):
+ *   s_i = 1/(M G) sum_{m,g} | (Deltabar_i^(g) b_i^(g))^T c_m^(g) |,
+ * Deltabar_i^(g) = mean of dt[i,h] over the heads of group g; i over the first n_vis rows,
+ * m over the last n_text rows of the same B, C, dt buffers the scan reads.
+ *   scores_out device [Bz,n_vis] fp32.   n_vis + n_text must equal T. */
+typedef struct {
+    int Bz, T, H, n, G, dtype;
+} str_ssm_score_shape;
+size_t str_mamba_importance_workspace_size(const str_ssm_score_shape *s, int n_vis, int n_text);
+int str_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text,
+                         const void *B, const void *C, const float *dt, float *scores_out,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+/* (2b) Attention importance, Section 3.1 "Attention Layers":
+ *   s_i = 1/(M Hq) sum_{m,h} softmax_i( q_m^(h) . k_i^(kv(h)) * softmax_scale ),
+ * softmax over the n_vis visual keys, m over the last n_text query rows, kv(h) = h/(Hq/Hkv).
+ *   q device [Bz,T,Hq,d] dtype (post-RoPE), k device [Bz,T,Hkv,d] dtype (post-RoPE),
+ *   scores_out device [Bz,n_vis] fp32.  Workspace holds the per-(head, query) row maxima and
+ *   sums of the first pass. */
+typedef struct {
+    int Bz, T, Hq, Hkv, d, dtype;
+} str_attn_score_shape;
+size_t str_attn_importance_workspace_size(const str_attn_score_shape *s, int n_vis, int n_text);
+int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
+                        const void *q, const void *k, float softmax_scale, float *scores_out,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * (3) Top-K selection preserving temporal order (Section 3.1 "Token Selection"): the indices of
+ * the k largest scores of each row, written in ascending index order.  Among equal scores the
+ * lower index is kept.  Radix select on the order-preserving integer image of fp32.
+ *   scores device [Bz,n_vis] fp32 (any finite values; NaN unsupported),
+ *   kept_idx_out device [Bz,k] int32.  k == n_vis gives 0..n_vis-1; k == 0 writes nothing;
+ *   k > n_vis or k < 0 -> INVALID_ARG. */
+size_t str_topk_select_workspace_size(int Bz, int n_vis, int k);
+int str_topk_select(str_ctx *ctx, int Bz, int n_vis, int k, const float *scores,
+                    int32_t *kept_idx_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/* (4) Compaction ("retain the top-K tokens", Section 3.1): per sequence, output row j < k is
+ * input row kept_idx[j]; output rows k .. k+n_text-1 are the text rows n_vis .. n_vis+n_text-1.
+ * The same gather is applied to hidden states, positions and the index map (which therefore
+ * composes back to original token ids over several reductions).  Bit-exact copy.
+ *   hidden device [Bz,T_in,D] dtype, positions/idx_map device [Bz,T_in] int32,
+ *   kept_idx device [Bz,k] int32 (ascending, each in [0,n_vis)),
+ *   outputs device [Bz,k+n_text,D], [Bz,k+n_text], [Bz,k+n_text].  T_in = n_vis + n_text.
+ *   positions / idx_map (and their outputs) may be NULL together.  D*sizeof(dtype) must be a
+ *   multiple of 16 bytes. */
+int str_compact(str_ctx *ctx, int Bz, int T_in, int n_vis, int n_text, int k, int D, int dtype,
+                const void *hidden, const int32_t *positions, const int32_t *idx_map,
+                const int32_t *kept_idx, void *hidden_out, int32_t *positions_out,
+                int32_t *idx_map_out, void *stream);
+
+/* (5) Retention schedule -> keep counts (Section 3.2; appendix "Reduction Schedule
+ * Configurations"; host only, no CUDA).  alpha_bp[l] is layer l's retention ratio in basis
+ * points of the ORIGINAL visual count n0; K_out[l] = min(n_cur, max(min_keep, floor(alpha n0)))
+ * is the visual count after layer l.  Layer l reduces iff K_out[l] < its incoming count. */
+int str_schedule_keep_counts(const int *alpha_bp, int L, int n0, int min_keep, int *K_out);
+/* Sigmoid retention alpha_l = a_end + (a_start - a_end) * sigmoid(k (x0 - l/L)), in basis points
+ * (rounded to nearest), l = 0..L-1.  Host only. */
+int str_sigmoid_schedule_bp(int L, double k, double x0, double a_start, double a_end, int *alpha_bp_out);
+
+/* ------------------------------------------------------------------------------------------
+ * Block glue.  The paper gives only the recurrence and the scores; these are the standard
+ * pre-norm Mamba-2 / GQA block pieces needed to run a layer stack.  Same conventions.
+ * ------------------------------------------------------------------------------------------ */
+
+/* out[M,N] = a[M,K] * w[N,K]^T (+ residual[M,N] if not NULL).  a, w, residual, out device, dtype.
+ * Weights are stored [out_features, in_features] (K contiguous). */
+size_t str_gemm_workspace_size(int M, int N, int K, int dtype);
+int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w,
+             const void *residual, void *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/* out[r,:] = in[r,:] / sqrt(mean(in[r,:]^2) + eps)  (unit weight), rows x D, dtype. */
+int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, const void *in, void *out,
+                void *stream);
+
+/* Mamba-2 pre-scan step on the in_proj output zxbcdt [Bz*T, 2*d_inner + 2*G*n + H] =
+ * [z | x B C | dt_raw]: causal depthwise conv (width W, zero left padding per sequence, taps
+ * conv_w [d_inner+2Gn, W] fp32, last tap on the current token, bias conv_b fp32) + SiLU on the
+ * x B C columns, split into x_out [Bz,T,H,p], B_out, C_out [Bz,T,G,n] (dtype), and
+ * dt_out [Bz,T,H] fp32 = softplus(dt_raw + dt_bias[h]). */
+int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, int n, int G, int W,
+                         const void *zxbcdt, const float *conv_w, const float *conv_b,
+                         const float *dt_bias, void *x_out, void *B_out, void *C_out, float *dt_out,
+                         void *stream);
+
+/* out[r,:] = RMSNorm( y[r,:] * SiLU(z[r,:]) ) over d_inner columns; z is read in place from the
+ * in_proj output (row stride ld_z elements, first d_inner columns). */
+int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps,
+                      const void *y, const void *z, void *out, void *stream);
+
+/* Splits qkv [Bz*T, (Hq+2Hkv)*d] into q_out [Bz,T,Hq,d], k_out, v_out [Bz,T,Hkv,d] and applies
+ * rotary embedding (half-split pairing (i, i+d/2), angle = position * theta^(-2i/d)) to q and k
+ * using the carried original positions [Bz,T] int32. */
+int str_rope_split(str_ctx *ctx, int dtype, int Bz, int T, int Hq, int Hkv, int d, float theta,
+                   const int32_t *positions, const void *qkv, void *q_out, void *k_out,
+                   void *v_out, void *stream);
+
+/* Causal GQA softmax attention over each sequence: o[t] = sum_{j<=t} softmax_j(q_t.k_j*scale) v_j.
+ * q,o device [Bz,T,Hq,d]; k,v device [Bz,T,Hkv,d]; dtype. */
+typedef struct {
+    int Bz, T, Hq, Hkv, d, dtype;
+} str_attn_shape;
+size_t str_attn_prefill_workspace_size(const str_attn_shape *s);
+int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k,
+                     const void *v, float softmax_scale, void *o, void *workspace,
+                     size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Whole stack: token-reduced prefill with a per-layer keep schedule (Sections 3.1-3.2).
+ * Layer l's mixer runs on the incoming tokens, its own importance score ranks the incoming
+ * visual tokens, and its OUTPUT is compacted to keep_counts[l] visual tokens when that is
+ * smaller than the incoming count.  Block wrapper: h <- h + Mixer(RMSNorm(h)).
+ * ------------------------------------------------------------------------------------------ */
+enum { STR_LAYER_MAMBA = 0, STR_LAYER_ATTN = 1 };
+typedef struct {
+    int kind;             /* STR_LAYER_MAMBA or STR_LAYER_ATTN                                  */
+    const void *w_in;     /* device: Mamba in_proj [2*d_inner+2Gn+H, D] | attention W_qkv [(Hq+2Hkv)d, D] */
+    const void *w_out;    /* device: Mamba out_proj [D, d_inner]        | attention W_o [D, Hq*d]         */
+    const float *conv_w;  /* device, Mamba only: [d_inner+2Gn, W]                                */
+    const float *conv_b;  /* device, Mamba only: [d_inner+2Gn]                                   */
+    const float *dt_bias; /* device, Mamba only: [H]                                             */
+    const float *A;       /* device, Mamba only: [H], negative                                   */
+} str_layer;
+typedef struct {
+    int Bz, n_vis, n_text, D, dtype;
+    int H, p, n, G, Q, conv_width;     /* Mamba-2 layer shape     */
+    int Hq, Hkv, d;                    /* attention layer shape   */
+    float rope_theta, norm_eps;
+    int n_layers;
+    const str_layer *layers;           /* host array [n_layers]                              */
+    const int *keep_counts;            /* host array [n_layers], from str_schedule_keep_counts */
+    int score_every_layer;             /* nonzero: also compute (not apply) the score at layers that do not reduce */
+} str_stack_desc;
+size_t str_stack_workspace_size(const str_stack_desc *d);
+/* hidden_in device [Bz, n_vis+n_text, D] dtype.  Outputs (device): hidden_out
+ * [Bz, K_last+n_text, D] dtype, positions_out / idx_map_out [Bz, K_last+n_text] int32 (original
+ * token ids of the surviving rows), where K_last = keep_counts[n_layers-1].
+ * kept_trace (device, optional, may be NULL): for each reducing layer in order, its kept
+ * indices [Bz,K_l] int32, packed one after the other; scores_trace likewise [Bz,n_cur] fp32. */
+int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in,
+                      void *hidden_out, int32_t *positions_out, int32_t *idx_map_out,
+                      int32_t *kept_trace, float *scores_trace, void *workspace,
+                      size_t workspace_bytes, void *stream);
+/* Same, with HOST hidden_in / hidden_out / idx_map_out buffers (pinned memory recommended):
+ * copies the input to the device, runs the stack, copies the results back, and synchronises
+ * `stream` before returning.  The device staging area is part of the workspace
+ * (str_stack_host_workspace_size). */
+size_t str_stack_host_workspace_size(const str_stack_desc *d);
+int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in_host,
+                           void *hidden_out_host, int32_t *idx_map_out_host, void *workspace,
+                           size_t workspace_bytes, void *stream);
+
+/* Number of kernels this library has launched on this context since creation (host counter). */
+long long str_launch_count(const str_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STR_H_ */

@@ -1,0 +1,383 @@
+"""Thin ctypes binding over libstr.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see ``include/str.h``) and takes torch
+CUDA tensors, which serve purely as device memory; all arithmetic runs in the library's kernels.
+There is no fallback: if the library is missing or a call fails, an exception is raised.
+"""
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libstr.so")
+
+STR_F32, STR_BF16 = 0, 1
+STR_LAYER_MAMBA, STR_LAYER_ATTN = 0, 1
+c_int, c_float, c_size_t, c_void_p = ctypes.c_int, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
+
+
+class StrError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s failed: %s (%d)" % (where, lib().str_strerror(code).decode(), code))
+
+
+class SsdShape(ctypes.Structure):
+    _fields_ = [(k, c_int) for k in ("Bz", "T", "H", "p", "n", "G", "Q", "dtype")]
+
+
+class SsmScoreShape(ctypes.Structure):
+    _fields_ = [(k, c_int) for k in ("Bz", "T", "H", "n", "G", "dtype")]
+
+
+class AttnScoreShape(ctypes.Structure):
+    _fields_ = [(k, c_int) for k in ("Bz", "T", "Hq", "Hkv", "d", "dtype")]
+
+
+class AttnShape(ctypes.Structure):
+    _fields_ = [(k, c_int) for k in ("Bz", "T", "Hq", "Hkv", "d", "dtype")]
+
+
+class Layer(ctypes.Structure):
+    _fields_ = [("kind", c_int), ("w_in", c_void_p), ("w_out", c_void_p), ("conv_w", c_void_p),
+                ("conv_b", c_void_p), ("dt_bias", c_void_p), ("A", c_void_p)]
+
+
+class StackDesc(ctypes.Structure):
+    _fields_ = ([(k, c_int) for k in ("Bz", "n_vis", "n_text", "D", "dtype", "H", "p", "n", "G", "Q",
+                                      "conv_width", "Hq", "Hkv", "d")]
+                + [("rope_theta", c_float), ("norm_eps", c_float), ("n_layers", c_int),
+                   ("layers", ctypes.POINTER(Layer)), ("keep_counts", ctypes.POINTER(c_int)),
+                   ("score_every_layer", c_int)])
+
+
+EXPORTS = [
+    "str_create", "str_destroy", "str_strerror", "str_check_status", "str_launch_count",
+    "str_mamba2_prefill_workspace_size", "str_mamba2_prefill",
+    "str_mamba_importance_workspace_size", "str_mamba_importance",
+    "str_attn_importance_workspace_size", "str_attn_importance",
+    "str_topk_select_workspace_size", "str_topk_select", "str_compact",
+    "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
+    "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_mamba_conv_split", "str_gated_rmsnorm",
+    "str_rope_split", "str_attn_prefill_workspace_size", "str_attn_prefill",
+    "str_stack_workspace_size", "str_stack_prefill", "str_stack_host_workspace_size",
+    "str_stack_prefill_host",
+]
+
+_LIB = None
+
+
+def lib():
+    """Load libstr.so once.  Raises if it has not been built (python -m paper_2603_00198_b200.build)."""
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libstr.so not found at %s; run `python -m paper_2603_00198_b200.build`" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        L.str_strerror.restype = ctypes.c_char_p
+        L.str_launch_count.restype = ctypes.c_longlong
+        L.str_launch_count.argtypes = [c_void_p]
+        for name in EXPORTS:
+            if name.endswith("_workspace_size"):
+                getattr(L, name).restype = c_size_t
+        _LIB = L
+    return _LIB
+
+
+def _dt(t):
+    if t.dtype == torch.bfloat16:
+        return STR_BF16
+    if t.dtype == torch.float32:
+        return STR_F32
+    raise TypeError("unsupported dtype %s" % t.dtype)
+
+
+def _p(t):
+    if t is None:
+        return c_void_p(None)
+    if isinstance(t, int):
+        return c_void_p(t)
+    assert t.is_contiguous(), "tensors must be contiguous"
+    return c_void_p(t.data_ptr())
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise StrError(rc, where)
+
+
+class Context:
+    """Owns a str_ctx for one device plus a grow-only device workspace (a torch byte tensor)."""
+
+    def __init__(self, device=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libstr needs a CUDA device; there is no CPU path")
+        self.device = device
+        torch.cuda.set_device(device)
+        self._h = c_void_p()
+        _check(lib().str_create(c_int(device), ctypes.byref(self._h)), "str_create")
+        self._ws = None
+
+    def close(self):
+        if self._h:
+            lib().str_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._h
+
+    def workspace(self, nbytes):
+        nbytes = max(int(nbytes), 256)
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda:%d" % self.device)
+        return self._ws
+
+    def check_status(self):
+        _check(lib().str_check_status(self._h, _stream()), "str_check_status")
+
+    def launch_count(self):
+        return int(lib().str_launch_count(self._h))
+
+
+def str_mamba2_prefill(ctx, x, dt, A, B, C, D=None, init_state=None, Q=0, want_final_state=False):
+    Bz, T, H, p = x.shape
+    G, n = B.shape[2], B.shape[3]
+    s = SsdShape(Bz, T, H, p, n, G, Q, _dt(x))
+    y = torch.empty_like(x)
+    fs = torch.empty((Bz, H, p, n), dtype=torch.float32, device=x.device) if want_final_state else None
+    nb = lib().str_mamba2_prefill_workspace_size(ctypes.byref(s))
+    ws = ctx.workspace(nb)
+    _check(lib().str_mamba2_prefill(ctx.handle, ctypes.byref(s), _p(x), _p(dt), _p(A), _p(B), _p(C), _p(D),
+                                    _p(init_state), _p(y), _p(fs), _p(ws), c_size_t(ws.numel()), _stream()),
+           "str_mamba2_prefill")
+    return (y, fs) if want_final_state else y
+
+
+def str_mamba_importance(ctx, B, C, dt, n_vis, n_text):
+    Bz, T, G, n = B.shape
+    H = dt.shape[2]
+    s = SsmScoreShape(Bz, T, H, n, G, _dt(B))
+    out = torch.empty((Bz, n_vis), dtype=torch.float32, device=B.device)
+    nb = lib().str_mamba_importance_workspace_size(ctypes.byref(s), c_int(n_vis), c_int(n_text))
+    ws = ctx.workspace(nb)
+    _check(lib().str_mamba_importance(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(B), _p(C), _p(dt),
+                                      _p(out), _p(ws), c_size_t(ws.numel()), _stream()), "str_mamba_importance")
+    return out
+
+
+def str_attn_importance(ctx, q, k, n_vis, n_text, softmax_scale):
+    Bz, T, Hq, d = q.shape
+    Hkv = k.shape[2]
+    s = AttnScoreShape(Bz, T, Hq, Hkv, d, _dt(q))
+    out = torch.empty((Bz, n_vis), dtype=torch.float32, device=q.device)
+    nb = lib().str_attn_importance_workspace_size(ctypes.byref(s), c_int(n_vis), c_int(n_text))
+    ws = ctx.workspace(nb)
+    _check(lib().str_attn_importance(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(q), _p(k),
+                                     c_float(softmax_scale), _p(out), _p(ws), c_size_t(ws.numel()), _stream()),
+           "str_attn_importance")
+    return out
+
+
+def str_topk_select(ctx, scores, k):
+    Bz, n_vis = scores.shape
+    out = torch.empty((Bz, k), dtype=torch.int32, device=scores.device)
+    nb = lib().str_topk_select_workspace_size(c_int(Bz), c_int(n_vis), c_int(k))
+    ws = ctx.workspace(nb)
+    _check(lib().str_topk_select(ctx.handle, c_int(Bz), c_int(n_vis), c_int(k), _p(scores), _p(out), _p(ws),
+                                 c_size_t(ws.numel()), _stream()), "str_topk_select")
+    return out
+
+
+def str_compact(ctx, hidden, positions, idx_map, kept_idx, n_text):
+    Bz, T_in, D = hidden.shape
+    k = kept_idx.shape[1]
+    n_vis = T_in - n_text
+    h_out = torch.empty((Bz, k + n_text, D), dtype=hidden.dtype, device=hidden.device)
+    p_out = torch.empty((Bz, k + n_text), dtype=torch.int32, device=hidden.device) if positions is not None else None
+    i_out = torch.empty((Bz, k + n_text), dtype=torch.int32, device=hidden.device) if idx_map is not None else None
+    _check(lib().str_compact(ctx.handle, c_int(Bz), c_int(T_in), c_int(n_vis), c_int(n_text), c_int(k), c_int(D),
+                             c_int(_dt(hidden)), _p(hidden), _p(positions), _p(idx_map), _p(kept_idx), _p(h_out),
+                             _p(p_out), _p(i_out), _stream()), "str_compact")
+    return h_out, p_out, i_out
+
+
+def str_schedule_keep_counts(alpha_bp, n0, min_keep):
+    L = len(alpha_bp)
+    a = (c_int * L)(*[int(v) for v in alpha_bp])
+    out = (c_int * L)()
+    _check(lib().str_schedule_keep_counts(a, c_int(L), c_int(n0), c_int(min_keep), out), "str_schedule_keep_counts")
+    return list(out)
+
+
+def str_sigmoid_schedule_bp(L, k, x0, a_start, a_end):
+    out = (c_int * L)()
+    _check(lib().str_sigmoid_schedule_bp(c_int(L), ctypes.c_double(k), ctypes.c_double(x0), ctypes.c_double(a_start),
+                                         ctypes.c_double(a_end), out), "str_sigmoid_schedule_bp")
+    return list(out)
+
+
+def str_gemm(ctx, a, w, residual=None):
+    M, K = a.shape
+    N = w.shape[0]
+    assert w.shape[1] == K
+    out = torch.empty((M, N), dtype=a.dtype, device=a.device)
+    nb = lib().str_gemm_workspace_size(c_int(M), c_int(N), c_int(K), c_int(_dt(a)))
+    ws = ctx.workspace(nb)
+    _check(lib().str_gemm(ctx.handle, c_int(_dt(a)), c_int(M), c_int(N), c_int(K), _p(a), _p(w), _p(residual), _p(out),
+                          _p(ws), c_size_t(ws.numel()), _stream()), "str_gemm")
+    return out
+
+
+def str_rmsnorm(ctx, x, eps=1e-5):
+    rows, D = x.shape
+    out = torch.empty_like(x)
+    _check(lib().str_rmsnorm(ctx.handle, c_int(_dt(x)), c_int(rows), c_int(D), c_float(eps), _p(x), _p(out), _stream()),
+           "str_rmsnorm")
+    return out
+
+
+def str_mamba_conv_split(ctx, zxbcdt, conv_w, conv_b, dt_bias, Bz, T, H, p, n, G):
+    W = conv_w.shape[1]
+    dev, dtp = zxbcdt.device, zxbcdt.dtype
+    x = torch.empty((Bz, T, H, p), dtype=dtp, device=dev)
+    Bm = torch.empty((Bz, T, G, n), dtype=dtp, device=dev)
+    Cm = torch.empty((Bz, T, G, n), dtype=dtp, device=dev)
+    dt = torch.empty((Bz, T, H), dtype=torch.float32, device=dev)
+    _check(lib().str_mamba_conv_split(ctx.handle, c_int(_dt(zxbcdt)), c_int(Bz), c_int(T), c_int(H), c_int(p), c_int(n),
+                                      c_int(G), c_int(W), _p(zxbcdt), _p(conv_w), _p(conv_b), _p(dt_bias), _p(x),
+                                      _p(Bm), _p(Cm), _p(dt), _stream()), "str_mamba_conv_split")
+    return x, Bm, Cm, dt
+
+
+def str_gated_rmsnorm(ctx, y, zxbcdt, d_inner, eps=1e-5):
+    rows = y.shape[0]
+    out = torch.empty_like(y)
+    _check(lib().str_gated_rmsnorm(ctx.handle, c_int(_dt(y)), c_int(rows), c_int(d_inner), c_int(zxbcdt.shape[1]),
+                                   c_float(eps), _p(y), _p(zxbcdt), _p(out), _stream()), "str_gated_rmsnorm")
+    return out
+
+
+def str_rope_split(ctx, qkv, positions, Bz, T, Hq, Hkv, d, theta):
+    dev, dtp = qkv.device, qkv.dtype
+    q = torch.empty((Bz, T, Hq, d), dtype=dtp, device=dev)
+    k = torch.empty((Bz, T, Hkv, d), dtype=dtp, device=dev)
+    v = torch.empty((Bz, T, Hkv, d), dtype=dtp, device=dev)
+    _check(lib().str_rope_split(ctx.handle, c_int(_dt(qkv)), c_int(Bz), c_int(T), c_int(Hq), c_int(Hkv), c_int(d),
+                                c_float(theta), _p(positions), _p(qkv), _p(q), _p(k), _p(v), _stream()),
+           "str_rope_split")
+    return q, k, v
+
+
+def str_attn_prefill(ctx, q, k, v, softmax_scale):
+    Bz, T, Hq, d = q.shape
+    Hkv = k.shape[2]
+    s = AttnShape(Bz, T, Hq, Hkv, d, _dt(q))
+    o = torch.empty_like(q)
+    nb = lib().str_attn_prefill_workspace_size(ctypes.byref(s))
+    ws = ctx.workspace(nb)
+    _check(lib().str_attn_prefill(ctx.handle, ctypes.byref(s), _p(q), _p(k), _p(v), c_float(softmax_scale), _p(o),
+                                  _p(ws), c_size_t(ws.numel()), _stream()), "str_attn_prefill")
+    return o
+
+
+class Stack:
+    """Device-resident parameters of a layer stack plus the str_stack_desc that describes it.
+
+    ``layers`` is the list produced by ``inputs.stack_params`` (host numpy, weights stored
+    [in_features, out_features]); they are uploaded once, transposed to the library's
+    [out_features, in_features] layout."""
+
+    def __init__(self, ctx, layers, dtype, Bz, n_vis, n_text, keep_counts, Q=0, score_every_layer=False,
+                 rope_theta=1.0e6, norm_eps=1e-5):
+        self.ctx = ctx
+        tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        dev = "cuda:%d" % ctx.device
+        self._keep = []          # keeps device tensors alive
+        arr = (Layer * len(layers))()
+        m_shape = a_shape = None
+        D = None
+        for i, (kind, prm) in enumerate(layers):
+            def up(a, t=tdt):
+                ten = torch.from_numpy(a).to(dev).to(t).contiguous()
+                self._keep.append(ten)
+                return ten.data_ptr()
+            D = prm["D"]
+            if kind == "M":
+                m_shape = prm
+                arr[i] = Layer(STR_LAYER_MAMBA, up(prm["W_in"].T.copy()), up(prm["W_out"].T.copy()),
+                               up(prm["conv_w"], torch.float32), up(prm["conv_b"], torch.float32),
+                               up(prm["dt_bias"], torch.float32), up(prm["A"], torch.float32))
+            else:
+                a_shape = prm
+                rope_theta = prm["theta"]
+                arr[i] = Layer(STR_LAYER_ATTN, up(prm["W_qkv"].T.copy()), up(prm["W_o"].T.copy()), None, None, None,
+                               None)
+        self._layers = arr
+        self._kc = (c_int * len(layers))(*[int(k) for k in keep_counts])
+        ms = m_shape or dict(H=0, p=0, n=0, G=0)
+        as_ = a_shape or dict(Hq=0, Hkv=0, d=0)
+        self.desc = StackDesc(Bz, n_vis, n_text, D, STR_BF16 if dtype == "bf16" else STR_F32,
+                              ms["H"], ms["p"], ms["n"], ms["G"], Q, 4 if m_shape else 0,
+                              as_["Hq"], as_["Hkv"], as_["d"], rope_theta, norm_eps, len(layers),
+                              ctypes.cast(arr, ctypes.POINTER(Layer)), ctypes.cast(self._kc, ctypes.POINTER(c_int)),
+                              1 if score_every_layer else 0)
+        self.tdt, self.dev = tdt, dev
+        self.Bz, self.n_vis, self.n_text, self.D = Bz, n_vis, n_text, D
+        self.keep_counts = [int(k) for k in keep_counts]
+        self.K_last = self.keep_counts[-1]
+        n_cur, self.trace_layout = n_vis, []
+        for l, K in enumerate(self.keep_counts):
+            if K < n_cur:
+                self.trace_layout.append((l, n_cur, K))
+                n_cur = K
+        self.ws_bytes = lib().str_stack_workspace_size(ctypes.byref(self.desc))
+        self.host_ws_bytes = lib().str_stack_host_workspace_size(ctypes.byref(self.desc))
+        if self.ws_bytes == 0:
+            raise StrError(-1, "str_stack_workspace_size")
+
+
+def str_stack_prefill(stack, hidden_in, want_trace=False):
+    """Runs the stack on device-resident hidden states [Bz, n_vis+n_text, D]."""
+    ctx = stack.ctx
+    T_out = stack.K_last + stack.n_text
+    out = torch.empty((stack.Bz, T_out, stack.D), dtype=stack.tdt, device=stack.dev)
+    pos = torch.empty((stack.Bz, T_out), dtype=torch.int32, device=stack.dev)
+    idx = torch.empty((stack.Bz, T_out), dtype=torch.int32, device=stack.dev)
+    kept_tr = score_tr = None
+    if want_trace and stack.trace_layout:
+        kept_tr = torch.empty(sum(stack.Bz * K for _, _, K in stack.trace_layout), dtype=torch.int32, device=stack.dev)
+        score_tr = torch.empty(sum(stack.Bz * n for _, n, _ in stack.trace_layout), dtype=torch.float32, device=stack.dev)
+    ws = ctx.workspace(stack.ws_bytes)
+    _check(lib().str_stack_prefill(ctx.handle, ctypes.byref(stack.desc), _p(hidden_in), _p(out), _p(pos), _p(idx),
+                                   _p(kept_tr), _p(score_tr), _p(ws), c_size_t(ws.numel()), _stream()),
+           "str_stack_prefill")
+    if not want_trace:
+        return out, pos, idx
+    trace, ko, so = [], 0, 0
+    for l, n_in, K in stack.trace_layout:
+        trace.append(dict(layer=l, n_in=n_in, kept=kept_tr[ko:ko + stack.Bz * K].view(stack.Bz, K),
+                          scores=score_tr[so:so + stack.Bz * n_in].view(stack.Bz, n_in)))
+        ko += stack.Bz * K
+        so += stack.Bz * n_in
+    return out, pos, idx, trace
+
+
+def str_stack_prefill_host(stack, hidden_in_host, hidden_out_host, idx_out_host):
+    """Host-buffer entry point: pinned host tensors in and out; copies are inside the call."""
+    ctx = stack.ctx
+    ws = ctx.workspace(stack.host_ws_bytes)
+    _check(lib().str_stack_prefill_host(ctx.handle, ctypes.byref(stack.desc), c_void_p(hidden_in_host.data_ptr()),
+                                        c_void_p(hidden_out_host.data_ptr()), c_void_p(idx_out_host.data_ptr()),
+                                        _p(ws), c_size_t(ws.numel()), _stream()), "str_stack_prefill_host")

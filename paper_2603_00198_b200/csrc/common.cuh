@@ -1,0 +1,50 @@
+// Shared host/device helpers for libstr (sm_100a).  Not part of the public ABI.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "str.h"
+
+struct str_ctx {
+    int device;
+    int sm_count;
+    int max_smem_optin;
+    int *status_dev;          // device status word: 0 or the first STR_ERR_* a kernel recorded
+    void *encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), or nullptr
+    long long launches;       // host-side count of kernels launched through this context
+};
+
+#define STR_CUDA_OK(call)                          \
+    do {                                           \
+        cudaError_t _e = (call);                   \
+        if (_e != cudaSuccess) return STR_ERR_CUDA; \
+    } while (0)
+
+static inline int str_launch_ok(str_ctx *ctx, int n = 1) {
+    ctx->launches += n;
+    return cudaGetLastError() == cudaSuccess ? STR_OK : STR_ERR_CUDA;
+}
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline size_t dtype_size(int dtype) { return dtype == STR_BF16 ? 2 : 4; }
+
+// ---- device: scalar load/store with widening to fp32 ----
+__device__ __forceinline__ float ldf(const float *p) { return *p; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float *p, float v) { *p = v; }
+__device__ __forceinline__ void stf(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float silu_f(float v) { return v / (1.0f + expf(-v)); }
+__device__ __forceinline__ float softplus_f(float v) { return v > 20.0f ? v : log1pf(expf(v)); }

@@ -1,0 +1,17 @@
+// Internal entry points shared between translation units of libstr (not exported).
+#pragma once
+#include "common.cuh"
+
+int str_mamba_importance_simt(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, const void *B,
+                              const void *C, const float *dt, float *scores, cudaStream_t st);
+int str_attn_importance_simt(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q,
+                             const void *k, float scale, float *scores, float *row_max, float *row_sum,
+                             cudaStream_t st);
+int str_ssd_simt(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float *dt, const float *A,
+                 const void *B, const void *C, const float *D, const float *init_state, void *y,
+                 float *final_state, cudaStream_t st);
+bool str_ssd_simt_supported(const str_ssd_shape *s);
+int str_gemm_simt(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w,
+                  const void *residual, void *out, cudaStream_t st);
+int str_attn_prefill_simt(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v,
+                          float scale, void *o, cudaStream_t st);

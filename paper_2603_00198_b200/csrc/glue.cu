@@ -1,0 +1,184 @@
+// Element-wise / row-wise block glue around the mixers: RMSNorm, the Mamba-2 pre-scan step
+// (causal depthwise conv + SiLU + split + softplus), gated RMSNorm, and RoPE + q/k/v split.
+// All HBM-bound; each activation is read once and written once.
+#include "common.cuh"
+
+namespace {
+
+__device__ __forceinline__ float block_sum(float v, float *red) {
+    v = warp_sum(v);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    const int nw = (blockDim.x + 31) >> 5;
+    for (int w = 0; w < nw; ++w) t += red[w];
+    return t;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(int D, float eps, const T *__restrict__ in, T *__restrict__ out) {
+    __shared__ float red[32];
+    const T *r = in + (size_t)blockIdx.x * D;
+    T *o = out + (size_t)blockIdx.x * D;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < D; c += blockDim.x) { const float v = ldf(r + c); ss = fmaf(v, v, ss); }
+    const float inv = rsqrtf(block_sum(ss, red) / (float)D + eps);
+    for (int c = threadIdx.x; c < D; c += blockDim.x) stf(o + c, ldf(r + c) * inv);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+gated_rmsnorm_kernel(int d_inner, int ld_z, float eps, const T *__restrict__ y, const T *__restrict__ z,
+                     T *__restrict__ out) {
+    __shared__ float red[32];
+    const T *yr = y + (size_t)blockIdx.x * d_inner;
+    const T *zr = z + (size_t)blockIdx.x * ld_z;
+    T *o = out + (size_t)blockIdx.x * d_inner;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d_inner; c += blockDim.x) {
+        const float v = ldf(yr + c) * silu_f(ldf(zr + c));
+        ss = fmaf(v, v, ss);
+    }
+    const float inv = rsqrtf(block_sum(ss, red) / (float)d_inner + eps);
+    for (int c = threadIdx.x; c < d_inner; c += blockDim.x)
+        stf(o + c, ldf(yr + c) * silu_f(ldf(zr + c)) * inv);
+}
+
+// One thread per (token, conv channel); consecutive threads walk consecutive channels.
+template <typename T>
+__global__ void __launch_bounds__(256)
+mamba_conv_split_kernel(int Tlen, int H, int p, int n, int G, int W, const T *__restrict__ zxbcdt,
+                        const float *__restrict__ conv_w, const float *__restrict__ conv_b,
+                        const float *__restrict__ dt_bias, T *__restrict__ x_out, T *__restrict__ B_out,
+                        T *__restrict__ C_out, float *__restrict__ dt_out) {
+    const int d_inner = H * p, gn = G * n;
+    const int conv_dim = d_inner + 2 * gn;
+    const int ld = 2 * d_inner + 2 * gn + H;
+    const int cols = conv_dim + H;                       // conv channels, then the H dt columns
+    const size_t row = blockIdx.y;                       // b * Tlen + t
+    const int t = (int)(row % Tlen);
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= cols) return;
+    const T *base = zxbcdt + row * ld;
+    if (c >= conv_dim) {
+        const int h = c - conv_dim;
+        dt_out[row * H + h] = softplus_f(ldf(base + d_inner + conv_dim + h) + dt_bias[h]);
+        return;
+    }
+    float acc = conv_b[c];
+    for (int j = 0; j < W; ++j) {
+        const int back = W - 1 - j;                      // tap j reads token t - (W-1) + j
+        if (t - back >= 0) acc = fmaf(conv_w[(size_t)c * W + j], ldf(base - (size_t)back * ld + d_inner + c), acc);
+    }
+    const float v = silu_f(acc);
+    if (c < d_inner) stf(x_out + row * d_inner + c, v);
+    else if (c < d_inner + gn) stf(B_out + row * gn + (c - d_inner), v);
+    else stf(C_out + row * gn + (c - d_inner - gn), v);
+}
+
+// One thread per (token, head, pair index i < d/2) for q and k; v columns are copied.
+template <typename T>
+__global__ void __launch_bounds__(256)
+rope_split_kernel(int Hq, int Hkv, int d, float log2_theta, const int32_t *__restrict__ positions,
+                  const T *__restrict__ qkv, T *__restrict__ q_out, T *__restrict__ k_out, T *__restrict__ v_out) {
+    const int half = d / 2;
+    const int ld = (Hq + 2 * Hkv) * d;
+    const size_t row = blockIdx.y;
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    const int n_rot = (Hq + Hkv) * half;
+    const int n_v = Hkv * d;
+    const T *base = qkv + row * ld;
+    if (e < n_rot) {
+        const int head = e / half, i = e % half;
+        // angle in fp64, reduced to [0, 2pi) before the fp32 sincos: positions reach tens of thousands
+        const double inv_freq = exp2(-2.0 * (double)i / (double)d * (double)log2_theta);
+        double ang = (double)positions[row] * inv_freq;
+        ang -= 6.283185307179586476925 * floor(ang * 0.15915494309189533576888);
+        float sn, cs;
+        sincosf((float)ang, &sn, &cs);
+        const float a = ldf(base + head * d + i), b = ldf(base + head * d + half + i);
+        T *dst = head < Hq ? q_out + (row * Hq + head) * d : k_out + (row * Hkv + (head - Hq)) * d;
+        stf(dst + i, a * cs - b * sn);
+        stf(dst + half + i, b * cs + a * sn);
+    } else if (e < n_rot + n_v) {
+        const int c = e - n_rot;
+        v_out[row * n_v + c] = base[(Hq + Hkv) * d + c];
+    }
+}
+
+}  // namespace
+
+#define STR_DTYPE_OK(dt) ((dt) == STR_F32 || (dt) == STR_BF16)
+
+extern "C" int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, const void *in, void *out,
+                           void *stream) {
+    if (!ctx || !in || !out || rows < 0 || D <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
+    if (rows == 0) return STR_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == STR_BF16)
+        rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>(D, eps, (const __nv_bfloat16 *)in, (__nv_bfloat16 *)out);
+    else
+        rmsnorm_kernel<float><<<rows, 256, 0, st>>>(D, eps, (const float *)in, (float *)out);
+    return str_launch_ok(ctx);
+}
+
+extern "C" int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps,
+                                 const void *y, const void *z, void *out, void *stream) {
+    if (!ctx || !y || !z || !out || rows < 0 || d_inner <= 0 || ld_z < d_inner || !STR_DTYPE_OK(dtype))
+        return STR_ERR_INVALID_ARG;
+    if (rows == 0) return STR_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == STR_BF16)
+        gated_rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const __nv_bfloat16 *)y,
+                                                                 (const __nv_bfloat16 *)z, (__nv_bfloat16 *)out);
+    else
+        gated_rmsnorm_kernel<float><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const float *)y, (const float *)z,
+                                                         (float *)out);
+    return str_launch_ok(ctx);
+}
+
+extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, int n, int G, int W,
+                                    const void *zxbcdt, const float *conv_w, const float *conv_b,
+                                    const float *dt_bias, void *x_out, void *B_out, void *C_out, float *dt_out,
+                                    void *stream) {
+    if (!ctx || !zxbcdt || !conv_w || !conv_b || !dt_bias || !x_out || !B_out || !C_out || !dt_out || Bz <= 0 ||
+        T <= 0 || H <= 0 || p <= 0 || n <= 0 || G <= 0 || W <= 0 || !STR_DTYPE_OK(dtype))
+        return STR_ERR_INVALID_ARG;
+    if ((long long)Bz * T > 2147483647LL) return STR_ERR_UNSUPPORTED_SHAPE;
+    const int cols = H * p + 2 * G * n + H;
+    dim3 grid(ceil_div(cols, 256), Bz * T);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == STR_BF16)
+        mamba_conv_split_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
+            T, H, p, n, G, W, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
+            (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out);
+    else
+        mamba_conv_split_kernel<float><<<grid, 256, 0, st>>>(T, H, p, n, G, W, (const float *)zxbcdt, conv_w, conv_b,
+                                                            dt_bias, (float *)x_out, (float *)B_out, (float *)C_out,
+                                                            dt_out);
+    return str_launch_ok(ctx);
+}
+
+extern "C" int str_rope_split(str_ctx *ctx, int dtype, int Bz, int T, int Hq, int Hkv, int d, float theta,
+                              const int32_t *positions, const void *qkv, void *q_out, void *k_out, void *v_out,
+                              void *stream) {
+    if (!ctx || !positions || !qkv || !q_out || !k_out || !v_out || Bz <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 ||
+        d <= 0 || (d & 1) || theta <= 0.f || !STR_DTYPE_OK(dtype))
+        return STR_ERR_INVALID_ARG;
+    if ((long long)Bz * T > 2147483647LL) return STR_ERR_UNSUPPORTED_SHAPE;
+    const int work = (Hq + Hkv) * (d / 2) + Hkv * d;
+    dim3 grid(ceil_div(work, 256), Bz * T);
+    cudaStream_t st = (cudaStream_t)stream;
+    const float l2t = log2f(theta);
+    if (dtype == STR_BF16)
+        rope_split_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(Hq, Hkv, d, l2t, positions, (const __nv_bfloat16 *)qkv,
+                                                              (__nv_bfloat16 *)q_out, (__nv_bfloat16 *)k_out,
+                                                              (__nv_bfloat16 *)v_out);
+    else
+        rope_split_kernel<float><<<grid, 256, 0, st>>>(Hq, Hkv, d, l2t, positions, (const float *)qkv, (float *)q_out,
+                                                      (float *)k_out, (float *)v_out);
+    return str_launch_ok(ctx);
+}

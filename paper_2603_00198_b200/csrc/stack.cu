@@ -1,0 +1,239 @@
+// str_stack_prefill: token-reduced prefill of a hybrid Mamba-2 / attention layer stack.
+// Host loop over layers; every step is a kernel of this library enqueued on one stream, with no
+// device->host synchronisation in between (the keep counts are known in advance because the
+// schedule does not depend on the input).
+#include <string.h>
+
+#include "dispatch.cuh"
+
+namespace {
+
+__global__ void iota_rows_kernel(int rows, int T, int32_t *a, int32_t *b) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < rows) { a[i] = i % T; b[i] = i % T; }
+}
+
+struct Regions {
+    size_t hidden[2], normed, proj, bufA, bufB, bufC, bufY, dt, pos[2], idx[2], scores, kept, sub, total;
+    size_t sub_bytes;
+};
+
+inline size_t imax(size_t a, size_t b) { return a > b ? a : b; }
+
+bool desc_ok(const str_stack_desc *d) {
+    if (!d || d->Bz <= 0 || d->n_vis < 0 || d->n_text <= 0 || d->D <= 0 || d->n_layers <= 0 || !d->layers ||
+        !d->keep_counts || (d->dtype != STR_F32 && d->dtype != STR_BF16))
+        return false;
+    bool has_m = false, has_a = false;
+    int n_cur = d->n_vis;
+    for (int l = 0; l < d->n_layers; ++l) {
+        const str_layer &L = d->layers[l];
+        if (L.kind == STR_LAYER_MAMBA) {
+            has_m = true;
+            if (!L.w_in || !L.w_out || !L.conv_w || !L.conv_b || !L.dt_bias || !L.A) return false;
+        } else if (L.kind == STR_LAYER_ATTN) {
+            has_a = true;
+            if (!L.w_in || !L.w_out) return false;
+        } else {
+            return false;
+        }
+        if (d->keep_counts[l] < 0 || d->keep_counts[l] > n_cur) return false;
+        n_cur = d->keep_counts[l];
+    }
+    if (has_m && (d->H <= 0 || d->p <= 0 || d->n <= 0 || d->G <= 0 || d->H % d->G != 0 || d->conv_width <= 0))
+        return false;
+    if (has_a && (d->Hq <= 0 || d->Hkv <= 0 || d->Hq % d->Hkv != 0 || d->d <= 0 || (d->d & 1) || d->rope_theta <= 0.f))
+        return false;
+    return true;
+}
+
+Regions plan(const str_stack_desc *d) {
+    Regions r;
+    const size_t e = dtype_size(d->dtype);
+    const size_t T0 = (size_t)d->n_vis + d->n_text, R = (size_t)d->Bz * T0;
+    bool has_m = false, has_a = false;
+    for (int l = 0; l < d->n_layers; ++l) (d->layers[l].kind == STR_LAYER_MAMBA ? has_m : has_a) = true;
+    const size_t d_inner = has_m ? (size_t)d->H * d->p : 0, gn = has_m ? (size_t)d->G * d->n : 0;
+    const size_t dip = has_m ? 2 * d_inner + 2 * gn + d->H : 0;
+    const size_t qd = has_a ? (size_t)d->Hq * d->d : 0, kd = has_a ? (size_t)d->Hkv * d->d : 0;
+    const size_t dqkv = qd + 2 * kd;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
+    r.hidden[0] = take(R * d->D * e);
+    r.hidden[1] = take(R * d->D * e);
+    r.normed = take(R * d->D * e);
+    r.proj = take(R * imax(dip, dqkv) * e);
+    r.bufA = take(R * imax(d_inner, qd) * e);
+    r.bufB = take(R * imax(gn, kd) * e);
+    r.bufC = take(R * imax(gn, kd) * e);
+    r.bufY = take(R * imax(d_inner, qd) * e);
+    r.dt = take(R * (has_m ? d->H : 1) * sizeof(float));
+    for (int i = 0; i < 2; ++i) { r.pos[i] = take(R * 4); r.idx[i] = take(R * 4); }
+    r.scores = take((size_t)d->Bz * imax(d->n_vis, 1) * 4);
+    r.kept = take((size_t)d->Bz * imax(d->n_vis, 1) * 4);
+    size_t sub = 0;
+    if (has_m) {
+        str_ssd_shape s = {d->Bz, (int)T0, d->H, d->p, d->n, d->G, d->Q, d->dtype};
+        sub = imax(sub, str_mamba2_prefill_workspace_size(&s));
+        str_ssm_score_shape ss = {d->Bz, (int)T0, d->H, d->n, d->G, d->dtype};
+        sub = imax(sub, str_mamba_importance_workspace_size(&ss, d->n_vis, d->n_text));
+        sub = imax(sub, str_gemm_workspace_size((int)R, (int)dip, d->D, d->dtype));
+    }
+    if (has_a) {
+        str_attn_score_shape as = {d->Bz, (int)T0, d->Hq, d->Hkv, d->d, d->dtype};
+        sub = imax(sub, str_attn_importance_workspace_size(&as, d->n_vis, d->n_text));
+        str_attn_shape at = {d->Bz, (int)T0, d->Hq, d->Hkv, d->d, d->dtype};
+        sub = imax(sub, str_attn_prefill_workspace_size(&at));
+        sub = imax(sub, str_gemm_workspace_size((int)R, (int)dqkv, d->D, d->dtype));
+    }
+    sub = imax(sub, str_topk_select_workspace_size(d->Bz, d->n_vis, d->n_vis));
+    r.sub_bytes = align_up(sub, 256);
+    r.sub = take(r.sub_bytes);
+    r.total = off;
+    return r;
+}
+
+}  // namespace
+
+extern "C" size_t str_stack_workspace_size(const str_stack_desc *d) {
+    if (!desc_ok(d)) return 0;
+    return plan(d).total;
+}
+
+#define STR_TRY(call)              \
+    do {                           \
+        int _rc = (call);          \
+        if (_rc != STR_OK) return _rc; \
+    } while (0)
+
+extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in, void *hidden_out,
+                                 int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace,
+                                 float *scores_trace, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!ctx || !desc_ok(d) || !hidden_in || !hidden_out || !workspace) return STR_ERR_INVALID_ARG;
+    if (((uintptr_t)workspace & 255) != 0) return STR_ERR_INVALID_ARG;
+    const Regions r = plan(d);
+    if (workspace_bytes < r.total) return STR_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = (char *)workspace;
+    const int Bz = d->Bz, M = d->n_text, D = d->D, dtype = d->dtype;
+    void *hid[2] = {ws + r.hidden[0], ws + r.hidden[1]};
+    int32_t *pos[2] = {(int32_t *)(ws + r.pos[0]), (int32_t *)(ws + r.pos[1])};
+    int32_t *idx[2] = {(int32_t *)(ws + r.idx[0]), (int32_t *)(ws + r.idx[1])};
+    void *normed = ws + r.normed, *proj = ws + r.proj, *bufA = ws + r.bufA, *bufB = ws + r.bufB;
+    void *bufC = ws + r.bufC, *bufY = ws + r.bufY, *sub = ws + r.sub;
+    float *dt = (float *)(ws + r.dt);
+    float *scores_int = (float *)(ws + r.scores);
+    int32_t *kept_int = (int32_t *)(ws + r.kept);
+
+    int n_cur = d->n_vis;
+    {
+        const int rows = Bz * (n_cur + M);
+        iota_rows_kernel<<<ceil_div(rows, 256), 256, 0, st>>>(rows, n_cur + M, pos[0], idx[0]);
+        STR_TRY(str_launch_ok(ctx));
+    }
+    const void *cur = hidden_in;
+    int hsel = 0;      // next free hidden buffer
+    int psel = 0;      // current positions / idx buffer
+    size_t kept_off = 0, score_off = 0;
+
+    for (int l = 0; l < d->n_layers; ++l) {
+        const str_layer &L = d->layers[l];
+        const int T = n_cur + M, rows = Bz * T;
+        const int K = d->keep_counts[l];
+        const bool reduce = K < n_cur;
+        const bool last = l == d->n_layers - 1;
+        const bool want_score = reduce || d->score_every_layer;
+        float *scores = (reduce && scores_trace) ? scores_trace + score_off : scores_int;
+        int32_t *kept = (reduce && kept_trace) ? kept_trace + kept_off : kept_int;
+        void *mix_out = (last && !reduce) ? hidden_out : hid[hsel];
+
+        STR_TRY(str_rmsnorm(ctx, dtype, rows, D, d->norm_eps, cur, normed, stream));
+        if (L.kind == STR_LAYER_MAMBA) {
+            const int d_inner = d->H * d->p, gn = d->G * d->n, dip = 2 * d_inner + 2 * gn + d->H;
+            STR_TRY(str_gemm(ctx, dtype, rows, dip, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+            STR_TRY(str_mamba_conv_split(ctx, dtype, Bz, T, d->H, d->p, d->n, d->G, d->conv_width, proj, L.conv_w,
+                                         L.conv_b, L.dt_bias, bufA, bufB, bufC, dt, stream));
+            str_ssd_shape s = {Bz, T, d->H, d->p, d->n, d->G, d->Q, dtype};
+            STR_TRY(str_mamba2_prefill(ctx, &s, bufA, dt, L.A, bufB, bufC, nullptr, nullptr, bufY, nullptr, sub,
+                                       r.sub_bytes, stream));
+            if (want_score && n_cur > 0) {
+                str_ssm_score_shape ss = {Bz, T, d->H, d->n, d->G, dtype};
+                STR_TRY(str_mamba_importance(ctx, &ss, n_cur, M, bufB, bufC, dt, scores, sub, r.sub_bytes, stream));
+            }
+            STR_TRY(str_gated_rmsnorm(ctx, dtype, rows, d_inner, dip, d->norm_eps, bufY, proj, bufA, stream));
+            STR_TRY(str_gemm(ctx, dtype, rows, D, d_inner, bufA, L.w_out, cur, mix_out, sub, r.sub_bytes, stream));
+        } else {
+            const int qd = d->Hq * d->d, kd = d->Hkv * d->d;
+            STR_TRY(str_gemm(ctx, dtype, rows, qd + 2 * kd, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+            STR_TRY(str_rope_split(ctx, dtype, Bz, T, d->Hq, d->Hkv, d->d, d->rope_theta, pos[psel], proj, bufA, bufB,
+                                   bufC, stream));
+            str_attn_shape as = {Bz, T, d->Hq, d->Hkv, d->d, dtype};
+            const float scale = 1.0f / sqrtf((float)d->d);
+            STR_TRY(str_attn_prefill(ctx, &as, bufA, bufB, bufC, scale, bufY, sub, r.sub_bytes, stream));
+            if (want_score && n_cur > 0) {
+                str_attn_score_shape ss = {Bz, T, d->Hq, d->Hkv, d->d, dtype};
+                STR_TRY(str_attn_importance(ctx, &ss, n_cur, M, bufA, bufB, scale, scores, sub, r.sub_bytes, stream));
+            }
+            STR_TRY(str_gemm(ctx, dtype, rows, D, qd, bufY, L.w_out, cur, mix_out, sub, r.sub_bytes, stream));
+        }
+        if (reduce) {
+            STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));
+            void *dst = last ? hidden_out : hid[1 - hsel];
+            int32_t *pdst = (last && positions_out) ? positions_out : pos[1 - psel];
+            int32_t *idst = (last && idx_map_out) ? idx_map_out : idx[1 - psel];
+            STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, mix_out, pos[psel], idx[psel], kept, dst, pdst,
+                                idst, stream));
+            cur = dst;
+            hsel = (dst == hid[0]) ? 1 : 0;
+            psel = 1 - psel;
+            kept_off += (size_t)Bz * K;
+            score_off += (size_t)Bz * n_cur;
+            n_cur = K;
+            if (last) {
+                // positions/idx already written where the caller wants them
+                return STR_OK;
+            }
+        } else {
+            cur = mix_out;
+            hsel = 1 - hsel;
+        }
+    }
+    // last layer did not reduce: hidden_out holds the result; hand back the carried ids
+    const size_t nb = (size_t)Bz * (n_cur + M) * 4;
+    if (positions_out) STR_CUDA_OK(cudaMemcpyAsync(positions_out, pos[psel], nb, cudaMemcpyDeviceToDevice, st));
+    if (idx_map_out) STR_CUDA_OK(cudaMemcpyAsync(idx_map_out, idx[psel], nb, cudaMemcpyDeviceToDevice, st));
+    return STR_OK;
+}
+
+extern "C" size_t str_stack_host_workspace_size(const str_stack_desc *d) {
+    if (!desc_ok(d)) return 0;
+    const size_t e = dtype_size(d->dtype);
+    const size_t Rin = (size_t)d->Bz * ((size_t)d->n_vis + d->n_text);
+    const size_t Rout = (size_t)d->Bz * ((size_t)d->keep_counts[d->n_layers - 1] + d->n_text);
+    return align_up(Rin * d->D * e, 256) + align_up(Rout * d->D * e, 256) + 2 * align_up(Rout * 4, 256) + plan(d).total;
+}
+
+extern "C" int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in_host,
+                                      void *hidden_out_host, int32_t *idx_map_out_host, void *workspace,
+                                      size_t workspace_bytes, void *stream) {
+    if (!ctx || !desc_ok(d) || !hidden_in_host || !hidden_out_host || !workspace) return STR_ERR_INVALID_ARG;
+    if (workspace_bytes < str_stack_host_workspace_size(d)) return STR_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t e = dtype_size(d->dtype);
+    const size_t Rin = (size_t)d->Bz * ((size_t)d->n_vis + d->n_text);
+    const size_t Rout = (size_t)d->Bz * ((size_t)d->keep_counts[d->n_layers - 1] + d->n_text);
+    char *ws = (char *)workspace;
+    void *in_dev = ws;  ws += align_up(Rin * d->D * e, 256);
+    void *out_dev = ws; ws += align_up(Rout * d->D * e, 256);
+    int32_t *pos_dev = (int32_t *)ws; ws += align_up(Rout * 4, 256);
+    int32_t *idx_dev = (int32_t *)ws; ws += align_up(Rout * 4, 256);
+    STR_CUDA_OK(cudaMemcpyAsync(in_dev, hidden_in_host, Rin * d->D * e, cudaMemcpyHostToDevice, st));
+    int rc = str_stack_prefill(ctx, d, in_dev, out_dev, pos_dev, idx_dev, nullptr, nullptr, ws,
+                               workspace_bytes - (size_t)(ws - (char *)workspace), stream);
+    if (rc != STR_OK) return rc;
+    STR_CUDA_OK(cudaMemcpyAsync(hidden_out_host, out_dev, Rout * d->D * e, cudaMemcpyDeviceToHost, st));
+    if (idx_map_out_host)
+        STR_CUDA_OK(cudaMemcpyAsync(idx_map_out_host, idx_dev, Rout * 4, cudaMemcpyDeviceToHost, st));
+    STR_CUDA_OK(cudaStreamSynchronize(st));
+    return STR_OK;
+}

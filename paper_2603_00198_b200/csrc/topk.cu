@@ -1,0 +1,134 @@
+// str_topk_select: per-sequence radix select of the k largest fp32 scores, emitted in
+// ascending index order (temporal order preserved; ties go to the lower index).
+//
+// One CTA per sequence.  Four 8-bit MSB-first passes over the order-preserving integer image
+// of the scores narrow down the k-th largest key; per-warp private histograms with
+// warp-aggregated increments keep shared-memory atomics uncontended even when every score
+// shares its top byte.  A last ordered pass emits the survivors: each warp owns a contiguous
+// index segment, so a single block-level exclusive scan of 32 warp counts orders the output.
+#include "common.cuh"
+
+namespace {
+
+constexpr int TOPK_THREADS = 1024;
+constexpr int TOPK_WARPS = TOPK_THREADS / 32;
+
+__device__ __forceinline__ uint32_t score_key(float s) {
+    const uint32_t u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);   // larger float <=> larger key
+}
+
+__global__ void __launch_bounds__(TOPK_THREADS)
+topk_select_kernel(int n, int k, const float *__restrict__ scores, int32_t *__restrict__ kept) {
+    __shared__ uint32_t hist[TOPK_WARPS][256];
+    __shared__ uint32_t total[256];
+    __shared__ uint32_t sh_prefix, sh_need;
+    __shared__ uint32_t warp_gt[TOPK_WARPS], warp_eq[TOPK_WARPS];
+
+    const float *s = scores + (size_t)blockIdx.x * n;
+    int32_t *out = kept + (size_t)blockIdx.x * k;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (k <= 0) return;
+
+    uint32_t prefix = 0, mask = 0, need = (uint32_t)k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = tid; i < TOPK_WARPS * 256; i += TOPK_THREADS) (&hist[0][0])[i] = 0;
+        __syncthreads();
+        const int n_round = (n + 31) & ~31;
+        for (int i = tid; i < n_round; i += TOPK_THREADS) {
+            const bool in = i < n;
+            const uint32_t key = in ? score_key(s[i]) : 0u;
+            const bool live = in && ((key & mask) == prefix);
+            const uint32_t bin = (key >> shift) & 255u;
+            // warp-aggregated increment: lanes with the same bin elect one leader
+            const uint32_t live_mask = __ballot_sync(0xffffffffu, live);
+            if (live) {
+                const uint32_t peers = __match_any_sync(live_mask, bin);
+                if (lane == __ffs(peers) - 1) hist[warp][bin] += __popc(peers);
+            }
+            __syncwarp();
+        }
+        __syncthreads();
+        if (tid < 256) {
+            uint32_t t = 0;
+#pragma unroll 8
+            for (int w = 0; w < TOPK_WARPS; ++w) t += hist[w][tid];
+            total[tid] = t;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane L owns bins 255-8L .. 248-8L (descending); find the bin holding the need-th largest
+            uint32_t c[8], lane_sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { c[j] = total[255 - 8 * lane - j]; lane_sum += c[j]; }
+            uint32_t incl = lane_sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const uint32_t before = incl - lane_sum;
+            if (before < need && need <= incl) {
+                uint32_t run = before;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (run < need && need <= run + c[j]) {
+                        sh_prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
+                        sh_need = need - run;
+                    }
+                    run += c[j];
+                }
+            }
+        }
+        __syncthreads();
+        prefix = sh_prefix;
+        need = sh_need;
+        mask |= 255u << shift;
+        __syncthreads();
+    }
+    // prefix = key of the k-th largest score; every key > prefix is kept, plus the first `need`
+    // (in index order) of the keys == prefix.
+    const int seg = (((n + TOPK_WARPS - 1) / TOPK_WARPS) + 31) & ~31;
+    const int lo = warp * seg, hi = min(n, lo + seg);
+    uint32_t gt = 0, eq = 0;
+    for (int i = lo + lane; i < lo + seg; i += 32) {
+        const bool in = i < hi;
+        const uint32_t key = in ? score_key(s[i]) : 0u;
+        gt += __popc(__ballot_sync(0xffffffffu, in && key > prefix));
+        eq += __popc(__ballot_sync(0xffffffffu, in && key == prefix));
+    }
+    if (lane == 0) { warp_gt[warp] = gt; warp_eq[warp] = eq; }
+    __syncthreads();
+    uint32_t gt_before = 0, eq_before = 0;
+    for (int w = 0; w < warp; ++w) { gt_before += warp_gt[w]; eq_before += warp_eq[w]; }
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    for (int i = lo + lane; i < lo + seg; i += 32) {
+        const bool in = i < hi;
+        const uint32_t key = in ? score_key(s[i]) : 0u;
+        const bool is_gt = in && key > prefix, is_eq = in && key == prefix;
+        const uint32_t gt_b = __ballot_sync(0xffffffffu, is_gt);
+        const uint32_t eq_b = __ballot_sync(0xffffffffu, is_eq);
+        const uint32_t eq_rank = eq_before + __popc(eq_b & lt_mask);
+        const bool take = is_gt || (is_eq && eq_rank < need);
+        const uint32_t take_b = __ballot_sync(0xffffffffu, take);
+        if (take) {
+            const uint32_t pos = gt_before + min(eq_before, need) + __popc(take_b & lt_mask);
+            out[pos] = i;
+        }
+        gt_before += __popc(gt_b);
+        eq_before += __popc(eq_b);
+    }
+}
+
+}  // namespace
+
+extern "C" size_t str_topk_select_workspace_size(int, int, int) { return 0; }
+
+extern "C" int str_topk_select(str_ctx *ctx, int Bz, int n_vis, int k, const float *scores,
+                               int32_t *kept_idx_out, void *, size_t, void *stream) {
+    if (!ctx || Bz <= 0 || n_vis < 0 || k < 0 || k > n_vis) return STR_ERR_INVALID_ARG;
+    if (k == 0) return STR_OK;
+    if (!scores || !kept_idx_out) return STR_ERR_INVALID_ARG;
+    topk_select_kernel<<<Bz, TOPK_THREADS, 0, (cudaStream_t)stream>>>(n_vis, k, scores, kept_idx_out);
+    return str_launch_ok(ctx);
+}

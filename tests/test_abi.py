@@ -1,0 +1,63 @@
+"""CPU checks of the C-ABI boundary: the library builds, loads, and exports every symbol that
+include/str.h declares; the host-only schedule helpers agree with the oracle."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import oracle
+from paper_2603_00198_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def libstr():
+    build.build()
+    return binding.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "str.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(str_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(libstr):
+    names = _declared()
+    assert len(names) >= 25
+    for n in names:
+        assert hasattr(libstr, n), n
+    assert set(binding.EXPORTS) <= set(names)
+
+
+def test_error_strings(libstr):
+    assert libstr.str_strerror(0) == b"ok"
+    for code in (-1, -2, -3, -4, -5):
+        assert len(libstr.str_strerror(code)) > 3
+
+
+def test_keep_counts_match_oracle(libstr):
+    cases = [([10000] * 4 + [5000] * 4 + [2500] * 4, 32768, 256), ([10000, 1000, 1000], 16384, 256),
+             ([5000, 100, 9000], 1000, 144), ([10000, 2500], 100, 144), ([10000, 3162, 1000], 65536, 256),
+             ([7071, 7071, 5000], 16384, 0)]
+    for alpha, n0, mk in cases:
+        assert binding.str_schedule_keep_counts(alpha, n0, mk) == oracle.schedule_keep_counts(alpha, n0, mk)
+    with pytest.raises(binding.StrError):
+        binding.str_schedule_keep_counts([10001], 10, 0)
+
+
+def test_sigmoid_schedule_matches_oracle(libstr):
+    for x0 in (0.11, 0.24, 0.41):
+        bp = binding.str_sigmoid_schedule_bp(62, 20.0, x0, 1.0, 0.125)
+        ref = oracle.sigmoid_schedule(62, 20.0, x0, 1.0, 0.125)
+        assert all(abs(b - r * 10000) <= 0.5 + 1e-6 for b, r in zip(bp, ref))
+        assert bp == sorted(bp, reverse=True)
+
+
+def test_argument_validation_needs_no_gpu(libstr):
+    # null context / null pointers are rejected on the host before anything touches CUDA
+    assert libstr.str_topk_select(None, 1, 8, 4, None, None, None, ctypes.c_size_t(0), None) == -1
+    assert libstr.str_compact(None, 1, 8, 6, 2, 3, 16, 1, None, None, None, None, None, None, None, None) == -1
+    assert libstr.str_destroy(None) == -1

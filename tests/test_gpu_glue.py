@@ -1,0 +1,94 @@
+"""GPU parity for the block glue (GEMM, norms, conv/split, RoPE, causal GQA attention) against the
+oracle's textbook definitions."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2603_00198_b200 import binding, inputs
+from util_gpu import dev, host, max_rel_err
+
+pytestmark = pytest.mark.gpu
+TOL = {"bf16": 2e-2, "f32": 2e-4}
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.check_status()
+    c.close()
+
+
+@pytest.mark.parametrize("dtype,M,N,K", [("bf16", 300, 200, 256), ("f32", 65, 130, 70), ("bf16", 1056, 1184, 256),
+                                         ("bf16", 4224, 1024, 4096), ("bf16", 128, 18560, 4096), ("f32", 1, 7, 3),
+                                         ("bf16", 257, 136, 8192)])
+def test_gemm_with_residual(ctx, dtype, M, N, K):
+    g = inputs.rng(51, M + N + K)
+    a = inputs.to_grid(g.standard_normal((M, K), dtype=np.float32), dtype)
+    w = inputs.to_grid(g.standard_normal((N, K), dtype=np.float32) / np.sqrt(K), dtype)
+    r = inputs.to_grid(g.standard_normal((M, N), dtype=np.float32), dtype)
+    ref = a.astype(np.float64) @ w.astype(np.float64).T
+    got = host(binding.str_gemm(ctx, dev(a, dtype), dev(w, dtype)))
+    assert max_rel_err(got, ref) <= TOL[dtype]
+    got = host(binding.str_gemm(ctx, dev(a, dtype), dev(w, dtype), residual=dev(r, dtype)))
+    assert max_rel_err(got, ref + r) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype,rows,D", [("bf16", 100, 4096), ("f32", 33, 256), ("bf16", 5, 40)])
+def test_rmsnorm(ctx, dtype, rows, D):
+    u = inputs.hidden_inputs(52, rows, D, dtype)[0] * 3.0
+    u = inputs.to_grid(u, dtype)
+    got = host(binding.str_rmsnorm(ctx, dev(u, dtype)))
+    assert max_rel_err(got, oracle.rmsnorm(u)) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype,Bz,T,H,p,n,G", [("bf16", 1, 300, 16, 64, 128, 2), ("f32", 2, 70, 8, 32, 16, 1)])
+def test_conv_split_and_gated_norm(ctx, dtype, Bz, T, H, p, n, G):
+    d_inner, gn = H * p, G * n
+    ld = 2 * d_inner + 2 * gn + H
+    g = inputs.rng(53, T)
+    z = inputs.to_grid(g.standard_normal((Bz * T, ld), dtype=np.float32), dtype)
+    cw = g.uniform(-0.5, 0.5, size=(d_inner + 2 * gn, 4)).astype(np.float32)
+    cb = g.uniform(-0.1, 0.1, size=(d_inner + 2 * gn,)).astype(np.float32)
+    dtb = inputs.softplus_inverse(g.uniform(1e-3, 1e-1, size=H)).astype(np.float32)
+    x, Bm, Cm, dt = binding.str_mamba_conv_split(ctx, dev(z, dtype), dev(cw), dev(cb), dev(dtb), Bz, T, H, p, n, G)
+    for b in range(Bz):
+        zz = z[b * T:(b + 1) * T].astype(np.float64)
+        ref = oracle.causal_conv1d_silu(zz[:, d_inner:2 * d_inner + 2 * gn], cw, cb)     # per sequence: no leak across b
+        assert max_rel_err(host(x)[b].reshape(T, d_inner), ref[:, :d_inner]) <= TOL[dtype]
+        assert max_rel_err(host(Bm)[b].reshape(T, gn), ref[:, d_inner:d_inner + gn]) <= TOL[dtype]
+        assert max_rel_err(host(Cm)[b].reshape(T, gn), ref[:, d_inner + gn:]) <= TOL[dtype]
+        rdt = oracle.softplus(zz[:, 2 * d_inner + 2 * gn:] + dtb[None, :])
+        assert np.abs(host(dt)[b] / rdt - 1).max() <= 1e-5
+    y = inputs.to_grid(g.standard_normal((Bz * T, d_inner), dtype=np.float32), dtype)
+    got = host(binding.str_gated_rmsnorm(ctx, dev(y, dtype), dev(z, dtype), d_inner))
+    ref = oracle.rmsnorm(y.astype(np.float64) * oracle.silu(z[:, :d_inner].astype(np.float64)))
+    assert max_rel_err(got, ref) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype,Bz,T,Hq,Hkv,d", [("bf16", 1, 200, 8, 2, 128), ("f32", 2, 50, 4, 4, 32)])
+def test_rope_split(ctx, dtype, Bz, T, Hq, Hkv, d):
+    g = inputs.rng(54, T)
+    qkv = inputs.to_grid(g.standard_normal((Bz * T, (Hq + 2 * Hkv) * d), dtype=np.float32), dtype)
+    pos = np.sort(g.choice(70000, size=(Bz, T)), axis=1).astype(np.int32)      # carried original positions
+    q, k, v = binding.str_rope_split(ctx, dev(qkv, dtype), dev(pos), Bz, T, Hq, Hkv, d, 1.0e6)
+    for b in range(Bz):
+        blk = qkv[b * T:(b + 1) * T].astype(np.float64)
+        rq = oracle.rope(blk[:, :Hq * d].reshape(T, Hq, d), pos[b], 1.0e6)
+        rk = oracle.rope(blk[:, Hq * d:(Hq + Hkv) * d].reshape(T, Hkv, d), pos[b], 1.0e6)
+        tol = 1e-2 if dtype == "bf16" else 1e-5
+        assert max_rel_err(host(q)[b], rq) <= tol and max_rel_err(host(k)[b], rk) <= tol
+        assert np.array_equal(host(v)[b].reshape(T, -1), blk[:, (Hq + Hkv) * d:])
+
+
+@pytest.mark.parametrize("dtype,Bz,T,Hq,Hkv,d", [("bf16", 1, 700, 8, 2, 128), ("f32", 2, 130, 4, 2, 32),
+                                                   ("bf16", 1, 64, 2, 1, 64), ("f32", 1, 1, 2, 2, 16)])
+def test_attention_forward(ctx, dtype, Bz, T, Hq, Hkv, d):
+    g = inputs.rng(55, T)
+    q = inputs.to_grid(g.standard_normal((Bz, T, Hq, d), dtype=np.float32), dtype)
+    k = inputs.to_grid(g.standard_normal((Bz, T, Hkv, d), dtype=np.float32), dtype)
+    v = inputs.to_grid(g.standard_normal((Bz, T, Hkv, d), dtype=np.float32), dtype)
+    scale = 1.0 / np.sqrt(d)
+    o = host(binding.str_attn_prefill(ctx, dev(q, dtype), dev(k, dtype), dev(v, dtype), scale))
+    for b in range(Bz):
+        assert max_rel_err(o[b], oracle.attention_forward(q[b], k[b], v[b], scale)) <= TOL[dtype]

@@ -1,0 +1,86 @@
+"""GPU parity: importance scores (attention-layer score and Eq. 2) against the oracle, and the
+score -> select pipeline with the swap tolerance."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2603_00198_b200 import binding, inputs
+from util_gpu import assert_kept_matches, dev, score_rel_err
+
+pytestmark = pytest.mark.gpu
+SCORE_TOL = 1e-3      # relative, fp32 (stated target)
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.check_status()
+    c.close()
+
+
+MAMBA_CASES = [
+    # dtype, n_vis, M, H, n, G, Bz
+    ("f32", 1024, 32, 8, 16, 1, 1),          # config 0
+    ("bf16", 4096, 128, 128, 128, 8, 1),     # config 1
+    ("bf16", 1000, 100, 16, 64, 4, 2),       # ragged tiles, batch
+    ("f32", 70, 3, 4, 32, 2, 1),
+    ("bf16", 5, 1, 2, 16, 1, 1),
+]
+
+
+@pytest.mark.parametrize("dtype,n_vis,M,H,n,G,Bz", MAMBA_CASES)
+def test_mamba_importance_matches_eq2(ctx, dtype, n_vis, M, H, n, G, Bz):
+    T = n_vis + M
+    d = inputs.ssd_inputs(31, T, H, 16, n, G, dtype, batch=Bz)
+    got = binding.str_mamba_importance(ctx, dev(d["B"], dtype), dev(d["C"], dtype), dev(d["dt"]), n_vis, M).cpu().numpy()
+    k = max(1, n_vis // 4)
+    for b in range(Bz):
+        ref = oracle.mamba_importance(d["B"][b], d["C"][b], d["dt"][b], n_vis, M)
+        assert score_rel_err(got[b], ref) <= SCORE_TOL
+        kept = binding.str_topk_select(ctx, dev(got[b:b + 1]), k).cpu().numpy()[0]
+        assert_kept_matches(kept, oracle.topk_select(ref, k), ref)
+
+
+ATTN_CASES = [
+    # dtype, n_vis, M, Hq, Hkv, d, Bz
+    ("bf16", 16384, 128, 32, 8, 128, 1),     # config 2
+    ("f32", 1000, 33, 4, 2, 64, 2),
+    ("bf16", 300, 5, 6, 2, 32, 1),
+    ("f32", 64, 1, 2, 2, 16, 1),
+    ("bf16", 3, 2, 4, 1, 128, 1),
+]
+
+
+@pytest.mark.parametrize("dtype,n_vis,M,Hq,Hkv,d,Bz", ATTN_CASES)
+def test_attn_importance_matches_definition(ctx, dtype, n_vis, M, Hq, Hkv, d, Bz):
+    T = n_vis + M
+    a = inputs.attn_score_inputs(32, T, Hq, Hkv, d, dtype, batch=Bz)
+    scale = 1.0 / np.sqrt(d)
+    got = binding.str_attn_importance(ctx, dev(a["q"], dtype), dev(a["k"], dtype), n_vis, M, scale).cpu().numpy()
+    k = max(1, n_vis // 4)
+    for b in range(Bz):
+        ref = oracle.attn_importance(a["q"][b], a["k"][b], n_vis, M, scale)
+        assert score_rel_err(got[b], ref) <= SCORE_TOL
+        assert abs(got[b].astype(np.float64).sum() - 1.0) < 1e-4          # softmax over the visual keys
+        kept = binding.str_topk_select(ctx, dev(got[b:b + 1]), k).cpu().numpy()[0]
+        assert_kept_matches(kept, oracle.topk_select(ref, k), ref)
+
+
+def test_attn_importance_large_logits_stay_finite(ctx):
+    a = inputs.attn_score_inputs(33, 200 + 4, 2, 1, 64, "f32")
+    a["q"] *= 30.0
+    got = binding.str_attn_importance(ctx, dev(a["q"]), dev(a["k"]), 200, 4, 1.0).cpu().numpy()[0]
+    ref = oracle.attn_importance(a["q"][0], a["k"][0], 200, 4, 1.0)
+    assert np.all(np.isfinite(got)) and abs(got.sum() - 1.0) < 1e-4
+    big = ref > 1e-6
+    assert score_rel_err(got[big], ref[big]) <= SCORE_TOL
+
+
+def test_score_argument_validation(ctx):
+    d = inputs.ssd_inputs(34, 40, 4, 16, 16, 2, "f32")
+    with pytest.raises(binding.StrError):      # n_vis + n_text != T
+        binding.str_mamba_importance(ctx, dev(d["B"]), dev(d["C"]), dev(d["dt"]), 30, 5)
+    a = inputs.attn_score_inputs(34, 40, 4, 2, 16, "f32")
+    with pytest.raises(binding.StrError):
+        binding.str_attn_importance(ctx, dev(a["q"]), dev(a["k"]), 41, 0, 1.0)

@@ -1,0 +1,87 @@
+"""GPU parity: str_topk_select and str_compact against the oracle's full sort and naive gather.
+Integer / byte work: bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_00198_b200 import binding, inputs
+from util_gpu import dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.check_status()
+    c.close()
+
+
+@pytest.mark.parametrize("kind", ["uniform", "heavy", "ties", "equal", "ascending", "descending"])
+@pytest.mark.parametrize("n,k", [(1, 1), (31, 7), (1000, 250), (1024, 256), (4096, 1024), (5000, 4999),
+                                 (32768, 16384), (65536, 6553)])
+def test_topk_matches_full_sort(ctx, kind, n, k):
+    s = inputs.score_vectors(11, n, kind, batch=2)
+    got = binding.str_topk_select(ctx, dev(s), k).cpu().numpy()
+    for b in range(2):
+        assert np.array_equal(got[b], oracle.topk_select(s[b], k)), (kind, n, k, b)
+
+
+def test_topk_edge_budgets(ctx):
+    s = inputs.score_vectors(12, 777, "uniform", batch=3)
+    full = binding.str_topk_select(ctx, dev(s), 777).cpu().numpy()
+    assert np.array_equal(full, np.tile(np.arange(777, dtype=np.int32), (3, 1)))     # 100% budget = identity
+    assert binding.str_topk_select(ctx, dev(s), 0).shape == (3, 0)
+    one = binding.str_topk_select(ctx, dev(s), 1).cpu().numpy()
+    assert np.array_equal(one[:, 0], s.argmax(axis=1))
+    with pytest.raises(binding.StrError):
+        binding.str_topk_select(ctx, dev(s), 778)
+
+
+def test_topk_negative_and_zero_scores(ctx):
+    s = np.array([[0.0, -1.0, 3.0, -0.5, 0.0, 2.0, -7.0, 1e-30]], dtype=np.float32)
+    for k in range(9):
+        got = binding.str_topk_select(ctx, dev(s), k).cpu().numpy()[0]
+        assert np.array_equal(got, oracle.topk_select(s[0], k))
+
+
+@pytest.mark.parametrize("dtype,D", [("bf16", 4096), ("f32", 256), ("bf16", 8), ("f32", 36)])
+@pytest.mark.parametrize("n_vis,n_text,k,Bz", [(1024, 32, 256, 1), (1000, 7, 333, 3), (64, 1, 64, 2), (50, 3, 0, 1)])
+def test_compact_is_a_bit_exact_gather(ctx, dtype, D, n_vis, n_text, k, Bz):
+    T = n_vis + n_text
+    h = inputs.hidden_inputs(21, T, D, dtype, batch=Bz)
+    g = inputs.rng(21, 9)
+    pos = np.sort(g.choice(10 * T, size=(Bz, T)), axis=1).astype(np.int32)
+    idx = g.integers(0, 1 << 30, size=(Bz, T)).astype(np.int32)
+    kept = np.stack([np.sort(g.choice(n_vis, size=k, replace=False)) for _ in range(Bz)]).astype(np.int32).reshape(Bz, k)
+    ho, po, io = binding.str_compact(ctx, dev(h, dtype), dev(pos), dev(idx), dev(kept), n_text)
+    ho = ho.float().cpu().numpy()
+    for b in range(Bz):
+        rh, rp, ri = oracle.compact(h[b], pos[b], idx[b], kept[b], n_text)
+        assert np.array_equal(ho[b], rh) and np.array_equal(po[b].cpu().numpy(), rp)
+        assert np.array_equal(io[b].cpu().numpy(), ri)
+
+
+def test_compact_twice_composes_to_original_ids(ctx):
+    n_vis, M, D = 2048, 16, 512
+    h = inputs.hidden_inputs(22, n_vis + M, D, "bf16")
+    ids = np.arange(n_vis + M, dtype=np.int32)[None]
+    g = inputs.rng(22, 9)
+    k1 = np.sort(g.choice(n_vis, size=1024, replace=False)).astype(np.int32)[None]
+    k2 = np.sort(g.choice(1024, size=512, replace=False)).astype(np.int32)[None]
+    h1, p1, i1 = binding.str_compact(ctx, dev(h, "bf16"), dev(ids), dev(ids), dev(k1), M)
+    h2, p2, i2 = binding.str_compact(ctx, h1, p1, i1, dev(k2), M)
+    i2 = i2.cpu().numpy()[0]
+    assert np.array_equal(i2[:512], k1[0][k2[0]]) and np.array_equal(i2[512:], np.arange(n_vis, n_vis + M))
+    assert np.array_equal(h2.float().cpu().numpy()[0], h[0][i2]) and np.all(np.diff(p2.cpu().numpy()[0]) > 0)
+
+
+def test_compact_rejects_bad_arguments(ctx):
+    h = dev(inputs.hidden_inputs(23, 10, 8, "f32"))
+    with pytest.raises(binding.StrError):       # k > n_vis
+        binding.str_compact(ctx, h, None, None, torch.zeros((1, 9), dtype=torch.int32, device="cuda"), 2)
+    with pytest.raises(binding.StrError):       # row not a multiple of 16 bytes
+        binding.str_compact(ctx, dev(inputs.hidden_inputs(23, 10, 3, "f32")), None, None,
+                            torch.zeros((1, 2), dtype=torch.int32, device="cuda"), 2)

@@ -1,0 +1,84 @@
+"""GPU parity: str_mamba2_prefill against the fp64 sequential recurrence."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2603_00198_b200 import binding, inputs
+from util_gpu import dev, host, max_rel_err
+
+pytestmark = pytest.mark.gpu
+TOL = {"bf16": 2e-2, "f32": 2e-4}     # max |err| / max |ref|; bf16 bound is the stated target
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.check_status()
+    c.close()
+
+
+CASES = [
+    # dtype, T, H, p, n, G, Q, Bz
+    ("f32", 1056, 8, 32, 16, 1, 64, 1),        # config 0 scan
+    ("bf16", 4224, 128, 64, 128, 8, 256, 1),   # config 1 scan
+    ("bf16", 1000, 16, 64, 128, 2, 256, 2),    # ragged tail, batch 2
+    ("f32", 333, 4, 16, 32, 2, 64, 1),
+    ("bf16", 1, 2, 64, 64, 1, 128, 1),         # single token
+    ("f32", 65, 2, 64, 16, 2, 0, 3),
+]
+
+
+@pytest.mark.parametrize("dtype,T,H,p,n,G,Q,Bz", CASES)
+def test_scan_matches_sequential_recurrence(ctx, dtype, T, H, p, n, G, Q, Bz):
+    d = inputs.ssd_inputs(41, T, H, p, n, G, dtype, batch=Bz)
+    y, fs = binding.str_mamba2_prefill(ctx, dev(d["x"], dtype), dev(d["dt"]), dev(d["A"]), dev(d["B"], dtype),
+                                       dev(d["C"], dtype), Q=Q, want_final_state=True)
+    y, fs = host(y), host(fs)
+    for b in range(Bz):
+        ry, rs = oracle.mamba2_recurrence(d["x"][b], d["dt"][b], d["A"], d["B"][b], d["C"][b])
+        assert max_rel_err(y[b], ry) <= TOL[dtype], (dtype, T, b)
+        assert max_rel_err(fs[b], rs) <= 1e-4
+
+
+def test_scan_initial_state_and_skip(ctx):
+    T, H, p, n, G = 200, 4, 32, 64, 2
+    d = inputs.ssd_inputs(42, T, H, p, n, G, "f32")
+    g = inputs.rng(42, 7)
+    S0 = g.standard_normal((1, H, p, n)).astype(np.float32)
+    D = g.standard_normal(H).astype(np.float32)
+    y = binding.str_mamba2_prefill(ctx, dev(d["x"]), dev(d["dt"]), dev(d["A"]), dev(d["B"]), dev(d["C"]),
+                                   D=dev(D), init_state=dev(S0))
+    ry, _ = oracle.mamba2_recurrence(d["x"][0], d["dt"][0], d["A"], d["B"][0], d["C"][0], D=D, init_state=S0[0])
+    assert max_rel_err(host(y)[0], ry) <= TOL["f32"]
+
+
+def test_scan_strong_decay_does_not_overflow(ctx):
+    # dt*|A| at its maximum for a whole chunk: cumulative log-decay ~ -400 over 256 tokens
+    T, H, p, n, G = 600, 2, 64, 128, 1
+    d = inputs.ssd_inputs(43, T, H, p, n, G, "bf16")
+    d["dt"][:] = 0.1
+    d["A"][:] = -16.0
+    y = binding.str_mamba2_prefill(ctx, dev(d["x"], "bf16"), dev(d["dt"]), dev(d["A"]), dev(d["B"], "bf16"),
+                                   dev(d["C"], "bf16"), Q=256)
+    ry, _ = oracle.mamba2_recurrence(d["x"][0], d["dt"][0], d["A"], d["B"][0], d["C"][0])
+    assert np.all(np.isfinite(host(y))) and max_rel_err(host(y)[0], ry) <= TOL["bf16"]
+
+
+def test_scan_result_does_not_depend_on_chunk_hint(ctx):
+    d = inputs.ssd_inputs(44, 500, 4, 32, 32, 2, "f32")
+    args = [dev(d["x"]), dev(d["dt"]), dev(d["A"]), dev(d["B"]), dev(d["C"])]
+    ys = [host(binding.str_mamba2_prefill(ctx, *args, Q=q)) for q in (0, 64, 128, 256)]
+    for y in ys[1:]:
+        assert max_rel_err(y, ys[0]) <= 1e-5
+
+
+def test_scan_argument_validation(ctx):
+    d = inputs.ssd_inputs(45, 10, 3, 16, 16, 1, "f32")
+    with pytest.raises(binding.StrError):     # H % G != 0
+        bad = inputs.ssd_inputs(45, 10, 3, 16, 16, 1, "f32")
+        B2 = np.concatenate([bad["B"], bad["B"]], axis=2)
+        binding.str_mamba2_prefill(ctx, dev(d["x"]), dev(d["dt"]), dev(d["A"]), dev(B2), dev(B2))
+    with pytest.raises(binding.StrError):     # head dimension the kernels do not tile
+        o = inputs.ssd_inputs(45, 10, 2, 24, 16, 1, "f32")
+        binding.str_mamba2_prefill(ctx, dev(o["x"]), dev(o["dt"]), dev(o["A"]), dev(o["B"]), dev(o["C"]))
