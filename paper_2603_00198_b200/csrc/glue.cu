@@ -82,7 +82,7 @@ mamba_conv_split_kernel(int Tlen, int H, int p, int n, int G, int W, const T *__
 // One thread per (token, head, pair index i < d/2) for q and k; v columns are copied.
 template <typename T>
 __global__ void __launch_bounds__(256)
-rope_split_kernel(int Hq, int Hkv, int d, float log2_theta, const int32_t *__restrict__ positions,
+rope_split_kernel(int Hq, int Hkv, int d, double log2_theta, const int32_t *__restrict__ positions,
                   const T *__restrict__ qkv, T *__restrict__ q_out, T *__restrict__ k_out, T *__restrict__ v_out) {
     const int half = d / 2;
     const int ld = (Hq + 2 * Hkv) * d;
@@ -94,7 +94,7 @@ rope_split_kernel(int Hq, int Hkv, int d, float log2_theta, const int32_t *__res
     if (e < n_rot) {
         const int head = e / half, i = e % half;
         // angle in fp64, reduced to [0, 2pi) before the fp32 sincos: positions reach tens of thousands
-        const double inv_freq = exp2(-2.0 * (double)i / (double)d * (double)log2_theta);
+        const double inv_freq = exp2(-2.0 * (double)i / (double)d * log2_theta);
         double ang = (double)positions[row] * inv_freq;
         ang -= 6.283185307179586476925 * floor(ang * 0.15915494309189533576888);
         float sn, cs;
@@ -172,7 +172,7 @@ extern "C" int str_rope_split(str_ctx *ctx, int dtype, int Bz, int T, int Hq, in
     const int work = (Hq + Hkv) * (d / 2) + Hkv * d;
     dim3 grid(ceil_div(work, 256), Bz * T);
     cudaStream_t st = (cudaStream_t)stream;
-    const float l2t = log2f(theta);
+    const double l2t = log2((double)theta);
     if (dtype == STR_BF16)
         rope_split_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(Hq, Hkv, d, l2t, positions, (const __nv_bfloat16 *)qkv,
                                                               (__nv_bfloat16 *)q_out, (__nv_bfloat16 *)k_out,
