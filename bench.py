@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark: token-reduced prefill of the 12-layer hybrid Mamba-2/attention stack on B200.
+
+One "step" = one whole prefill of the stack (all layers: projections, conv, scan, importance score,
+top-K select, compaction, attention) over one synthetic batch.  Metric: tokens/s = Bz*(N+M)/time.
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle on a bounded sample.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "token-reduced prefill tokens/s per layer stack"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM traffic per launch of the dominant kernel, from an ncu capture (bytes), or None.
+NCU_TRAFFIC = {}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+def workload(args):
+    from paper_2603_00198_b200 import inputs
+    cfg = dict(inputs.CONFIGS["C3"])
+    if args.n_vis:
+        cfg["n_vis"] = args.n_vis
+    if args.final_bp:
+        cfg["alpha_bp"] = inputs.sweep_alpha_bp(args.final_bp, len(cfg["pattern"]))
+    cfg["batch"] = args.batch
+    return cfg
+
+
+# ------------------------------------------------------------------ algorithmic work per category
+def work_model(cfg, keep_counts):
+    """Algorithmic flops / bytes of one step, per kernel category (formulas in the design doc)."""
+    ms, at = cfg["mamba"], cfg["attn"]
+    D, M, Bz = ms["D"], cfg["n_text"], cfg["batch"]
+    H, p, n, G, Q = ms["H"], ms["p"], ms["n"], ms["G"], ms["Q"]
+    Hq, Hkv, d = at["Hq"], at["Hkv"], at["d"]
+    d_inner, gn = H * p, G * n
+    dip, dqkv = 2 * d_inner + 2 * gn + H, (Hq + 2 * Hkv) * d
+    w = {k: dict(flops=0.0, bytes=0.0) for k in
+         ("gemm", "ssd_scan", "mamba_score", "attn_score", "topk", "compact", "attn_fwd")}
+    n_cur = cfg["n_vis"]
+    for kind, K in zip(cfg["pattern"], keep_counts):
+        T = n_cur + M
+        if kind == "M":
+            w["gemm"]["flops"] += 2.0 * Bz * T * D * dip + 2.0 * Bz * T * d_inner * D
+            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dip) + D * dip) + 2.0 * (Bz * T * (d_inner + 2 * D) + d_inner * D)
+            w["ssd_scan"]["flops"] += Bz * T * (G * 2 * n * (Q + 1) / 2 + H * (2 * p * (Q + 1) / 2 + 4 * n * p))
+            w["ssd_scan"]["bytes"] += Bz * T * (2 * (2 * H * p + 2 * G * n) + 4 * H)
+            if K < n_cur:
+                w["mamba_score"]["flops"] += Bz * n_cur * 2.0 * M * n * G
+                w["mamba_score"]["bytes"] += Bz * n_cur * (2 * G * n + 4 * H + 4)
+        else:
+            w["gemm"]["flops"] += 2.0 * Bz * T * D * dqkv + 2.0 * Bz * T * Hq * d * D
+            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dqkv) + D * dqkv) + 2.0 * (Bz * T * (Hq * d + 2 * D) + Hq * d * D)
+            w["attn_fwd"]["flops"] += Bz * Hq * 4.0 * d * T * (T + 1) / 2
+            w["attn_fwd"]["bytes"] += Bz * T * 2.0 * (2 * Hq * d + 2 * Hkv * d)
+            if K < n_cur:
+                w["attn_score"]["flops"] += 2 * Bz * n_cur * 2.0 * M * d * Hq
+                w["attn_score"]["bytes"] += 2 * Bz * n_cur * 2.0 * Hkv * d
+        if K < n_cur:
+            w["topk"]["bytes"] += Bz * (4.0 * n_cur + 4.0 * K)
+            w["compact"]["bytes"] += Bz * 2.0 * (K + M) * (2 * D + 8)
+            n_cur = K
+    return w
+
+
+BOUND = {"gemm": "tensor", "attn_fwd": "tensor", "ssd_scan": "tensor", "mamba_score": "hbm", "attn_score": "tensor",
+         "topk": "hbm", "compact": "hbm"}
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out["sm_mhz"] = float(np.median(sm))
+            out["sm_max_mhz"] = float(max(mx))
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------ CPU oracle leg
+def oracle_sample_tokens_per_s(cfg, n_vis_s, n_text_s, seed):
+    """Times the fp64 oracle, as it stands, on a short sequence with the full layer shapes and the
+    same schedule.  Returns (tokens/s, seconds, threads)."""
+    import oracle
+    from paper_2603_00198_b200 import inputs
+    layers = inputs.stack_params(seed, cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"])
+    h0 = inputs.hidden_inputs(seed, n_vis_s + n_text_s, cfg["mamba"]["D"], cfg["dtype"])[0]
+    K = oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0)
+    t0 = time.perf_counter()
+    oracle.stack_prefill(h0, n_text_s, layers, K, oracle.round_to_bf16)
+    sec = time.perf_counter() - t0
+    return (n_vis_s + n_text_s) / sec, sec, layers
+
+
+def run_reference(args):
+    """--impl reference: the oracle on host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2603_00198_b200 import inputs
+    cfg = workload(args)
+    cores = os.cpu_count() or 1
+    n_text_s = 16
+    n_vis_s = args.ref_tokens - n_text_s
+    layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"])
+    h0 = inputs.hidden_inputs(cfg["seed"], n_vis_s + n_text_s, cfg["mamba"]["D"], cfg["dtype"])[0]
+    K = oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0)
+
+    def step():
+        oracle.stack_prefill(h0, n_text_s, layers, K, oracle.round_to_bf16)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    sec = (time.perf_counter() - t0) / max(1, args.steps)
+    val = (n_vis_s + n_text_s) / sec
+    sample = ("fp64 oracle stack_prefill, full layer shapes, %d visual + %d text tokens per step, same schedule"
+              % (n_vis_s, n_text_s))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "C3 12-layer hybrid stack [M,M,M,M,M,A]x2 (sampled: %d tokens)" % (n_vis_s + n_text_s),
+                   "schedule_bp": cfg["alpha_bp"]},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2603_00198_b200 import binding, inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    cfg = workload(args)
+    Bz, n_vis, M, D = cfg["batch"], cfg["n_vis"], cfg["n_text"], cfg["mamba"]["D"]
+    T0 = n_vis + M
+    K = binding.str_schedule_keep_counts(cfg["alpha_bp"], n_vis, cfg["min_keep"])
+
+    ctx = binding.Context(local)
+    # weights: seeded on the host, one replica per rank (the path does not shard: replicas only)
+    layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], "f32")
+    stack = binding.Stack(ctx, layers, cfg["dtype"], Bz, n_vis, M, K, Q=cfg["mamba"]["Q"])
+    del layers
+    h_host = torch.from_numpy(inputs.hidden_inputs(cfg["seed"] + 1000 * rank, T0, D, "bf16", batch=Bz)).to(torch.bfloat16)
+    h_pin = h_host.pin_memory()
+    h_dev = h_pin.cuda()
+    out_pin = torch.empty((Bz, K[-1] + M, D), dtype=torch.bfloat16).pin_memory()
+    idx_pin = torch.empty((Bz, K[-1] + M), dtype=torch.int32).pin_memory()
+    ctx.workspace(max(stack.ws_bytes, stack.host_ws_bytes))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for _ in range(args.warmup):
+        binding.str_stack_prefill(stack, h_dev)
+    ctx.check_status()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    l0 = ctx.launch_count()
+    ctx.profile_enable(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        out, pos, idx = binding.str_stack_prefill(stack, h_dev)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    ctx.profile_enable(False)
+    prof = ctx.profile_collect()
+    launches = ctx.launch_count() - l0
+    clocks = sampler.stop() if sampler else None
+    ctx.check_status()
+
+    # ---- end to end through the host-buffer entry point (H2D + stack + D2H inside the timed region)
+    for _ in range(max(1, min(args.warmup, 2))):
+        binding.str_stack_prefill_host(stack, h_pin, out_pin, idx_pin)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(1, min(args.steps, 5))
+    e0.record()
+    for _ in range(e2e_steps):
+        binding.str_stack_prefill_host(stack, h_pin, out_pin, idx_pin)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    same = bool((out_pin.cuda() == out).all()) and bool((idx_pin.cuda() == idx).all())
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_step = ms_total / args.steps
+    tokens = Bz * T0 * world
+    value = tokens / (ms_step * 1e-3)
+    e2e_value = tokens / (ms_e2e / e2e_steps * 1e-3)
+    pk = peaks()
+    work = work_model(cfg, K)
+    kernels = {}
+    for cat, (ms, calls) in prof.items():
+        if calls == 0:
+            continue
+        per_step_ms = ms / args.steps
+        ent = {"ms_per_step": per_step_ms, "calls_per_step": calls / args.steps, "share": ms / ms_total}
+        if cat in work:
+            wk = work[cat]
+            ent["tflops"] = wk["flops"] / (per_step_ms * 1e-3) / 1e12 if wk["flops"] else None
+            ent["gbs"] = wk["bytes"] / (per_step_ms * 1e-3) / 1e9
+            if BOUND[cat] == "tensor":
+                ent["frac_of_tensor_peak"] = ent["tflops"] / pk["bf16_tflops_sustained"]
+            else:
+                ent["frac_of_hbm_peak"] = ent["gbs"] / pk["hbm_gbs"]
+        kernels[cat] = ent
+    dom = max((c for c in kernels if c in work), key=lambda c: kernels[c]["ms_per_step"])
+    if BOUND[dom] == "tensor":
+        roof = {"bound": "tensor", "achieved": kernels[dom]["tflops"], "peak": pk["bf16_tflops_sustained"],
+                "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC.get(dom)
+    roof["kernel"] = dom
+    roof["peak_source"] = "%s (sustained figure: kernel timed inside a long step)" % pk["source"]
+    roof["launch_ms"] = kernels[dom]["ms_per_step"] / kernels[dom]["calls_per_step"]
+
+    # ---- CPU oracle on a bounded sample of the same workload (rank 0, N=1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_text_s = 16
+        val, sec, _ = oracle_sample_tokens_per_s(cfg, args.ref_tokens - n_text_s, n_text_s, cfg["seed"])
+        cpu = {"value": val, "unit": UNIT, "cores": os.cpu_count() or 1, "kind": "oracle",
+               "sample": "fp64 oracle stack_prefill, full layer shapes and schedule, %d visual + %d text tokens, %.1f s"
+                         % (args.ref_tokens - n_text_s, n_text_s, sec)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "C3 12-layer hybrid stack [M,M,M,M,M,A]x2, %d visual + %d text tokens, batch %d, "
+                               "schedule %s" % (n_vis, M, Bz, "/".join(str(a // 100) for a in cfg["alpha_bp"][::4])),
+                   "keep_counts": K, "l2": "inputs larger than L2 (hidden %d MB, workspace %d MB)"
+                                           % (h_dev.numel() * 2 >> 20, stack.ws_bytes >> 20),
+                   "multi_gpu": "replicas only (the path does not shard)"},
+        "roofline": roof, "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h_pin.numel() * 2),
+                "d2h_bytes_per_step": int(out_pin.numel() * 2 + idx_pin.numel() * 4), "matches_device_run": same},
+        "gpu_launches": int(launches), "clocks": clocks, "kernels": kernels,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n-vis", type=int, default=0, help="override the visual token count (default: 32768)")
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--final-bp", type=int, default=0, help="final keep budget in basis points (sweep)")
+    ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the CPU oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

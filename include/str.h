@@ -225,6 +225,16 @@ int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, const void *hi
                            void *hidden_out_host, int32_t *idx_map_out_host, void *workspace,
                            size_t workspace_bytes, void *stream);
 
+/* Optional device timing by kernel category.  While enabled, every leaf entry point records a CUDA
+ * event pair around its launches on the caller's stream (str_profile_enable allocates events lazily on
+ * first use).  str_profile_collect synchronises on the recorded events, adds the elapsed milliseconds
+ * and the number of calls per category into the caller's host arrays (n >= STR_PROF_CATEGORIES) and
+ * forgets the recorded spans.  Categories: 0 GEMM, 1 Mamba-2 scan, 2 Mamba importance, 3 attention
+ * importance, 4 top-K select, 5 compaction, 6 attention forward, 7 element-wise glue. */
+#define STR_PROF_CATEGORIES 8
+int str_profile_enable(str_ctx *ctx, int on);
+int str_profile_collect(str_ctx *ctx, double *ms_by_category, long long *calls_by_category, int n);
+
 /* Number of kernels this library has launched on this context since creation (host counter). */
 long long str_launch_count(const str_ctx *ctx);
 

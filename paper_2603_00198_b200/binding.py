@@ -52,8 +52,11 @@ class StackDesc(ctypes.Structure):
                    ("score_every_layer", c_int)])
 
 
+PROF_CATEGORIES = ["gemm", "ssd_scan", "mamba_score", "attn_score", "topk", "compact", "attn_fwd", "elementwise"]
+
 EXPORTS = [
     "str_create", "str_destroy", "str_strerror", "str_check_status", "str_launch_count",
+    "str_profile_enable", "str_profile_collect",
     "str_mamba2_prefill_workspace_size", "str_mamba2_prefill",
     "str_mamba_importance_workspace_size", "str_mamba_importance",
     "str_attn_importance_workspace_size", "str_attn_importance",
@@ -149,6 +152,17 @@ class Context:
 
     def launch_count(self):
         return int(lib().str_launch_count(self._h))
+
+    def profile_enable(self, on=True):
+        _check(lib().str_profile_enable(self._h, c_int(1 if on else 0)), "str_profile_enable")
+
+    def profile_collect(self):
+        """Returns {category: (milliseconds, calls)} accumulated since the last collect."""
+        n = len(PROF_CATEGORIES)
+        ms = (ctypes.c_double * n)()
+        calls = (ctypes.c_longlong * n)()
+        _check(lib().str_profile_collect(self._h, ms, calls, c_int(n)), "str_profile_collect")
+        return {PROF_CATEGORIES[i]: (float(ms[i]), int(calls[i])) for i in range(n)}
 
 
 def str_mamba2_prefill(ctx, x, dt, A, B, C, D=None, init_state=None, Q=0, want_final_state=False):

@@ -13,6 +13,7 @@ extern "C" int str_mamba2_prefill(str_ctx *ctx, const str_ssd_shape *s, const vo
                                   const float *A, const void *B, const void *C, const float *D,
                                   const float *init_state, void *y, float *final_state, void *workspace,
                                   size_t workspace_bytes, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_SSD, stream);
     (void)workspace;
     if (!ctx || !s || !x || !dt || !A || !B || !C || !y) return STR_ERR_INVALID_ARG;
     if (s->Bz <= 0 || s->T < 0 || s->H <= 0 || s->p <= 0 || s->n <= 0 || s->G <= 0 || s->H % s->G != 0 || s->Q < 0 ||
@@ -32,6 +33,7 @@ extern "C" size_t str_mamba_importance_workspace_size(const str_ssm_score_shape 
 extern "C" int str_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text,
                                     const void *B, const void *C, const float *dt, float *scores_out,
                                     void *workspace, size_t workspace_bytes, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_MAMBA_SCORE, stream);
     (void)workspace; (void)workspace_bytes;
     if (!ctx || !s || !B || !C || !dt) return STR_ERR_INVALID_ARG;
     if (s->Bz <= 0 || s->H <= 0 || s->n <= 0 || s->G <= 0 || s->H % s->G != 0 || n_vis < 0 || n_text <= 0 ||
@@ -52,6 +54,7 @@ extern "C" size_t str_attn_importance_workspace_size(const str_attn_score_shape 
 extern "C" int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
                                    const void *q, const void *k, float softmax_scale, float *scores_out,
                                    void *workspace, size_t workspace_bytes, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ATTN_SCORE, stream);
     if (!ctx || !s || !q || !k) return STR_ERR_INVALID_ARG;
     if (s->Bz <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Hq % s->Hkv != 0 || s->d <= 0 || n_vis < 0 || n_text <= 0 ||
         n_vis + n_text != s->T || !STR_DTYPE_OK(s->dtype))
@@ -70,6 +73,7 @@ extern "C" size_t str_gemm_workspace_size(int, int, int, int) { return 0; }
 
 extern "C" int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w,
                         const void *residual, void *out, void *workspace, size_t workspace_bytes, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_GEMM, stream);
     (void)workspace; (void)workspace_bytes;
     if (!ctx || !a || !w || !out || M < 0 || N <= 0 || K <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
     if (M == 0) return STR_OK;
@@ -81,6 +85,7 @@ extern "C" size_t str_attn_prefill_workspace_size(const str_attn_shape *) { retu
 extern "C" int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v,
                                 float softmax_scale, void *o, void *workspace, size_t workspace_bytes,
                                 void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ATTN_FWD, stream);
     (void)workspace; (void)workspace_bytes;
     if (!ctx || !s || !q || !k || !v || !o) return STR_ERR_INVALID_ARG;
     if (s->Bz <= 0 || s->T <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Hq % s->Hkv != 0 || s->d <= 0 ||

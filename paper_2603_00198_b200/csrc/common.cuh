@@ -4,7 +4,16 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "str.h"
+
+// Per-category device timing (optional): an event pair around each leaf entry point.
+enum {
+    STR_CAT_GEMM = 0, STR_CAT_SSD, STR_CAT_MAMBA_SCORE, STR_CAT_ATTN_SCORE, STR_CAT_TOPK, STR_CAT_COMPACT,
+    STR_CAT_ATTN_FWD, STR_CAT_ELEMENTWISE, STR_CAT_COUNT
+};
+struct str_prof_span { int cat; cudaEvent_t beg, end; };
 
 struct str_ctx {
     int device;
@@ -13,6 +22,26 @@ struct str_ctx {
     int *status_dev;          // device status word: 0 or the first STR_ERR_* a kernel recorded
     void *encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), or nullptr
     long long launches;       // host-side count of kernels launched through this context
+    bool prof_on;             // record an event pair per leaf call
+    std::vector<str_prof_span> prof_spans;
+    std::vector<cudaEvent_t> prof_free;
+};
+
+struct StrProfScope {
+    str_ctx *ctx; cudaStream_t st; cudaEvent_t end; bool on;
+    StrProfScope(str_ctx *c, int cat, void *stream) : ctx(c), st((cudaStream_t)stream), end(nullptr), on(false) {
+        if (!c || !c->prof_on) return;
+        cudaEvent_t ev[2];
+        for (int i = 0; i < 2; ++i) {
+            if (!c->prof_free.empty()) { ev[i] = c->prof_free.back(); c->prof_free.pop_back(); }
+            else if (cudaEventCreate(&ev[i]) != cudaSuccess) return;
+        }
+        cudaEventRecord(ev[0], st);
+        c->prof_spans.push_back({cat, ev[0], ev[1]});
+        end = ev[1];
+        on = true;
+    }
+    ~StrProfScope() { if (on) cudaEventRecord(end, st); }
 };
 
 #define STR_CUDA_OK(call)                          \

@@ -57,6 +57,7 @@ extern "C" int str_compact(str_ctx *ctx, int Bz, int T_in, int n_vis, int n_text
                            const void *hidden, const int32_t *positions, const int32_t *idx_map,
                            const int32_t *kept_idx, void *hidden_out, int32_t *positions_out,
                            int32_t *idx_map_out, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_COMPACT, stream);
     if (!ctx || Bz <= 0 || n_vis < 0 || n_text < 0 || k < 0 || k > n_vis || D <= 0 ||
         T_in != n_vis + n_text || (dtype != STR_F32 && dtype != STR_BF16))
         return STR_ERR_INVALID_ARG;

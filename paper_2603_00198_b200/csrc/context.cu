@@ -14,6 +14,7 @@ extern "C" int str_create(int device, str_ctx **out) {
     if (!c) return STR_ERR_CUDA;
     c->device = device;
     c->launches = 0;
+    c->prof_on = false;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return STR_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;
@@ -34,6 +35,8 @@ extern "C" int str_create(int device, str_ctx **out) {
 extern "C" int str_destroy(str_ctx *ctx) {
     if (!ctx) return STR_ERR_INVALID_ARG;
     cudaFree(ctx->status_dev);
+    for (auto &sp : ctx->prof_spans) { cudaEventDestroy(sp.beg); cudaEventDestroy(sp.end); }
+    for (auto &ev : ctx->prof_free) cudaEventDestroy(ev);
     delete ctx;
     return STR_OK;
 }
@@ -61,6 +64,28 @@ extern "C" int str_check_status(str_ctx *ctx, void *stream) {
         STR_CUDA_OK(cudaStreamSynchronize(st));
     }
     return host;
+}
+
+extern "C" int str_profile_enable(str_ctx *ctx, int on) {
+    if (!ctx) return STR_ERR_INVALID_ARG;
+    ctx->prof_on = on != 0;
+    return STR_OK;
+}
+
+extern "C" int str_profile_collect(str_ctx *ctx, double *ms_by_category, long long *calls_by_category, int n) {
+    if (!ctx || !ms_by_category || !calls_by_category || n < STR_CAT_COUNT) return STR_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i) { ms_by_category[i] = 0.0; calls_by_category[i] = 0; }
+    for (auto &sp : ctx->prof_spans) {
+        if (cudaEventSynchronize(sp.end) != cudaSuccess) return STR_ERR_CUDA;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, sp.beg, sp.end) != cudaSuccess) return STR_ERR_CUDA;
+        ms_by_category[sp.cat] += ms;
+        calls_by_category[sp.cat] += 1;
+        ctx->prof_free.push_back(sp.beg);
+        ctx->prof_free.push_back(sp.end);
+    }
+    ctx->prof_spans.clear();
+    return STR_OK;
 }
 
 extern "C" long long str_launch_count(const str_ctx *ctx) { return ctx ? ctx->launches : -1; }

@@ -115,6 +115,7 @@ rope_split_kernel(int Hq, int Hkv, int d, double log2_theta, const int32_t *__re
 
 extern "C" int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, const void *in, void *out,
                            void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
     if (!ctx || !in || !out || rows < 0 || D <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
     if (rows == 0) return STR_OK;
     cudaStream_t st = (cudaStream_t)stream;
@@ -127,6 +128,7 @@ extern "C" int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, 
 
 extern "C" int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps,
                                  const void *y, const void *z, void *out, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
     if (!ctx || !y || !z || !out || rows < 0 || d_inner <= 0 || ld_z < d_inner || !STR_DTYPE_OK(dtype))
         return STR_ERR_INVALID_ARG;
     if (rows == 0) return STR_OK;
@@ -144,6 +146,7 @@ extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int 
                                     const void *zxbcdt, const float *conv_w, const float *conv_b,
                                     const float *dt_bias, void *x_out, void *B_out, void *C_out, float *dt_out,
                                     void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
     if (!ctx || !zxbcdt || !conv_w || !conv_b || !dt_bias || !x_out || !B_out || !C_out || !dt_out || Bz <= 0 ||
         T <= 0 || H <= 0 || p <= 0 || n <= 0 || G <= 0 || W <= 0 || !STR_DTYPE_OK(dtype))
         return STR_ERR_INVALID_ARG;
@@ -165,6 +168,7 @@ extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int 
 extern "C" int str_rope_split(str_ctx *ctx, int dtype, int Bz, int T, int Hq, int Hkv, int d, float theta,
                               const int32_t *positions, const void *qkv, void *q_out, void *k_out, void *v_out,
                               void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
     if (!ctx || !positions || !qkv || !q_out || !k_out || !v_out || Bz <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 ||
         d <= 0 || (d & 1) || theta <= 0.f || !STR_DTYPE_OK(dtype))
         return STR_ERR_INVALID_ARG;

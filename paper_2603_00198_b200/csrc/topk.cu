@@ -126,6 +126,7 @@ extern "C" size_t str_topk_select_workspace_size(int, int, int) { return 0; }
 
 extern "C" int str_topk_select(str_ctx *ctx, int Bz, int n_vis, int k, const float *scores,
                                int32_t *kept_idx_out, void *, size_t, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_TOPK, stream);
     if (!ctx || Bz <= 0 || n_vis < 0 || k < 0 || k > n_vis) return STR_ERR_INVALID_ARG;
     if (k == 0) return STR_OK;
     if (!scores || !kept_idx_out) return STR_ERR_INVALID_ARG;

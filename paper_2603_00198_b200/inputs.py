@@ -41,9 +41,9 @@ def to_grid(a, dtype):
         return a
     if dtype != "bf16":
         raise ValueError(dtype)
-    u = a.view(np.uint32).astype(np.uint64)
-    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
-    return u.astype(np.uint32).view(np.float32).reshape(a.shape)
+    u = a.view(np.uint32)
+    u = (u + (((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF))) & np.uint32(0xFFFF0000)
+    return u.view(np.float32).reshape(a.shape)
 
 
 def bf16_bits(a):
