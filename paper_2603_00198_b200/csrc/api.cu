@@ -1,7 +1,16 @@
 // extern "C" entry points of the hot path: argument validation and kernel selection.
 #include "dispatch.cuh"
 
+#include <stdlib.h>
+
 #define STR_DTYPE_OK(dt) ((dt) == STR_F32 || (dt) == STR_BF16)
+
+// Debug switch: STR_FORCE_SIMT=1 routes every call to the plain FFMA kernels (for A/B parity runs).
+bool str_force_simt() {
+    static int v = -1;
+    if (v < 0) { const char *e = getenv("STR_FORCE_SIMT"); v = (e && e[0] == '1') ? 1 : 0; }
+    return v == 1;
+}
 
 // ---------------------------------------------------------------- (1) Mamba-2 SSD scan
 extern "C" size_t str_mamba2_prefill_workspace_size(const str_ssd_shape *s) {
@@ -77,6 +86,8 @@ extern "C" int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void
     (void)workspace; (void)workspace_bytes;
     if (!ctx || !a || !w || !out || M < 0 || N <= 0 || K <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
     if (M == 0) return STR_OK;
+    if (!str_force_simt() && ctx->encode_tiled && str_gemm_tc_supported(dtype, M, N, K, a, w, residual, out))
+        return str_gemm_tc(ctx, M, N, K, a, w, residual, out, (cudaStream_t)stream);
     return str_gemm_simt(ctx, dtype, M, N, K, a, w, residual, out, (cudaStream_t)stream);
 }
 

@@ -15,3 +15,8 @@ int str_gemm_simt(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, c
                   const void *residual, void *out, cudaStream_t st);
 int str_attn_prefill_simt(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v,
                           float scale, void *o, cudaStream_t st);
+bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const void *w, const void *residual,
+                           const void *out);
+int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
+                cudaStream_t st);
+bool str_force_simt();

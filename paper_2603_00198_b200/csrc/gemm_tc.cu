@@ -1,0 +1,198 @@
+// bf16 GEMM on the 5th-generation tensor cores: out[M,N] = a[M,K] * w[N,K]^T (+ residual).
+//
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warp 0     TMA producer: streams 128x64 A tiles and 256x64 W tiles (128-byte swizzle) through a
+//              4-stage shared-memory ring guarded by full/empty mbarriers.
+//   warp 1     MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16) into one of two
+//              256-column fp32 accumulators in tensor memory; tcgen05.commit frees smem stages and
+//              publishes finished accumulators.
+//   warps 2-5  epilogue: tcgen05.ld the accumulator (each warp its own 32-lane quadrant), add the
+//              residual, narrow to bf16, 16-byte stores.  Runs concurrently with the next tile's
+//              main loop thanks to the double-buffered accumulator.
+// Tiles are walked in bands of 8 column tiles so that a band of W stays in L2 while A streams.
+// Every mbarrier wait is bounded; on give-up the kernel records STR_ERR_TIMEOUT and tears down.
+#include "dispatch.cuh"
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + W_BYTES;
+constexpr int NUM_THREADS = 192;            // 6 warps
+constexpr int BAND = 8;                     // column tiles per L2 band
+constexpr size_t SMEM_BYTES = 1024 /*align slack*/ + (size_t)STAGES * STAGE_BYTES + 256;
+
+struct TileCoord { int m, n; };
+__device__ __forceinline__ TileCoord tile_coord(int t, int tiles_m, int tiles_n) {
+    const int per_band = BAND * tiles_m;
+    const int band = t / per_band, r = t % per_band;
+    const int n0 = band * BAND;
+    const int width = min(BAND, tiles_n - n0);
+    return {r / width, n0 + r % width};
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w, int M, int N,
+               int K, const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ out, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
+    uint64_t *full = bars, *empty = bars + STAGES, *acc_full = bars + 2 * STAGES, *acc_empty = bars + 2 * STAGES + 2;
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN, tiles = tiles_m * tiles_n;
+    const int k_blocks = (K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, 1); }
+        for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, 4); }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        tc::fence_mbar_init();
+        tc::prefetch_tmap(&tmap_a);
+        tc::prefetch_tmap(&tmap_w);
+    }
+    if (warp == 1) { tc::tmem_alloc(tmem_slot, 512); tc::tmem_relinquish(); }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+                const TileCoord tc_ = tile_coord(t, tiles_m, tiles_n);
+                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!tc::mbar_wait(empty + s, ph ^ 1, abort_flag)) { ok = false; break; }
+                    tc::mbar_arrive_expect_tx(full + s, STAGE_BYTES);
+                    uint8_t *sa = smem + (size_t)s * STAGE_BYTES;
+                    tc::tma_load_2d(sa, &tmap_a, full + s, kb * BK, tc_.m * BM);
+                    tc::tma_load_2d(sa + A_BYTES, &tmap_w, full + s, kb * BK, tc_.n * BN);
+                }
+            }
+            if (!ok) {
+                atomicCAS(status, 0, STR_ERR_TIMEOUT);
+                // let copies already issued land before the CTA's shared memory goes away
+                for (int back = 1; back <= STAGES && back <= it; ++back) {
+                    const int j = it - back;
+                    tc::mbar_wait(full + j % STAGES, (j / STAGES) & 1, abort_flag + 1);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = tc::make_idesc_bf16(BM, BN, 0, 0);
+            int it = 0, local = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++local) {
+                const int acc = local & 1;
+                const uint32_t aph = (local >> 1) & 1;
+                if (!tc::mbar_wait(acc_empty + acc, aph ^ 1, abort_flag)) { ok = false; break; }
+                tc::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
+                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!tc::mbar_wait(full + s, ph, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint32_t sa = tc::smem_u32(smem + (size_t)s * STAGE_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk)
+                        tc::mma_ss(d_tmem, tc::desc_kmajor_sw128(sa, kk * UMMA_K),
+                                   tc::desc_kmajor_sw128(sa + A_BYTES, kk * UMMA_K), idesc, (kb | kk) != 0);
+                    tc::mma_commit(empty + s);
+                }
+                if (ok) tc::mma_commit(acc_full + acc);
+            }
+            if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+        }
+    } else {
+        const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
+        int local = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++local) {
+            const TileCoord tc_ = tile_coord(t, tiles_m, tiles_n);
+            const int acc = local & 1;
+            const uint32_t aph = (local >> 1) & 1;
+            if (!tc::mbar_wait(acc_full + acc, aph, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after();
+            const int row = tc_.m * BM + quad * 32 + lane;
+            const int col0 = tc_.n * BN;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t v[32];
+                tc::tmem_ld32(taddr + c, v);
+                tc::tmem_ld_wait();
+                if (row < M && col0 + c < N) {
+                    const size_t off = (size_t)row * N + col0 + c;
+                    const int valid = min(32, N - (col0 + c));       // multiple of 8 (N % 8 == 0)
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (g * 8 < valid) {
+                            float f[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]);
+                            if (residual) {
+                                const uint4 r = *reinterpret_cast<const uint4 *>(residual + off + g * 8);
+                                const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    f[2 * j] += __uint_as_float(rw[j] << 16);
+                                    f[2 * j + 1] += __uint_as_float(rw[j] & 0xFFFF0000u);
+                                }
+                            }
+                            uint4 o;
+                            o.x = tc::pack_bf16x2(f[0], f[1]);
+                            o.y = tc::pack_bf16x2(f[2], f[3]);
+                            o.z = tc::pack_bf16x2(f[4], f[5]);
+                            o.w = tc::pack_bf16x2(f[6], f[7]);
+                            *reinterpret_cast<uint4 *>(out + off + g * 8) = o;
+                        }
+                    }
+                }
+            }
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(acc_empty + acc);
+        }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, 512); }
+}
+
+}  // namespace
+
+bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const void *w, const void *residual,
+                           const void *out) {
+    if (dtype != STR_BF16 || M < 1 || N % 8 != 0 || K % 8 != 0 || K < 8) return false;
+    const uintptr_t al = (uintptr_t)a | (uintptr_t)w | (uintptr_t)residual | (uintptr_t)out;
+    return (al & 15) == 0;
+}
+
+int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
+                cudaStream_t st) {
+    CUtensorMap ta, tw;
+    int rc = str_make_tmap_2d_bf16(ctx, &ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != STR_OK) return rc;
+    rc = str_make_tmap_2d_bf16(ctx, &tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN, BK, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != STR_OK) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        STR_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+        attr_set = true;
+    }
+    const int tiles = ceil_div(M, BM) * ceil_div(N, BN);
+    const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tw, M, N, K, (const __nv_bfloat16 *)residual,
+                                                         (__nv_bfloat16 *)out, ctx->status_dev);
+    return str_launch_ok(ctx);
+}
