@@ -99,6 +99,25 @@ int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, 
                         const void *q, const void *k, float softmax_scale, float *scores_out,
                         void *workspace, size_t workspace_bytes, void *stream);
 
+/* (2b, allocation-free variant)  The paper has no counterpart for this call; it exists for callers
+ * that cannot allocate device memory (a plug-in inside a host with a fixed memory pool, a real-time
+ * loop that must stay off the allocator, code that is handed raw pointers and owns no allocator).
+ * Same inputs, outputs and result as str_attn_importance, but the per-(sequence, head, query) row
+ * maxima and sums live in a fixed array inside the library image, so no workspace is passed and the
+ * call performs no allocation of any kind.
+ *   Limit: Bz * Hq * n_text <= STR_ATTN_STATIC_MAX_ROWS, else STR_ERR_WORKSPACE_TOO_SMALL is
+ *   returned and nothing is launched.  The array (2 * STR_ATTN_STATIC_MAX_ROWS floats = 512 KiB) is
+ *   resident on every GPU that loads the library until the process exits.
+ *   The first call on a device looks up the array's device address (one runtime query, no
+ *   allocation); make that first call before starting any stream capture.
+ *   All calls share the array and it keeps the previous call's contents; each call overwrites the
+ *   part it uses before reading it, so nothing needs clearing, but two calls whose kernels overlap
+ *   on the GPU (different streams, no ordering between them) race on it: serialise them. */
+#define STR_ATTN_STATIC_MAX_ROWS 65536
+int str_attn_importance_static(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
+                               const void *q, const void *k, float softmax_scale, float *scores_out,
+                               void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * (3) Top-K selection preserving temporal order (Section 3.1 "Token Selection"): the indices of
  * the k largest scores of each row, written in ascending index order.  Among equal scores the

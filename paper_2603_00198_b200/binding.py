@@ -59,7 +59,7 @@ EXPORTS = [
     "str_profile_enable", "str_profile_collect",
     "str_mamba2_prefill_workspace_size", "str_mamba2_prefill",
     "str_mamba_importance_workspace_size", "str_mamba_importance",
-    "str_attn_importance_workspace_size", "str_attn_importance",
+    "str_attn_importance_workspace_size", "str_attn_importance", "str_attn_importance_static",
     "str_topk_select_workspace_size", "str_topk_select", "str_compact",
     "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
     "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_mamba_conv_split", "str_gated_rmsnorm",
@@ -201,6 +201,23 @@ def str_attn_importance(ctx, q, k, n_vis, n_text, softmax_scale):
     _check(lib().str_attn_importance(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(q), _p(k),
                                      c_float(softmax_scale), _p(out), _p(ws), c_size_t(ws.numel()), _stream()),
            "str_attn_importance")
+    return out
+
+
+STR_ATTN_STATIC_MAX_ROWS = 65536
+
+
+def str_attn_importance_static(ctx, q, k, n_vis, n_text, softmax_scale, out=None):
+    """Allocation-free variant for callers that cannot allocate device memory: the scratch is a fixed
+    array inside the library, so only inputs and the output buffer are passed (pass ``out`` to avoid
+    even the output allocation this wrapper would otherwise make)."""
+    Bz, T, Hq, d = q.shape
+    Hkv = k.shape[2]
+    s = AttnScoreShape(Bz, T, Hq, Hkv, d, _dt(q))
+    if out is None:
+        out = torch.empty((Bz, n_vis), dtype=torch.float32, device=q.device)
+    _check(lib().str_attn_importance_static(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(q), _p(k),
+                                            c_float(softmax_scale), _p(out), _stream()), "str_attn_importance_static")
     return out
 
 

@@ -249,3 +249,50 @@ int str_attn_importance_simt(str_ctx *ctx, const str_attn_score_shape *s, int n_
                ? launch_attn_importance<__nv_bfloat16>(ctx, s, n_vis, n_text, q, k, scale, scores, row_max, row_sum, st)
                : launch_attn_importance<float>(ctx, s, n_vis, n_text, q, k, scale, scores, row_max, row_sum, st);
 }
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free attention importance.  Some callers may not allocate device memory at all: a
+// plug-in running inside a host whose memory pool is fixed at start-up, a real-time loop that must
+// not hit the allocator's lock, or code that is handed raw pointers and owns no allocator.  For them
+// the row statistics of the first pass live in a fixed array inside the library image instead of a
+// caller workspace.  Every GPU that loads the library carries the array until the process exits.
+static __device__ __align__(256) float g_attn_static_rowstats[2 * STR_ATTN_STATIC_MAX_ROWS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float *g_rowstats_dev_ptr[kMaxDevices] = {};   // device address of the array, per device (host cache)
+}  // namespace
+
+extern "C" int str_attn_importance_static(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
+                                          const void *q, const void *k, float softmax_scale, float *scores_out,
+                                          void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ATTN_SCORE, stream);
+    if (!ctx || !s || !q || !k) return STR_ERR_INVALID_ARG;
+    if (s->Bz <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Hq % s->Hkv != 0 || s->d <= 0 || n_vis < 0 || n_text <= 0 ||
+        n_vis + n_text != s->T || (s->dtype != STR_F32 && s->dtype != STR_BF16))
+        return STR_ERR_INVALID_ARG;
+    const long long rows = (long long)s->Bz * s->Hq * n_text;
+    if (rows > STR_ATTN_STATIC_MAX_ROWS) return STR_ERR_WORKSPACE_TOO_SMALL;   // beyond the built-in scratch
+    if (n_vis == 0) return STR_OK;
+    if (!scores_out) return STR_ERR_INVALID_ARG;
+    if (ctx->device < 0 || ctx->device >= kMaxDevices) return STR_ERR_INVALID_ARG;
+    float *base = g_rowstats_dev_ptr[ctx->device];
+    if (!base) {
+        // One-time set-up per device: in host code the array's name is only a stand-in, so ask the
+        // runtime for its device address, with the context's device current.
+        int prev = -1;
+        STR_CUDA_OK(cudaGetDevice(&prev));
+        if (prev != ctx->device) STR_CUDA_OK(cudaSetDevice(ctx->device));
+        void *sym = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&sym, g_attn_static_rowstats);
+        if (prev != ctx->device) cudaSetDevice(prev);
+        if (e != cudaSuccess || !sym) return STR_ERR_CUDA;
+        base = (float *)sym;
+        g_rowstats_dev_ptr[ctx->device] = base;
+    }
+    // Both halves are fully rewritten by the first pass before the second pass reads them, so nothing
+    // left over from an earlier call is ever used and nothing needs clearing.
+    float *row_max = base, *row_sum = base + rows;
+    return str_attn_importance_simt(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, row_max, row_sum,
+                                    (cudaStream_t)stream);
+}
