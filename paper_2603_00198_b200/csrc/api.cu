@@ -29,6 +29,9 @@ extern "C" int str_mamba2_prefill(str_ctx *ctx, const str_ssd_shape *s, const vo
         !STR_DTYPE_OK(s->dtype))
         return STR_ERR_INVALID_ARG;
     if (workspace_bytes < str_mamba2_prefill_workspace_size(s)) return STR_ERR_WORKSPACE_TOO_SMALL;
+    if (s->T == 0) return STR_OK;
+    if (!str_force_simt() && ctx->encode_tiled && str_ssd_tc_supported(s, x, B, C, y, D, init_state))
+        return str_ssd_tc(ctx, s, x, dt, A, B, C, y, final_state, (cudaStream_t)stream);
     if (!str_ssd_simt_supported(s)) return STR_ERR_UNSUPPORTED_SHAPE;
     return str_ssd_simt(ctx, s, x, dt, A, B, C, D, init_state, y, final_state, (cudaStream_t)stream);
 }

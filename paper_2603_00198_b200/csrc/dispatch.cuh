@@ -20,3 +20,7 @@ bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const 
 int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
                 cudaStream_t st);
 bool str_force_simt();
+bool str_ssd_tc_supported(const str_ssd_shape *s, const void *x, const void *B, const void *C, const void *y,
+                          const float *D, const float *init_state);
+int str_ssd_tc(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float *dt, const float *A, const void *B,
+               const void *C, void *y, float *final_state, cudaStream_t st);

@@ -38,7 +38,9 @@ def test_scan_matches_sequential_recurrence(ctx, dtype, T, H, p, n, G, Q, Bz):
     for b in range(Bz):
         ry, rs = oracle.mamba2_recurrence(d["x"][b], d["dt"][b], d["A"], d["B"][b], d["C"][b])
         assert max_rel_err(y[b], ry) <= TOL[dtype], (dtype, T, b)
-        assert max_rel_err(fs[b], rs) <= 1e-4
+        # the state update contracts bf16 copies of the decay-scaled inputs, so the final state carries
+        # bf16-level rounding on the bf16 path
+        assert max_rel_err(fs[b], rs) <= (1e-2 if dtype == "bf16" else 1e-4)
 
 
 def test_scan_initial_state_and_skip(ctx):
