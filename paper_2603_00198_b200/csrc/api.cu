@@ -105,5 +105,7 @@ extern "C" int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const voi
     if (s->Bz <= 0 || s->T <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Hq % s->Hkv != 0 || s->d <= 0 ||
         !STR_DTYPE_OK(s->dtype))
         return STR_ERR_INVALID_ARG;
+    if (!str_force_simt() && ctx->encode_tiled && str_attn_prefill_tc_supported(s, q, k, v, o))
+        return str_attn_prefill_tc(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
     return str_attn_prefill_simt(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
 }

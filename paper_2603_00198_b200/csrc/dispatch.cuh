@@ -24,3 +24,6 @@ bool str_ssd_tc_supported(const str_ssd_shape *s, const void *x, const void *B, 
                           const float *D, const float *init_state);
 int str_ssd_tc(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float *dt, const float *A, const void *B,
                const void *C, void *y, float *final_state, cudaStream_t st);
+bool str_attn_prefill_tc_supported(const str_attn_shape *s, const void *q, const void *k, const void *v, const void *o);
+int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v, float scale,
+                        void *o, cudaStream_t st);

@@ -82,7 +82,13 @@ def test_rope_split(ctx, dtype, Bz, T, Hq, Hkv, d):
 
 
 @pytest.mark.parametrize("dtype,Bz,T,Hq,Hkv,d", [("bf16", 1, 700, 8, 2, 128), ("f32", 2, 130, 4, 2, 32),
-                                                   ("bf16", 1, 64, 2, 1, 64), ("f32", 1, 1, 2, 2, 16)])
+                                                   ("bf16", 1, 64, 2, 1, 64), ("f32", 1, 1, 2, 2, 16),
+                                                   # head_dim 128 in bf16 runs on the tensor cores: tile edges,
+                                                   # ragged tails, one query-tile pair and several, no GQA, batch
+                                                   ("bf16", 1, 1, 2, 1, 128), ("bf16", 1, 128, 2, 2, 128),
+                                                   ("bf16", 1, 129, 4, 1, 128), ("bf16", 2, 256, 2, 1, 128),
+                                                   ("bf16", 1, 257, 2, 2, 128), ("bf16", 2, 1000, 4, 2, 128),
+                                                   ("bf16", 1, 1536, 4, 4, 128)])
 def test_attention_forward(ctx, dtype, Bz, T, Hq, Hkv, d):
     g = inputs.rng(55, T)
     q = inputs.to_grid(g.standard_normal((Bz, T, Hq, d), dtype=np.float32), dtype)
@@ -92,3 +98,25 @@ def test_attention_forward(ctx, dtype, Bz, T, Hq, Hkv, d):
     o = host(binding.str_attn_prefill(ctx, dev(q, dtype), dev(k, dtype), dev(v, dtype), scale))
     for b in range(Bz):
         assert max_rel_err(o[b], oracle.attention_forward(q[b], k[b], v[b], scale)) <= TOL[dtype]
+
+
+def test_attention_forward_growing_logits_rescale(ctx):
+    """Logits that keep growing along the key axis force the running row maximum up tile after tile, so
+    the accumulator rescaling path runs many times; a second input has one huge late key."""
+    T, Hq, Hkv, d = 900, 2, 1, 128
+    g = inputs.rng(56, T)
+    q = inputs.to_grid(g.standard_normal((1, T, Hq, d), dtype=np.float32), "bf16")
+    k = inputs.to_grid(g.standard_normal((1, T, Hkv, d), dtype=np.float32), "bf16")
+    v = inputs.to_grid(g.standard_normal((1, T, Hkv, d), dtype=np.float32), "bf16")
+    u = g.standard_normal(d).astype(np.float32)
+    u /= np.linalg.norm(u)
+    ramp = (np.arange(T, dtype=np.float32) / T * 60.0)[:, None, None]
+    q2 = inputs.to_grid(q + 4.0 * u, "bf16")
+    k2 = inputs.to_grid(k + ramp * u, "bf16")               # q.k grows by ~240/sqrt(d)*... along the keys
+    k3 = k.copy()
+    k3[0, 700] = inputs.to_grid(40.0 * u, "bf16")           # one dominant key late in the sequence
+    scale = 1.0 / np.sqrt(d)
+    for kk in (k2, k3):
+        o = host(binding.str_attn_prefill(ctx, dev(q2, "bf16"), dev(kk, "bf16"), dev(v, "bf16"), scale))
+        assert np.all(np.isfinite(o))
+        assert max_rel_err(o[0], oracle.attention_forward(q2[0], kk[0], v[0], scale)) <= TOL["bf16"]
