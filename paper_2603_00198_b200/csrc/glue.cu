@@ -109,6 +109,178 @@ rope_split_kernel(int Hq, int Hkv, int d, double log2_theta, const int32_t *__re
     }
 }
 
+
+// ---- 16-byte vectorised bf16 versions (used when the row length and strides are multiples of 8) ----
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[2 * j] = __uint_as_float(w[j] << 16);
+        f[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+    }
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+    return make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+}
+
+// RMSNorm, one warp per row, the row held in registers between the reduction and the scaling
+// (rows of up to 32 * 8 * VPL elements): each element is read once and written once.
+template <int VPL>
+__global__ void __launch_bounds__(256)
+rmsnorm_bf16_vec_kernel(int rows, int D, float eps, const __nv_bfloat16 *__restrict__ in, __nv_bfloat16 *__restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int nvec = D >> 3;
+    const uint4 *r = reinterpret_cast<const uint4 *>(in + (size_t)row * D);
+    uint4 *o = reinterpret_cast<uint4 *>(out + (size_t)row * D);
+    uint4 v[VPL];
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+        const int c = lane + 32 * i;
+        v[i] = c < nvec ? __ldg(r + c) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+        float f[8];
+        unpack8(v[i], f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) ss = fmaf(f[j], f[j], ss);
+    }
+    const float inv = rsqrtf(warp_sum(ss) / (float)D + eps);
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+        const int c = lane + 32 * i;
+        if (c < nvec) {
+            float f[8];
+            unpack8(v[i], f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) f[j] *= inv;
+            o[c] = pack8(f);
+        }
+    }
+}
+
+// Gated RMSNorm, one CTA per row, y * SiLU(z) held in registers (rows of up to 256 * 8 * VPT elements).
+template <int VPT>
+__global__ void __launch_bounds__(256)
+gated_rmsnorm_bf16_vec_kernel(int d_inner, int ld_z, float eps, const __nv_bfloat16 *__restrict__ y,
+                              const __nv_bfloat16 *__restrict__ z, __nv_bfloat16 *__restrict__ out) {
+    __shared__ float red[32];
+    const int nvec = d_inner >> 3;
+    const uint4 *yr = reinterpret_cast<const uint4 *>(y + (size_t)blockIdx.x * d_inner);
+    const uint4 *zr = reinterpret_cast<const uint4 *>(z + (size_t)blockIdx.x * ld_z);
+    uint4 *o = reinterpret_cast<uint4 *>(out + (size_t)blockIdx.x * d_inner);
+    uint4 yv[VPT], zv[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int c = threadIdx.x + 256 * i;
+        yv[i] = c < nvec ? __ldg(yr + c) : make_uint4(0u, 0u, 0u, 0u);
+        zv[i] = c < nvec ? __ldg(zr + c) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    float g[VPT][8];
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        float fy[8], fz[8];
+        unpack8(yv[i], fy);
+        unpack8(zv[i], fz);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            g[i][j] = fy[j] * silu_f(fz[j]);
+            ss = fmaf(g[i][j], g[i][j], ss);
+        }
+    }
+    const float inv = rsqrtf(block_sum(ss, red) / (float)d_inner + eps);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int c = threadIdx.x + 256 * i;
+        if (c < nvec) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) g[i][j] *= inv;
+            o[c] = pack8(g[i]);
+        }
+    }
+}
+
+// Mamba-2 pre-scan step, width-4 conv: one thread owns 8 consecutive conv channels and walks CONV_TT
+// consecutive tokens with the three previous inputs held in registers, so every input element is
+// read once (plus a 3-token halo per tile) and every output written once, all as 16-byte vectors.
+// The last block column handles the dt columns.
+constexpr int CONV_TT = 32;
+__global__ void __launch_bounds__(256)
+mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __nv_bfloat16 *__restrict__ zxbcdt,
+                                 const float *__restrict__ conv_w, const float *__restrict__ conv_b,
+                                 const float *__restrict__ dt_bias, __nv_bfloat16 *__restrict__ x_out,
+                                 __nv_bfloat16 *__restrict__ B_out, __nv_bfloat16 *__restrict__ C_out,
+                                 float *__restrict__ dt_out) {
+    const int d_inner = H * p, gn = G * n;
+    const int conv_dim = d_inner + 2 * gn;
+    const int ld = 2 * d_inner + 2 * gn + H;
+    const int tiles = (Tlen + CONV_TT - 1) / CONV_TT;
+    const int b = blockIdx.y / tiles, t0 = (blockIdx.y % tiles) * CONV_TT;
+    const int t1 = min(Tlen, t0 + CONV_TT);
+    const size_t row0 = (size_t)b * Tlen;
+    if (blockIdx.x == gridDim.x - 1) {
+        for (int e = threadIdx.x; e < (t1 - t0) * H; e += blockDim.x) {
+            const int t = t0 + e / H, h = e % H;
+            dt_out[(row0 + t) * H + h] =
+                softplus_f(__bfloat162float(zxbcdt[(row0 + t) * ld + d_inner + conv_dim + h]) + dt_bias[h]);
+        }
+        return;
+    }
+    const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    if (c0 >= conv_dim) return;
+    float w[8][4], bias[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float4 wv = __ldg(reinterpret_cast<const float4 *>(conv_w) + c0 + j);
+        w[j][0] = wv.x; w[j][1] = wv.y; w[j][2] = wv.z; w[j][3] = wv.w;
+        bias[j] = __ldg(conv_b + c0 + j);
+    }
+    __nv_bfloat16 *dst;
+    int dst_ld;
+    if (c0 < d_inner) { dst = x_out + c0; dst_ld = d_inner; }
+    else if (c0 < d_inner + gn) { dst = B_out + (c0 - d_inner); dst_ld = gn; }
+    else { dst = C_out + (c0 - d_inner - gn); dst_ld = gn; }
+    const __nv_bfloat16 *src = zxbcdt + d_inner + c0;
+    float h3[8], h2[8], h1[8];     // inputs of tokens t-3, t-2, t-1
+    {
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        unpack8(t0 >= 3 ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + t0 - 3) * ld)) : zero, h3);
+        unpack8(t0 >= 2 ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + t0 - 2) * ld)) : zero, h2);
+        unpack8(t0 >= 1 ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + t0 - 1) * ld)) : zero, h1);
+    }
+    for (int tb = t0; tb < t1; tb += 4) {
+        uint4 raw[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            raw[u] = (tb + u < t1) ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + tb + u) * ld))
+                                   : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            float cur[8], o[8];
+            unpack8(raw[u], cur);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float acc = bias[j];
+                acc = fmaf(w[j][0], h3[j], acc);
+                acc = fmaf(w[j][1], h2[j], acc);
+                acc = fmaf(w[j][2], h1[j], acc);
+                acc = fmaf(w[j][3], cur[j], acc);
+                o[j] = silu_f(acc);
+                h3[j] = h2[j]; h2[j] = h1[j]; h1[j] = cur[j];
+            }
+            if (tb + u < t1) *reinterpret_cast<uint4 *>(dst + (row0 + tb + u) * dst_ld) = pack8(o);
+        }
+    }
+}
+
 }  // namespace
 
 #define STR_DTYPE_OK(dt) ((dt) == STR_F32 || (dt) == STR_BF16)
@@ -119,7 +291,10 @@ extern "C" int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, 
     if (!ctx || !in || !out || rows < 0 || D <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
     if (rows == 0) return STR_OK;
     cudaStream_t st = (cudaStream_t)stream;
-    if (dtype == STR_BF16)
+    if (dtype == STR_BF16 && D % 8 == 0 && D <= 32 * 8 * 16 && (((uintptr_t)in | (uintptr_t)out) & 15) == 0)
+        rmsnorm_bf16_vec_kernel<16><<<ceil_div(rows, 8), 256, 0, st>>>(rows, D, eps, (const __nv_bfloat16 *)in,
+                                                                         (__nv_bfloat16 *)out);
+    else if (dtype == STR_BF16)
         rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>(D, eps, (const __nv_bfloat16 *)in, (__nv_bfloat16 *)out);
     else
         rmsnorm_kernel<float><<<rows, 256, 0, st>>>(D, eps, (const float *)in, (float *)out);
@@ -133,7 +308,11 @@ extern "C" int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner,
         return STR_ERR_INVALID_ARG;
     if (rows == 0) return STR_OK;
     cudaStream_t st = (cudaStream_t)stream;
-    if (dtype == STR_BF16)
+    if (dtype == STR_BF16 && d_inner % 8 == 0 && ld_z % 8 == 0 && d_inner <= 256 * 8 * 4 &&
+        (((uintptr_t)y | (uintptr_t)z | (uintptr_t)out) & 15) == 0)
+        gated_rmsnorm_bf16_vec_kernel<4><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const __nv_bfloat16 *)y,
+                                                                (const __nv_bfloat16 *)z, (__nv_bfloat16 *)out);
+    else if (dtype == STR_BF16)
         gated_rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const __nv_bfloat16 *)y,
                                                                  (const __nv_bfloat16 *)z, (__nv_bfloat16 *)out);
     else
@@ -154,6 +333,20 @@ extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int 
     const int cols = H * p + 2 * G * n + H;
     dim3 grid(ceil_div(cols, 256), Bz * T);
     cudaStream_t st = (cudaStream_t)stream;
+    const int d_inner_ = H * p, gn_ = G * n;
+    if (dtype == STR_BF16 && W == 4 && d_inner_ % 8 == 0 && gn_ % 8 == 0 && H % 8 == 0 &&
+        (((uintptr_t)zxbcdt | (uintptr_t)x_out | (uintptr_t)B_out | (uintptr_t)C_out | (uintptr_t)conv_w) & 15) == 0) {
+        const int tiles = ceil_div(T, CONV_TT);
+        if ((long long)Bz * tiles > 65535) {
+            // grid.y limit: fall through to the generic kernel below
+        } else {
+            dim3 vgrid(ceil_div((d_inner_ + 2 * gn_) / 8, 256) + 1, Bz * tiles);
+            mamba_conv_split_bf16_vec_kernel<<<vgrid, 256, 0, st>>>(
+                T, H, p, n, G, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
+                (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out);
+            return str_launch_ok(ctx);
+        }
+    }
     if (dtype == STR_BF16)
         mamba_conv_split_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
             T, H, p, n, G, W, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,

@@ -34,7 +34,8 @@ def test_gemm_with_residual(ctx, dtype, M, N, K):
     assert max_rel_err(got, ref + r) <= TOL[dtype]
 
 
-@pytest.mark.parametrize("dtype,rows,D", [("bf16", 100, 4096), ("f32", 33, 256), ("bf16", 5, 40)])
+@pytest.mark.parametrize("dtype,rows,D", [("bf16", 100, 4096), ("f32", 33, 256), ("bf16", 5, 40), ("bf16", 9, 8192),
+                                          ("bf16", 3, 36)])
 def test_rmsnorm(ctx, dtype, rows, D):
     u = inputs.hidden_inputs(52, rows, D, dtype)[0] * 3.0
     u = inputs.to_grid(u, dtype)
@@ -42,7 +43,9 @@ def test_rmsnorm(ctx, dtype, rows, D):
     assert max_rel_err(got, oracle.rmsnorm(u)) <= TOL[dtype]
 
 
-@pytest.mark.parametrize("dtype,Bz,T,H,p,n,G", [("bf16", 1, 300, 16, 64, 128, 2), ("f32", 2, 70, 8, 32, 16, 1)])
+@pytest.mark.parametrize("dtype,Bz,T,H,p,n,G", [("bf16", 1, 300, 16, 64, 128, 2), ("f32", 2, 70, 8, 32, 16, 1),
+                                                ("bf16", 3, 70, 8, 64, 64, 1), ("bf16", 2, 33, 4, 16, 32, 2),
+                                                ("bf16", 1, 2, 8, 64, 128, 8)])
 def test_conv_split_and_gated_norm(ctx, dtype, Bz, T, H, p, n, G):
     d_inner, gn = H * p, G * n
     ld = 2 * d_inner + 2 * gn + H
