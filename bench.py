@@ -333,6 +333,112 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+
+# ------------------------------------------------------------------ single-kernel microbenchmarks
+def run_micro(args):
+    """--micro NAME: times one entry point of the hot path alone (CUDA events, L2 flushed between launches)
+    on seeded device-side inputs of the C1/C2 layer shapes and prints one JSON line with its roofline."""
+    import torch
+    from paper_2603_00198_b200 import binding, inputs
+    torch.cuda.set_device(0)
+    torch.manual_seed(1234)
+    ctx = binding.Context(0)
+    pk = peaks()
+    ms_, at_ = inputs.MAMBA_8B, inputs.ATTN_8B
+    Bz, n_vis, M = args.batch, (args.n_vis or 32768), 128
+    T = n_vis + M
+    dev = "cuda:0"
+    bf = torch.bfloat16
+    name = args.micro
+    flops = nbytes = 0.0
+    bound = "hbm"
+    if name == "ssd":
+        H, p, n, G, Q = ms_["H"], ms_["p"], ms_["n"], ms_["G"], ms_["Q"]
+        x = torch.randn(Bz, T, H, p, device=dev).to(bf)
+        Bm = torch.randn(Bz, T, G, n, device=dev).to(bf)
+        Cm = torch.randn(Bz, T, G, n, device=dev).to(bf)
+        dt = torch.empty(Bz, T, H, device=dev).uniform_(1e-3, 1e-1)
+        A = -torch.exp(torch.empty(H, device=dev).uniform_(0.0, float(np.log(16.0))))
+        fn = lambda: binding.str_mamba2_prefill(ctx, x, dt, A, Bm, Cm, Q=Q)
+        flops = Bz * T * (G * 2 * n * (Q + 1) / 2 + H * (2 * p * (Q + 1) / 2 + 4 * n * p))
+        nbytes = Bz * T * (2 * (2 * H * p + 2 * G * n) + 4 * H)
+        bound = "tensor"
+    elif name == "mamba_score":
+        H, n, G = ms_["H"], ms_["n"], ms_["G"]
+        Bm = torch.randn(Bz, T, G, n, device=dev).to(bf)
+        Cm = torch.randn(Bz, T, G, n, device=dev).to(bf)
+        dt = torch.empty(Bz, T, H, device=dev).uniform_(1e-3, 1e-1)
+        fn = lambda: binding.str_mamba_importance(ctx, Bm, Cm, dt, n_vis, M)
+        flops = Bz * n_vis * 2.0 * M * n * G
+        nbytes = Bz * n_vis * (2 * G * n + 4 * H + 4)
+    elif name == "attn_score":
+        Hq, Hkv, d = at_["Hq"], at_["Hkv"], at_["d"]
+        q = torch.randn(Bz, T, Hq, d, device=dev).to(bf)
+        k = torch.randn(Bz, T, Hkv, d, device=dev).to(bf)
+        fn = lambda: binding.str_attn_importance(ctx, q, k, n_vis, M, 1.0 / np.sqrt(d))
+        flops = 2 * Bz * n_vis * 2.0 * M * d * Hq
+        nbytes = 2 * Bz * n_vis * 2.0 * Hkv * d
+        bound = "tensor"
+    elif name == "attn_fwd":
+        Hq, Hkv, d = at_["Hq"], at_["Hkv"], at_["d"]
+        q = torch.randn(Bz, T, Hq, d, device=dev).to(bf)
+        k = torch.randn(Bz, T, Hkv, d, device=dev).to(bf)
+        v = torch.randn(Bz, T, Hkv, d, device=dev).to(bf)
+        fn = lambda: binding.str_attn_prefill(ctx, q, k, v, 1.0 / np.sqrt(d))
+        flops = Bz * Hq * 4.0 * d * T * (T + 1) / 2
+        nbytes = Bz * T * 2.0 * (2 * Hq * d + 2 * Hkv * d)
+        bound = "tensor"
+    elif name == "topk":
+        K = max(1, n_vis * (args.final_bp or 5000) // 10000)
+        sc = torch.rand(Bz, n_vis, device=dev)
+        fn = lambda: binding.str_topk_select(ctx, sc, K)
+        nbytes = Bz * (4.0 * n_vis + 4.0 * K)
+    elif name == "compact":
+        D = ms_["D"]
+        K = max(1, n_vis * (args.final_bp or 5000) // 10000)
+        hid = torch.randn(Bz, T, D, device=dev).to(bf)
+        pos = torch.arange(T, device=dev, dtype=torch.int32).repeat(Bz, 1).contiguous()
+        kept = torch.sort(torch.rand(Bz, n_vis, device=dev).argsort(dim=1)[:, :K], dim=1).values.to(torch.int32).contiguous()
+        fn = lambda: binding.str_compact(ctx, hid, pos, pos, kept, M)
+        nbytes = Bz * 2.0 * (K + M) * (2 * D + 8)
+    elif name == "gemm":
+        D = ms_["D"]
+        N = 2 * ms_["H"] * ms_["p"] + 2 * ms_["G"] * ms_["n"] + ms_["H"]
+        a = torch.randn(Bz * T, D, device=dev).to(bf)
+        w = (torch.randn(N, D, device=dev) / 64.0).to(bf)
+        fn = lambda: binding.str_gemm(ctx, a, w)
+        flops = 2.0 * Bz * T * N * D
+        nbytes = 2.0 * (Bz * T * (D + N) + N * D)
+        bound = "tensor"
+    else:
+        raise SystemExit("unknown --micro " + name)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for _ in range(max(3, args.warmup)):
+        fn()
+    ctx.check_status()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ctx.check_status()
+    ms = float(np.median(times))
+    if bound == "tensor":
+        ach, peak, unit = flops / (ms * 1e-3) / 1e12, pk["bf16_tflops"], "TFLOP/s"
+    else:
+        ach, peak, unit = nbytes / (ms * 1e-3) / 1e9, pk["hbm_gbs"], "GB/s"
+    print(json.dumps({"micro": name, "batch": Bz, "n_vis": n_vis, "n_text": M, "ms": ms, "ms_min": float(min(times)),
+                      "steps": args.steps, "l2": "256 MB buffer written between launches",
+                      "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                                   "peak_source": pk["source"] + " (burst figure: kernel timed alone)"},
+                      "gbs": nbytes / (ms * 1e-3) / 1e9, "tflops": flops / (ms * 1e-3) / 1e12 if flops else None}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -344,10 +450,14 @@ def main():
     ap.add_argument("--final-bp", type=int, default=0, help="final keep budget in basis points (sweep)")
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the CPU oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | attn_score | attn_fwd | "
+                                                "topk | compact | gemm")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    if args.impl == "reference":
+    if args.micro:
+        run_micro(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

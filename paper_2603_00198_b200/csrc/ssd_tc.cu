@@ -2,20 +2,28 @@
 // state dim n = 128.  One CTA per (sequence, head) walks the sequence in chunks of 128 tokens and
 // carries the running state in registers, so chunk states never travel through global memory.
 //
-// Per chunk, with l_t the in-chunk inclusive cumulative log-decay (l_t = sum_{u<=t} dt_u A_h <= 0):
+// Per chunk c, with l_t the in-chunk inclusive cumulative log-decay (l_t = sum_{u<=t} dt_u A_h <= 0):
 //   CB      = C B^T                                  [128 x 128]   tcgen05, K-major operands
-//   W[t,j]  = CB[t,j] exp(l_t - l_j) dt_j 1[j<=t]    fp32 on CUDA cores -> bf16 -> shared memory
-//   Y_intra = W X                                    [128 x 64]    tcgen05, X as MN-major operand
+//   W[t,j]  = CB[t,j] exp(l_t - l_j) dt_j 1[j<=t]    fp32 on CUDA cores -> bf16, written back over CB in
+//                                                    tensor memory: the A operand of the next product
+//   Y_intra = W X                                    [128 x 64]    tcgen05, A from tensor memory, X MN-major
 //   Y_inter = C S_prev^T                             [128 x 64]    tcgen05, bf16 copy of the state
 //   y_t     = Y_intra[t] + exp(l_t) Y_inter[t]                     fp32 epilogue -> bf16 -> global
 //   dS^T    = B^T Xs,  Xs_j = exp(l_end - l_j) dt_j x_j  [128 x 64] tcgen05, both operands MN-major
 //   S^T    <- exp(l_end) S^T + dS^T                                fp32 registers (the master state)
 // Every decay factor is formed from a difference of cumulative sums that is <= 0.  Off the
 // diagonal 32x32 blocks exp(l_t - l_j) is split into three factors, each <= 1 (row part, block-pair
-// scalar, column part), which turns 128x128 exponentials per chunk into O(128) plus the diagonal blocks.
+// scalar, column part); the diagonal blocks take one exponential per element.
 //
-// Warp roles: 0-7 compute (256 threads; warp w owns TMEM lane quadrant w%4 and column half w/4),
-// 8 = TMA producer (x, B, C tiles, 128-byte swizzle, 2 stages), 9 = MMA issuer (one thread).
+// The chunk loop is software-pipelined across warp roles that only meet at mbarriers, so the only
+// serial chain from chunk to chunk is  dS_c -> state update -> Y_inter_{c+1}:
+//   warps 0-3    W_c from CB_c                       (one thread per token row)
+//   warps 4-7    Xs_c, then the state update         (one thread per state row n)
+//   warps 8-11   epilogue of chunk c                 (one thread per token row)
+//   warp 12      TMA producer: B,C ring of 2, X ring of 3 (128-byte swizzle)
+//   warp 13      MMA issuer; iteration c issues  CB_c, Y_inter_c, dS_c, Y_intra_{c-1}
+//   warp 14      decay vectors of chunk c (cumulative sum, exponentials) into a ring of 4
+// Tensor memory: CB/W 2 x 128 columns | Y_inter 2 x 64 | Y_intra 64 | dS 64.
 // All mbarrier waits are bounded; a give-up records STR_ERR_TIMEOUT and tears the CTA down.
 #include "dispatch.cuh"
 #include "tc_common.cuh"
@@ -24,30 +32,24 @@ namespace {
 
 constexpr int Q = 128, P = 64, NS = 128;
 constexpr int TILE_16K = 16384;
-constexpr int OFF_X = 0, OFF_B = TILE_16K, OFF_C = 3 * TILE_16K, STAGE_BYTES = 5 * TILE_16K;   // X | B0 B1 | C0 C1
-constexpr int OFF_W = 2 * STAGE_BYTES, OFF_XT = OFF_W + 2 * TILE_16K, OFF_SB = OFF_XT + TILE_16K;
-constexpr int OFF_MISC = OFF_SB + TILE_16K;
-constexpr int MISC_BYTES = 4 * 512 + 32 + 64 + 14 * 8 + 16;
-constexpr size_t SMEM_BYTES = (size_t)OFF_MISC + MISC_BYTES;
-constexpr int COMPUTE_THREADS = 256, NUM_THREADS = 320;
-// TMEM columns
-constexpr uint32_t TM_CB = 0, TM_YI = 256, TM_YO = 320, TM_DS = 384;
-
-enum { B_FULL0 = 0, B_FULL1, B_EMPTY0, B_EMPTY1, B_CBR0, B_CBR1, B_CBF0, B_CBF1, B_XT, B_DS, B_W, B_S, B_Y, B_YF, B_COUNT };
-
-__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-// Barrier over the 256 compute threads that also ANDs a predicate, so that every compute warp takes
-// the same decision to leave the chunk loop (a warp that left alone would strand the others).
-__device__ __forceinline__ bool compute_sync_and(bool v) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 1, 256, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r) : "r"((uint32_t)v) : "memory");
-    return r != 0;
-}
+constexpr int X_SLOTS = 3, DEC_DEPTH = 4, DEC_FLOATS = 800;
+constexpr int OFF_X = 0;                                  // 3 x 16 KB
+constexpr int OFF_B = OFF_X + X_SLOTS * TILE_16K;         // 2 x 32 KB
+constexpr int OFF_C = OFF_B + 4 * TILE_16K;               // 2 x 32 KB
+constexpr int OFF_XS = OFF_C + 4 * TILE_16K;              // 16 KB
+constexpr int OFF_SB = OFF_XS + TILE_16K;                 // 16 KB
+constexpr int OFF_DEC = OFF_SB + TILE_16K;                // 4 x 3200 B
+constexpr int OFF_BARS = OFF_DEC + DEC_DEPTH * DEC_FLOATS * 4;
+// decay vectors of one chunk (floats): log2-domain cumulative decay, dt, column / state / row factors
+constexpr int D_LS = 0, D_DT = 128, D_COLF = 256, D_XW = 384, D_ROWF = 512, D_EROW = 640, D_BLK = 768, D_EEND = 784;
+enum {
+    B_XF = 0, B_XE = 3, B_BCF = 6, B_BCE = 8, B_DECF = 10, B_DECE = 14, B_CBF = 18, B_WF = 20, B_XSF = 22, B_DSF, B_DSE,
+    B_SF, B_YF, B_YE, B_COUNT
+};
+constexpr size_t SMEM_BYTES = (size_t)OFF_BARS + B_COUNT * 8 + 32;
+constexpr int NUM_THREADS = 480;
+constexpr uint32_t TM_CB = 0, TM_YO = 256, TM_YI = 384, TM_DS = 448;
+constexpr float LOG2E = 1.4426950408889634f;
 
 __device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane) {
     __syncwarp();
@@ -59,14 +61,8 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
               const __grid_constant__ CUtensorMap tmap_c, int Tlen, int H, int G, const float *__restrict__ dt,
               const float *__restrict__ A, __nv_bfloat16 *__restrict__ y, float *__restrict__ final_state, int *status) {
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint8_t *misc = smem + OFF_MISC;
-    float *ls = (float *)misc;            // [128] cumulative log-decay
-    float *dts = ls + 128;                // [128] dt
-    float *colf = dts + 128;              // [128] exp(l_blockend - l_j) * dt_j
-    float *xw = colf + 128;               // [128] exp(l_end - l_j) * dt_j
-    float *wsum = xw + 128;               // [4] per-block sums of dt*A, then [4] block-start values
-    float *blk = wsum + 8;                // [4][4] exp(l_blockstart(bt) - l_blockend(bj))
-    uint64_t *bars = (uint64_t *)(blk + 16);
+    float *decs = (float *)(smem + OFF_DEC);
+    uint64_t *bars = (uint64_t *)(smem + OFF_BARS);
     uint32_t *tmem_slot = (uint32_t *)(bars + B_COUNT);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
@@ -78,167 +74,247 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (threadIdx.x == 0) atomicCAS(status, 0, STR_ERR_CUDA);
         return;
     }
+    if (*(volatile int *)status != 0) return;         // an earlier CTA failed: leave at once
     if (threadIdx.x == 0) {
-        tc::mbar_init(bars + B_FULL0, 1); tc::mbar_init(bars + B_FULL1, 1);
-        tc::mbar_init(bars + B_EMPTY0, 1); tc::mbar_init(bars + B_EMPTY1, 1);
-        tc::mbar_init(bars + B_CBR0, 1); tc::mbar_init(bars + B_CBR1, 1);
-        tc::mbar_init(bars + B_CBF0, 8); tc::mbar_init(bars + B_CBF1, 8);
-        tc::mbar_init(bars + B_XT, 8); tc::mbar_init(bars + B_DS, 1); tc::mbar_init(bars + B_W, 8);
-        tc::mbar_init(bars + B_S, 8); tc::mbar_init(bars + B_Y, 1); tc::mbar_init(bars + B_YF, 8);
+        for (int i = 0; i < X_SLOTS; ++i) { tc::mbar_init(bars + B_XF + i, 1); tc::mbar_init(bars + B_XE + i, 5); }
+        for (int i = 0; i < 2; ++i) {
+            tc::mbar_init(bars + B_BCF + i, 1); tc::mbar_init(bars + B_BCE + i, 1);
+            tc::mbar_init(bars + B_CBF + i, 1); tc::mbar_init(bars + B_WF + i, 4);
+        }
+        for (int i = 0; i < DEC_DEPTH; ++i) { tc::mbar_init(bars + B_DECF + i, 1); tc::mbar_init(bars + B_DECE + i, 12); }
+        tc::mbar_init(bars + B_XSF, 4); tc::mbar_init(bars + B_DSF, 1); tc::mbar_init(bars + B_DSE, 4);
+        tc::mbar_init(bars + B_SF, 4); tc::mbar_init(bars + B_YF, 1); tc::mbar_init(bars + B_YE, 4);
         abort_flag[0] = 0; abort_flag[1] = 0;
         tc::fence_mbar_init();
         tc::prefetch_tmap(&tmap_x); tc::prefetch_tmap(&tmap_b); tc::prefetch_tmap(&tmap_c);
     }
-    if (warp == 9) { tc::tmem_alloc(tmem_slot, 512); tc::tmem_relinquish(); }
+    if (warp == 13) { tc::tmem_alloc(tmem_slot, 512); tc::tmem_relinquish(); }
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 8) {
+    if (warp == 12) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             bool ok = true;
-            int c = 0;
-            for (; c < nchunks; ++c) {
-                const int s = c & 1;
-                if (!tc::mbar_wait(bars + B_EMPTY0 + s, ((c >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                uint64_t *fb = bars + B_FULL0 + s;
-                tc::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-                uint8_t *st = smem + (size_t)s * STAGE_BYTES;
-                const int t0 = c * Q;
-                tc::tma_load_3d(st + OFF_X, &tmap_x, fb, h * P, t0, b);
-                tc::tma_load_3d(st + OFF_B, &tmap_b, fb, g * NS, t0, b);
-                tc::tma_load_3d(st + OFF_B + TILE_16K, &tmap_b, fb, g * NS + 64, t0, b);
-                tc::tma_load_3d(st + OFF_C, &tmap_c, fb, g * NS, t0, b);
-                tc::tma_load_3d(st + OFF_C + TILE_16K, &tmap_c, fb, g * NS + 64, t0, b);
+            int n_bc = 0, n_x = 0;
+            for (int c = 0; c < nchunks; ++c) {
+                const int t0 = c * Q, s = c & 1, sx = c % X_SLOTS;
+                if (!tc::mbar_wait(bars + B_BCE + s, ((c >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                uint64_t *fb = bars + B_BCF + s;
+                tc::mbar_arrive_expect_tx(fb, 4 * TILE_16K);
+                tc::tma_load_3d(smem + OFF_B + (s * 2) * TILE_16K, &tmap_b, fb, g * NS, t0, b);
+                tc::tma_load_3d(smem + OFF_B + (s * 2 + 1) * TILE_16K, &tmap_b, fb, g * NS + 64, t0, b);
+                tc::tma_load_3d(smem + OFF_C + (s * 2) * TILE_16K, &tmap_c, fb, g * NS, t0, b);
+                tc::tma_load_3d(smem + OFF_C + (s * 2 + 1) * TILE_16K, &tmap_c, fb, g * NS + 64, t0, b);
+                ++n_bc;
+                if (!tc::mbar_wait(bars + B_XE + sx, ((c / X_SLOTS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                tc::mbar_arrive_expect_tx(bars + B_XF + sx, TILE_16K);
+                tc::tma_load_3d(smem + OFF_X + sx * TILE_16K, &tmap_x, bars + B_XF + sx, h * P, t0, b);
+                ++n_x;
             }
             if (!ok) {
                 atomicCAS(status, 0, STR_ERR_TIMEOUT);
-                for (int back = 1; back <= 2 && back <= c; ++back) {      // let issued copies land
-                    const int j = c - back;
-                    tc::mbar_wait(bars + B_FULL0 + (j & 1), (j >> 1) & 1, abort_flag + 1);
+                for (int back = 1; back <= 2 && back <= n_bc; ++back) {      // let issued copies land
+                    const int j = n_bc - back;
+                    tc::mbar_wait(bars + B_BCF + (j & 1), (j >> 1) & 1, abort_flag + 1);
+                }
+                for (int back = 1; back <= X_SLOTS && back <= n_x; ++back) {
+                    const int j = n_x - back;
+                    tc::mbar_wait(bars + B_XF + j % X_SLOTS, (j / X_SLOTS) & 1, abort_flag + 1);
                 }
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == 13) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t id_cb = tc::make_idesc_bf16(128, 128, 0, 0);   // C (K-major) x B (K-major)
-            const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major A x MN-major B
+            const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major / tensor-memory A x MN-major B
             const uint32_t id_nn = tc::make_idesc_bf16(128, 64, 1, 1);    // MN-major A x MN-major B
             const uint32_t sbase = tc::smem_u32(smem);
             bool ok = true;
-            auto issue_cb = [&](int c) {
-                const uint32_t st = sbase + (uint32_t)(c & 1) * STAGE_BYTES;
-                const uint32_t d = tmem + TM_CB + (uint32_t)(c & 1) * 128;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    tc::mma_ss(d, tc::desc_kmajor_sw128(st + OFF_C + (ks >> 2) * TILE_16K, (ks & 3) * 16),
-                               tc::desc_kmajor_sw128(st + OFF_B + (ks >> 2) * TILE_16K, (ks & 3) * 16), id_cb, ks != 0);
-                tc::mma_commit(bars + B_CBR0 + (c & 1));
-            };
-            if (nchunks > 0) {
-                ok = tc::mbar_wait(bars + B_FULL0, 0, abort_flag);
-                if (ok) { tc::tc_fence_after(); issue_cb(0); }
-            }
-            for (int c = 0; c < nchunks && ok; ++c) {
-                const uint32_t st = sbase + (uint32_t)(c & 1) * STAGE_BYTES;
-                if (c > 0) {
-                    // state of chunk c-1 is in shared memory; Y accumulators have been read out
-                    if (!tc::mbar_wait(bars + B_S, (c - 1) & 1, abort_flag)) { ok = false; break; }
-                    if (!tc::mbar_wait(bars + B_YF, (c - 1) & 1, abort_flag)) { ok = false; break; }
+            for (int c = 0; c <= nchunks && ok; ++c) {
+                const int s = c & 1;
+                if (c >= 2) {        // the epilogue has read the Y accumulators of chunk c-2
+                    if (!tc::mbar_wait(bars + B_YE, (c - 2) & 1, abort_flag)) { ok = false; break; }
+                }
+                if (c < nchunks) {
+                    const uint32_t bt = sbase + OFF_B + (uint32_t)s * 2 * TILE_16K;
+                    const uint32_t ct = sbase + OFF_C + (uint32_t)s * 2 * TILE_16K;
+                    if (!tc::mbar_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc::tc_fence_after();
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)      // Y_inter = C S_prev^T
-                        tc::mma_ss(tmem + TM_YO, tc::desc_kmajor_sw128(st + OFF_C + (ks >> 2) * TILE_16K, (ks & 3) * 16),
-                                   tc::make_smem_desc(sbase + OFF_SB + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_kn,
-                                   ks != 0);
-                }
-                if (!tc::mbar_wait(bars + B_XT, c & 1, abort_flag)) { ok = false; break; }
-                tc::tc_fence_after();
+                    for (int ks = 0; ks < 8; ++ks)      // CB_c = C B^T
+                        tc::mma_ss(tmem + TM_CB + (uint32_t)s * 128, tc::desc_kmajor_sw128(ct + (ks >> 2) * TILE_16K, (ks & 3) * 16),
+                                   tc::desc_kmajor_sw128(bt + (ks >> 2) * TILE_16K, (ks & 3) * 16), id_cb, ks != 0);
+                    tc::mma_commit(bars + B_CBF + s);
+                    if (c > 0) {
+                        if (!tc::mbar_wait(bars + B_SF, (c - 1) & 1, abort_flag)) { ok = false; break; }
+                        tc::tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)          // dS^T = B^T Xs
-                    tc::mma_ss(tmem + TM_DS, tc::make_smem_desc(st + OFF_B + ks * 2048, TILE_16K, 1024, tc::SWZ_128B),
-                               tc::make_smem_desc(sbase + OFF_XT + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_nn,
-                               ks != 0);
-                tc::mma_commit(bars + B_DS);
-                if (c + 1 < nchunks) {
-                    const int nb = (c + 1) & 1;
-                    if (!tc::mbar_wait(bars + B_FULL0 + nb, ((c + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-                    if (c >= 1 && !tc::mbar_wait(bars + B_CBF0 + nb, ((c - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                        for (int ks = 0; ks < 8; ++ks)  // Y_inter_c = C S_{c-1}^T
+                            tc::mma_ss(tmem + TM_YO + (uint32_t)s * 64, tc::desc_kmajor_sw128(ct + (ks >> 2) * TILE_16K, (ks & 3) * 16),
+                                       tc::make_smem_desc(sbase + OFF_SB + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_kn, ks != 0);
+                    }
+                    if (!tc::mbar_wait(bars + B_XSF, c & 1, abort_flag)) { ok = false; break; }
+                    if (c > 0 && !tc::mbar_wait(bars + B_DSE, (c - 1) & 1, abort_flag)) { ok = false; break; }
                     tc::tc_fence_after();
-                    issue_cb(c + 1);
-                }
-                if (!tc::mbar_wait(bars + B_W, c & 1, abort_flag)) { ok = false; break; }
-                tc::tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)          // Y_intra = W X
-                    tc::mma_ss(tmem + TM_YI, tc::desc_kmajor_sw128(sbase + OFF_W + (ks >> 2) * TILE_16K, (ks & 3) * 16),
-                               tc::make_smem_desc(st + OFF_X + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_kn, ks != 0);
-                tc::mma_commit(bars + B_Y);
-                tc::mma_commit(bars + B_EMPTY0 + (c & 1));
+                    for (int ks = 0; ks < 8; ++ks)      // dS_c^T = B^T Xs
+                        tc::mma_ss(tmem + TM_DS, tc::make_smem_desc(bt + ks * 2048, TILE_16K, 1024, tc::SWZ_128B),
+                                   tc::make_smem_desc(sbase + OFF_XS + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_nn, ks != 0);
+                    tc::mma_commit(bars + B_DSF);
+                    tc::mma_commit(bars + B_BCE + s);
+                }
+                if (c >= 1) {
+                    const int cp = c - 1, sp = cp & 1;
+                    if (!tc::mbar_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint32_t xt = sbase + OFF_X + (uint32_t)(cp % X_SLOTS) * TILE_16K;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)      // Y_intra_{c-1} = W X
+                        tc::mma_ts(tmem + TM_YI, tmem + TM_CB + (uint32_t)sp * 128 + (uint32_t)ks * 8,
+                                   tc::make_smem_desc(xt + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_kn, ks != 0);
+                    tc::mma_commit(bars + B_YF);
+                    tc::mma_commit(bars + B_XE + cp % X_SLOTS);
+                }
             }
             if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         }
-    } else {
-        // ------------------------------------------------------------------ compute warps
-        const int tid = threadIdx.x;                  // 0..255
-        const int quad = warp & 3, hf = warp >> 2;
-        const int row = quad * 32 + lane;             // token (W, Y) or state index n (state)
-        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const float Ah = A[h];
+    } else if (warp == 14) {
+        // ------------------------------------------------------------------ decay vectors
+        const float Ah2 = A[h] * LOG2E;
         const float *dtb = dt + (size_t)b * Tlen * H + h;
-        __nv_bfloat16 *yb = y + ((size_t)b * Tlen * H + h) * P;
-        float S[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) S[i] = 0.f;
         bool ok = true;
         for (int c = 0; c < nchunks; ++c) {
-            const int s = c & 1, t0 = c * Q;
-            uint8_t *st = smem + (size_t)s * STAGE_BYTES;
-            // ---- 1. cumulative log-decay and factors
-            float a_incl = 0.f, d_me = 0.f;
-            if (tid < 128) {
-                d_me = (t0 + tid < Tlen) ? dtb[(size_t)(t0 + tid) * H] : 0.f;
-                a_incl = d_me * Ah;
+            const int d = c & (DEC_DEPTH - 1), t0 = c * Q;
+            if (!tc::mbar_wait(bars + B_DECE + d, ((c >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
+            float dv[4], l[4];
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const float v = __shfl_up_sync(0xffffffffu, a_incl, o);
-                    if (lane >= o) a_incl += v;
-                }
-                if (lane == 31) wsum[warp] = a_incl;
+            for (int i = 0; i < 4; ++i) {
+                const int t = t0 + 4 * lane + i;
+                dv[i] = t < Tlen ? __ldg(dtb + (size_t)t * H) : 0.f;
             }
-            ok = compute_sync_and(ok);       // uniform: a failed wait anywhere ends the loop for all warps
-            if (!ok) break;
-            if (tid < 128) {
-                float l_start = 0.f;
-                for (int w = 0; w < warp; ++w) l_start += wsum[w];
-                const float l_end_blk = l_start + wsum[warp];
-                const float l_end = wsum[0] + wsum[1] + wsum[2] + wsum[3];
-                const float l = l_start + a_incl;
-                ls[tid] = l;
-                dts[tid] = d_me;
-                colf[tid] = __expf(l_end_blk - l) * d_me;
-                xw[tid] = __expf(l_end - l) * d_me;
-                if (lane == 0) wsum[4 + warp] = l_start;
-                if (lane < 4 && lane < warp) {            // blk[bt = warp][bj = lane], bj < bt
-                    float l_end_bj = 0.f;
-                    for (int w = 0; w <= lane; ++w) l_end_bj += wsum[w];
-                    blk[warp * 4 + lane] = __expf(l_start - l_end_bj);
-                }
+            l[0] = dv[0] * Ah2;
+#pragma unroll
+            for (int i = 1; i < 4; ++i) l[i] = fmaf(dv[i], Ah2, l[i - 1]);
+            float incl = l[3];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
             }
-            ok &= tc::mbar_wait(bars + B_FULL0 + s, (c >> 1) & 1, abort_flag);
-            compute_sync();
-            // ---- 2. Xs = exp(l_end - l_j) dt_j x_j  (same swizzled layout as the X tile)
+            const float excl = incl - l[3];
+            const float l_start = __shfl_sync(0xffffffffu, excl, lane & ~7);     // start of this 32-token block
+            const float l_endb = __shfl_sync(0xffffffffu, incl, lane | 7);       // end of this 32-token block
+            const float l_end = __shfl_sync(0xffffffffu, incl, 31);
+            // blk[bt][bj] = exp(l_start(bt) - l_endblock(bj)), bj < bt; lanes 0..15 hold (bt, bj) = (lane/4, lane%4)
+            const float bs = __shfl_sync(0xffffffffu, excl, (lane >> 2 & 3) * 8);
+            const float be = __shfl_sync(0xffffffffu, incl, (lane & 3) * 8 + 7);
+            float *dec = decs + d * DEC_FLOATS;
+            float4 v_ls, v_colf, v_xw, v_rowf, v_erow;
+            float *p_ls = &v_ls.x, *p_colf = &v_colf.x, *p_xw = &v_xw.x, *p_rowf = &v_rowf.x, *p_erow = &v_erow.x;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float li = excl + l[i];
+                p_ls[i] = li;
+                p_colf[i] = tc::ex2(l_endb - li) * dv[i];
+                p_xw[i] = tc::ex2(l_end - li) * dv[i];
+                p_rowf[i] = tc::ex2(li - l_start);
+                p_erow[i] = tc::ex2(li);
+            }
+            *(float4 *)(dec + D_LS + 4 * lane) = v_ls;
+            *(float4 *)(dec + D_DT + 4 * lane) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+            *(float4 *)(dec + D_COLF + 4 * lane) = v_colf;
+            *(float4 *)(dec + D_XW + 4 * lane) = v_xw;
+            *(float4 *)(dec + D_ROWF + 4 * lane) = v_rowf;
+            *(float4 *)(dec + D_EROW + 4 * lane) = v_erow;
+            if (lane < 16) dec[D_BLK + lane] = ((lane & 3) < (lane >> 2)) ? tc::ex2(bs - be) : 0.f;
+            if (lane == 0) dec[D_EEND] = tc::ex2(l_end);
+            warp_arrive(bars + B_DECF + d, lane);
+        }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+    } else if (warp < 4) {
+        // ------------------------------------------------------------------ W_c = CB_c o decay
+        const int quad = warp, row = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        bool ok = true;
+        for (int c = 0; c < nchunks; ++c) {
+            const int d = c & (DEC_DEPTH - 1), s = c & 1;
+            const float *dec = decs + d * DEC_FLOATS;
+            if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
+            const float l_t = dec[D_LS + row], rf = dec[D_ROWF + row];
+            if (!tc::mbar_wait(bars + B_CBF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after();
+            const uint32_t tW = tmem + lane_base + TM_CB + (uint32_t)s * 128;
+#pragma unroll
+            for (int bj = 0; bj < 4; ++bj) {
+                uint32_t packed[16];
+                if (bj > quad) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) packed[i] = 0u;
+                } else {
+                    uint32_t v[32];
+                    tc::tmem_ld32(tW + (uint32_t)(bj * 32), v);
+                    tc::tmem_ld_wait();
+                    if (bj == quad) {
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const float4 lj = *(const float4 *)(dec + D_LS + bj * 32 + 4 * i4);
+                            const float4 dj = *(const float4 *)(dec + D_DT + bj * 32 + 4 * i4);
+                            const int j0 = bj * 32 + 4 * i4;
+                            const float f0 = (j0 <= row) ? tc::ex2(l_t - lj.x) * dj.x : 0.f;
+                            const float f1 = (j0 + 1 <= row) ? tc::ex2(l_t - lj.y) * dj.y : 0.f;
+                            const float f2 = (j0 + 2 <= row) ? tc::ex2(l_t - lj.z) * dj.z : 0.f;
+                            const float f3 = (j0 + 3 <= row) ? tc::ex2(l_t - lj.w) * dj.w : 0.f;
+                            packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * f0, __uint_as_float(v[4 * i4 + 1]) * f1);
+                            packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * f2, __uint_as_float(v[4 * i4 + 3]) * f3);
+                        }
+                    } else {
+                        const float f = rf * dec[D_BLK + quad * 4 + bj];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const float4 cf = *(const float4 *)(dec + D_COLF + bj * 32 + 4 * i4);
+                            packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * (f * cf.x), __uint_as_float(v[4 * i4 + 1]) * (f * cf.y));
+                            packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * (f * cf.z), __uint_as_float(v[4 * i4 + 3]) * (f * cf.w));
+                        }
+                    }
+                }
+                // bf16 pairs of columns [32 bj, 32 bj + 32) go to 32-bit columns [16 bj, 16 bj + 16): only over
+                // accumulator columns this thread has already read
+                tc::tmem_st16(tW + (uint32_t)(bj * 16), packed);
+            }
+            tc::tmem_st_wait();
+            tc::tc_fence_before();
+            warp_arrive(bars + B_WF + s, lane);
+            if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
+        }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+    } else if (warp < 8) {
+        // ------------------------------------------------------------------ Xs_c and the state update
+        const int quad = warp & 3, row = quad * 32 + lane;        // row = state index n
+        const int tid_g = threadIdx.x - 128;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        float S[64];
+#pragma unroll
+        for (int i = 0; i < 64; ++i) S[i] = 0.f;
+        bool ok = true;
+        for (int c = 0; c < nchunks; ++c) {
+            const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
+            const float *dec = decs + d * DEC_FLOATS;
+            if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
+            if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
+            // Xs = exp(l_end - l_j) dt_j x_j, same swizzled layout as the X tile (the Xs buffer is free:
+            // this warp has already seen dS_{c-1} complete)
             {
-                const uint4 *src = (const uint4 *)(st + OFF_X);
-                uint4 *dst = (uint4 *)(smem + OFF_XT);
+                const uint4 *src = (const uint4 *)(smem + OFF_X + sx * TILE_16K);
+                uint4 *dst = (uint4 *)(smem + OFF_XS);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int u = tid + 256 * i;
-                    const float sc = xw[u >> 3];
-                    uint4 v = src[u];
+                for (int i = 0; i < 8; ++i) {
+                    const int u = tid_g + 128 * i;
+                    const float sc = dec[D_XW + (u >> 3)];
+                    const uint4 v = src[u];
                     uint32_t wv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
@@ -247,132 +323,87 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 }
             }
             tc::fence_proxy_async();
-            warp_arrive(bars + B_XT, lane);
-            // ---- 3. W = CB o decay (bf16, K-major swizzled tile; this warp: rows of block `quad`, 64 columns)
-            ok &= tc::mbar_wait(bars + B_CBR0 + s, (c >> 1) & 1, abort_flag);
+            __syncwarp();
+            if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
+            const float eend = dec[D_EEND];
+            if (!tc::mbar_wait(bars + B_DSF, c & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
-            {
-                const float l_t = ls[row], rf = __expf(l_t - wsum[4 + quad]);
-                uint8_t *wrow = smem + OFF_W + hf * TILE_16K + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
-                for (int cg = 0; cg < 2; ++cg) {
-                    const int bj = 2 * hf + cg;
-                    uint32_t packed[16];
-                    if (bj > quad) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) packed[i] = 0u;
-                    } else {
-                        uint32_t v[32];
-                        tc::tmem_ld32(tmem + lane_base + TM_CB + (uint32_t)s * 128 + (uint32_t)(bj * 32), v);
-                        tc::tmem_ld_wait();
-                        if (bj == quad) {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int j0 = bj * 32 + 2 * i, j1 = j0 + 1;
-                                const float f0 = (j0 <= row) ? __expf(l_t - ls[j0]) * dts[j0] : 0.f;
-                                const float f1 = (j1 <= row) ? __expf(l_t - ls[j1]) * dts[j1] : 0.f;
-                                packed[i] = tc::pack_bf16x2(__uint_as_float(v[2 * i]) * f0, __uint_as_float(v[2 * i + 1]) * f1);
-                            }
-                        } else {
-                            const float f = rf * blk[quad * 4 + bj];
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int j0 = bj * 32 + 2 * i;
-                                packed[i] = tc::pack_bf16x2(__uint_as_float(v[2 * i]) * (f * colf[j0]),
-                                                            __uint_as_float(v[2 * i + 1]) * (f * colf[j0 + 1]));
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int ci = 0; ci < 4; ++ci) {
-                        const int chunk = cg * 4 + ci;
-                        *(uint4 *)(wrow + ((chunk ^ (row & 7)) << 4)) =
-                            make_uint4(packed[4 * ci], packed[4 * ci + 1], packed[4 * ci + 2], packed[4 * ci + 3]);
-                    }
-                }
-            }
-            tc::tc_fence_before();
-            tc::fence_proxy_async();
-            warp_arrive(bars + B_W, lane);
-            warp_arrive(bars + B_CBF0 + s, lane);
-            // ---- 4. state: S^T <- exp(l_end) S^T + dS^T ; bf16 copy for the next chunk's Y_inter
-            ok &= tc::mbar_wait(bars + B_DS, c & 1, abort_flag);
-            tc::tc_fence_after();
-            {
+            for (int hf = 0; hf < 2; ++hf) {
                 uint32_t v[32];
                 tc::tmem_ld32(tmem + lane_base + TM_DS + (uint32_t)(hf * 32), v);
                 tc::tmem_ld_wait();
-                const float eend = __expf(ls[127]);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) S[i] = fmaf(eend, S[i], __uint_as_float(v[i]));
+                for (int i = 0; i < 32; ++i) S[hf * 32 + i] = fmaf(eend, S[hf * 32 + i], __uint_as_float(v[i]));
+            }
+            tc::tc_fence_before();
+            warp_arrive(bars + B_DSE, lane);
+            // bf16 copy of S^T for the next chunk's Y_inter (dS_c complete implies Y_inter_c complete, so the
+            // previous copy is no longer being read)
+            {
                 uint8_t *srow = smem + OFF_SB + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
-                for (int ci = 0; ci < 4; ++ci) {
-                    const int chunk = hf * 4 + ci;
-                    *(uint4 *)(srow + ((chunk ^ (row & 7)) << 4)) =
+                for (int ci = 0; ci < 8; ++ci)
+                    *(uint4 *)(srow + ((ci ^ (row & 7)) << 4)) =
                         make_uint4(tc::pack_bf16x2(S[8 * ci], S[8 * ci + 1]), tc::pack_bf16x2(S[8 * ci + 2], S[8 * ci + 3]),
                                    tc::pack_bf16x2(S[8 * ci + 4], S[8 * ci + 5]), tc::pack_bf16x2(S[8 * ci + 6], S[8 * ci + 7]));
-                }
             }
-            tc::tc_fence_before();
             tc::fence_proxy_async();
-            warp_arrive(bars + B_S, lane);
-            // ---- 5. epilogue: y_t = Y_intra + exp(l_t) Y_inter
-            ok &= tc::mbar_wait(bars + B_Y, c & 1, abort_flag);
-            tc::tc_fence_after();
-            {
-                uint32_t yi[32];
-                tc::tmem_ld32(tmem + lane_base + TM_YI + (uint32_t)(hf * 32), yi);
-                float out[32];
-                if (c > 0) {
-                    uint32_t yo[32];
-                    tc::tmem_ld32(tmem + lane_base + TM_YO + (uint32_t)(hf * 32), yo);
-                    tc::tmem_ld_wait();
-                    const float er = __expf(ls[row]);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) out[i] = fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yi[i]));
-                } else {
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) out[i] = __uint_as_float(yi[i]);
-                }
-                if (t0 + row < Tlen) {
-                    uint4 *dst = (uint4 *)(yb + (size_t)(t0 + row) * H * P + hf * 32);
-#pragma unroll
-                    for (int ci = 0; ci < 4; ++ci)
-                        dst[ci] = make_uint4(tc::pack_bf16x2(out[8 * ci], out[8 * ci + 1]), tc::pack_bf16x2(out[8 * ci + 2], out[8 * ci + 3]),
-                                             tc::pack_bf16x2(out[8 * ci + 4], out[8 * ci + 5]), tc::pack_bf16x2(out[8 * ci + 6], out[8 * ci + 7]));
-                }
-            }
-            tc::tc_fence_before();
-            warp_arrive(bars + B_YF, lane);
+            __syncwarp();
+            if (lane == 0) { tc::mbar_arrive(bars + B_SF); tc::mbar_arrive(bars + B_DECE + d); }
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         if (ok && final_state) {
             float *fs = final_state + ((size_t)b * H + h) * P * NS;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) fs[(size_t)(hf * 32 + i) * NS + row] = S[i];
+            for (int i = 0; i < 64; ++i) fs[(size_t)i * NS + row] = S[i];
         }
+    } else if (warp < 12) {
+        // ------------------------------------------------------------------ epilogue: y_t = Y_intra + exp(l_t) Y_inter
+        const int quad = warp & 3, row = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        __nv_bfloat16 *yb = y + ((size_t)b * Tlen * H + h) * P;
+        bool ok = true;
+        for (int c = 0; c < nchunks; ++c) {
+            const int d = c & (DEC_DEPTH - 1), t0 = c * Q;
+            if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
+            const float er = decs[d * DEC_FLOATS + D_EROW + row];
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
+            if (!tc::mbar_wait(bars + B_YF, c & 1, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after();
+            float out[64];
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t yi[32];
+                tc::tmem_ld32(tmem + lane_base + TM_YI + (uint32_t)(hf * 32), yi);
+                if (c > 0) {
+                    uint32_t yo[32];
+                    tc::tmem_ld32(tmem + lane_base + TM_YO + (uint32_t)((c & 1) * 64 + hf * 32), yo);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) out[hf * 32 + i] = fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yi[i]));
+                } else {
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) out[hf * 32 + i] = __uint_as_float(yi[i]);
+                }
+            }
+            tc::tc_fence_before();
+            warp_arrive(bars + B_YE, lane);
+            if (t0 + row < Tlen) {
+                uint4 *dst = (uint4 *)(yb + (size_t)(t0 + row) * H * P);
+#pragma unroll
+                for (int ci = 0; ci < 8; ++ci)
+                    dst[ci] = make_uint4(tc::pack_bf16x2(out[8 * ci], out[8 * ci + 1]), tc::pack_bf16x2(out[8 * ci + 2], out[8 * ci + 3]),
+                                         tc::pack_bf16x2(out[8 * ci + 4], out[8 * ci + 5]), tc::pack_bf16x2(out[8 * ci + 6], out[8 * ci + 7]));
+            }
+        }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 9) { tc::tc_fence_after(); tc::tmem_dealloc(tmem, 512); }
-}
-
-int make_tmap_3d(str_ctx *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t T, uint64_t Bz) {
-    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-    if (!ctx->encode_tiled) return STR_ERR_CUDA;
-    cuuint64_t dims[3] = {inner, T, Bz};
-    cuuint64_t strides[2] = {inner * 2, inner * T * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)Q, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = ((encode_fn)ctx->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims,
-                                                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? STR_OK : STR_ERR_CUDA;
+    if (warp == 13) { tc::tc_fence_after(); tc::tmem_dealloc(tmem, 512); }
 }
 
 }  // namespace
@@ -387,9 +418,9 @@ int str_ssd_tc(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float 
                const void *C, void *y, float *final_state, cudaStream_t st) {
     if (SMEM_BYTES > (size_t)ctx->max_smem_optin) return STR_ERR_UNSUPPORTED_SHAPE;
     CUtensorMap tx, tb, tcm;
-    int rc = make_tmap_3d(ctx, &tx, x, (uint64_t)s->H * P, (uint64_t)s->T, (uint64_t)s->Bz);
-    if (rc == STR_OK) rc = make_tmap_3d(ctx, &tb, B, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz);
-    if (rc == STR_OK) rc = make_tmap_3d(ctx, &tcm, C, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz);
+    int rc = str_make_tmap_3d_bf16_sw128(ctx, &tx, x, (uint64_t)s->H * P, (uint64_t)s->T, (uint64_t)s->Bz, Q);
+    if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tb, B, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz, Q);
+    if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tcm, C, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz, Q);
     if (rc != STR_OK) return rc;
     static bool attr_set = false;
     if (!attr_set) {
