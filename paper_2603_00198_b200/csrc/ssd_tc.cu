@@ -15,15 +15,21 @@
 // diagonal 32x32 blocks exp(l_t - l_j) is split into three factors, each <= 1 (row part, block-pair
 // scalar, column part); the diagonal blocks take one exponential per element.
 //
-// The chunk loop is software-pipelined across warp roles that only meet at mbarriers, so the only
-// serial chain from chunk to chunk is  dS_c -> state update -> Y_inter_{c+1}:
-//   warps 0-3    W_c from CB_c                       (one thread per token row)
-//   warps 4-7    Xs_c, then the state update         (one thread per state row n)
-//   warps 8-11   epilogue of chunk c                 (one thread per token row)
-//   warp 12      TMA producer: B,C ring of 2, X ring of 3 (128-byte swizzle)
-//   warp 13      MMA issuer; iteration c issues  CB_c, Y_inter_c, dS_c, Y_intra_{c-1}
-//   warp 14      decay vectors of chunk c (cumulative sum, exponentials) into a ring of 4
-// Tensor memory: CB/W 2 x 128 columns | Y_inter 2 x 64 | Y_intra 64 | dS 64.
+// The chunk loop is software-pipelined across warp roles that only meet at mbarriers; the only
+// serial chains from chunk to chunk are  dS_c -> state update -> Y_inter_{c+1}  and
+// dS_c -> Xs_{c+1} -> dS_{c+1}  (single Xs buffer):
+//   warps 0-3, 14, 15  W_c from CB_c (one thread per token row and 64-column half; the upper halves of
+//                      row blocks 0 and 1 are all zero and are written by warps 0 and 1)
+//   warps 4-7          state update (one thread per state row n, 64 fp32 registers of state)
+//   warps 8-11         Xs_{c+1}, then the epilogue of chunk c (one thread per token row)
+//   warp 12            TMA producer (lane 0): B,C ring of 2, X ring of 3 (128-byte swizzle); then, all lanes,
+//                      the decay vectors of the chunk (cumulative sum, exponentials) into a ring of 4
+//   warp 13            MMA issuer; iteration c issues  CB_c, Y_inter_c, dS_c, Y_intra_{c-1}
+// Loops are kept rolled where registers allow: the instruction footprint of all roles together has to
+// stay inside the instruction cache, or every role slows down together.
+// Tensor memory: CB/W 2 x 128 columns | Y_inter 2 x 64 | Y_intra 64 | dS 64.  W's K-slices 0-3 (keys
+// 0-63) sit in columns [0,32) of the CB buffer and K-slices 4-7 in columns [64,96), so each W warp
+// only overwrites accumulator columns that it has read itself.
 // All mbarrier waits are bounded; a give-up records STR_ERR_TIMEOUT and tears the CTA down.
 #include "dispatch.cuh"
 #include "tc_common.cuh"
@@ -47,7 +53,9 @@ enum {
     B_SF, B_YF, B_YE, B_COUNT
 };
 constexpr size_t SMEM_BYTES = (size_t)OFF_BARS + B_COUNT * 8 + 32;
-constexpr int NUM_THREADS = 480;
+constexpr int NUM_WARPS = 16, NUM_THREADS = NUM_WARPS * 32;
+constexpr int W_WARPS = 6;
+constexpr int DEC_READERS = W_WARPS + 4 + 4;              // warps that read a chunk's decay vectors
 constexpr uint32_t TM_CB = 0, TM_YO = 256, TM_YI = 384, TM_DS = 448;
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -55,6 +63,10 @@ __device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane) {
     __syncwarp();
     if (lane == 0) tc::mbar_arrive(bar);
 }
+
+// Descriptor arithmetic: the 14-bit start-address field holds (shared address >> 4); every operand of
+// this kernel lies below 256 KB, so adding a byte offset >> 4 to the descriptor never carries out of it.
+__device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_b,
@@ -79,9 +91,9 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         for (int i = 0; i < X_SLOTS; ++i) { tc::mbar_init(bars + B_XF + i, 1); tc::mbar_init(bars + B_XE + i, 5); }
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(bars + B_BCF + i, 1); tc::mbar_init(bars + B_BCE + i, 1);
-            tc::mbar_init(bars + B_CBF + i, 1); tc::mbar_init(bars + B_WF + i, 4);
+            tc::mbar_init(bars + B_CBF + i, 1); tc::mbar_init(bars + B_WF + i, W_WARPS);
         }
-        for (int i = 0; i < DEC_DEPTH; ++i) { tc::mbar_init(bars + B_DECF + i, 1); tc::mbar_init(bars + B_DECE + i, 12); }
+        for (int i = 0; i < DEC_DEPTH; ++i) { tc::mbar_init(bars + B_DECF + i, 1); tc::mbar_init(bars + B_DECE + i, DEC_READERS); }
         tc::mbar_init(bars + B_XSF, 4); tc::mbar_init(bars + B_DSF, 1); tc::mbar_init(bars + B_DSE, 4);
         tc::mbar_init(bars + B_SF, 4); tc::mbar_init(bars + B_YF, 1); tc::mbar_init(bars + B_YE, 4);
         abort_flag[0] = 0; abort_flag[1] = 0;
@@ -95,107 +107,47 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 12) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            bool ok = true;
-            int n_bc = 0, n_x = 0;
-            for (int c = 0; c < nchunks; ++c) {
-                const int t0 = c * Q, s = c & 1, sx = c % X_SLOTS;
-                if (!tc::mbar_wait(bars + B_BCE + s, ((c >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                uint64_t *fb = bars + B_BCF + s;
-                tc::mbar_arrive_expect_tx(fb, 4 * TILE_16K);
-                tc::tma_load_3d(smem + OFF_B + (s * 2) * TILE_16K, &tmap_b, fb, g * NS, t0, b);
-                tc::tma_load_3d(smem + OFF_B + (s * 2 + 1) * TILE_16K, &tmap_b, fb, g * NS + 64, t0, b);
-                tc::tma_load_3d(smem + OFF_C + (s * 2) * TILE_16K, &tmap_c, fb, g * NS, t0, b);
-                tc::tma_load_3d(smem + OFF_C + (s * 2 + 1) * TILE_16K, &tmap_c, fb, g * NS + 64, t0, b);
-                ++n_bc;
-                if (!tc::mbar_wait(bars + B_XE + sx, ((c / X_SLOTS) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                tc::mbar_arrive_expect_tx(bars + B_XF + sx, TILE_16K);
-                tc::tma_load_3d(smem + OFF_X + sx * TILE_16K, &tmap_x, bars + B_XF + sx, h * P, t0, b);
-                ++n_x;
-            }
-            if (!ok) {
-                atomicCAS(status, 0, STR_ERR_TIMEOUT);
-                for (int back = 1; back <= 2 && back <= n_bc; ++back) {      // let issued copies land
-                    const int j = n_bc - back;
-                    tc::mbar_wait(bars + B_BCF + (j & 1), (j >> 1) & 1, abort_flag + 1);
-                }
-                for (int back = 1; back <= X_SLOTS && back <= n_x; ++back) {
-                    const int j = n_x - back;
-                    tc::mbar_wait(bars + B_XF + j % X_SLOTS, (j / X_SLOTS) & 1, abort_flag + 1);
-                }
-            }
-        }
-    } else if (warp == 13) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t id_cb = tc::make_idesc_bf16(128, 128, 0, 0);   // C (K-major) x B (K-major)
-            const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major / tensor-memory A x MN-major B
-            const uint32_t id_nn = tc::make_idesc_bf16(128, 64, 1, 1);    // MN-major A x MN-major B
-            const uint32_t sbase = tc::smem_u32(smem);
-            bool ok = true;
-            for (int c = 0; c <= nchunks && ok; ++c) {
-                const int s = c & 1;
-                if (c >= 2) {        // the epilogue has read the Y accumulators of chunk c-2
-                    if (!tc::mbar_wait(bars + B_YE, (c - 2) & 1, abort_flag)) { ok = false; break; }
-                }
-                if (c < nchunks) {
-                    const uint32_t bt = sbase + OFF_B + (uint32_t)s * 2 * TILE_16K;
-                    const uint32_t ct = sbase + OFF_C + (uint32_t)s * 2 * TILE_16K;
-                    if (!tc::mbar_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)      // CB_c = C B^T
-                        tc::mma_ss(tmem + TM_CB + (uint32_t)s * 128, tc::desc_kmajor_sw128(ct + (ks >> 2) * TILE_16K, (ks & 3) * 16),
-                                   tc::desc_kmajor_sw128(bt + (ks >> 2) * TILE_16K, (ks & 3) * 16), id_cb, ks != 0);
-                    tc::mma_commit(bars + B_CBF + s);
-                    if (c > 0) {
-                        if (!tc::mbar_wait(bars + B_SF, (c - 1) & 1, abort_flag)) { ok = false; break; }
-                        tc::tc_fence_after();
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)  // Y_inter_c = C S_{c-1}^T
-                            tc::mma_ss(tmem + TM_YO + (uint32_t)s * 64, tc::desc_kmajor_sw128(ct + (ks >> 2) * TILE_16K, (ks & 3) * 16),
-                                       tc::make_smem_desc(sbase + OFF_SB + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_kn, ks != 0);
-                    }
-                    if (!tc::mbar_wait(bars + B_XSF, c & 1, abort_flag)) { ok = false; break; }
-                    if (c > 0 && !tc::mbar_wait(bars + B_DSE, (c - 1) & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)      // dS_c^T = B^T Xs
-                        tc::mma_ss(tmem + TM_DS, tc::make_smem_desc(bt + ks * 2048, TILE_16K, 1024, tc::SWZ_128B),
-                                   tc::make_smem_desc(sbase + OFF_XS + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_nn, ks != 0);
-                    tc::mma_commit(bars + B_DSF);
-                    tc::mma_commit(bars + B_BCE + s);
-                }
-                if (c >= 1) {
-                    const int cp = c - 1, sp = cp & 1;
-                    if (!tc::mbar_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-                    const uint32_t xt = sbase + OFF_X + (uint32_t)(cp % X_SLOTS) * TILE_16K;
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)      // Y_intra_{c-1} = W X
-                        tc::mma_ts(tmem + TM_YI, tmem + TM_CB + (uint32_t)sp * 128 + (uint32_t)ks * 8,
-                                   tc::make_smem_desc(xt + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_kn, ks != 0);
-                    tc::mma_commit(bars + B_YF);
-                    tc::mma_commit(bars + B_XE + cp % X_SLOTS);
-                }
-            }
-            if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
-        }
-    } else if (warp == 14) {
-        // ------------------------------------------------------------------ decay vectors
+        // ------------------------------------------------------------------ TMA producer + decay vectors
         const float Ah2 = A[h] * LOG2E;
         const float *dtb = dt + (size_t)b * Tlen * H + h;
         bool ok = true;
-        for (int c = 0; c < nchunks; ++c) {
-            const int d = c & (DEC_DEPTH - 1), t0 = c * Q;
-            if (!tc::mbar_wait(bars + B_DECE + d, ((c >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
-            float dv[4], l[4];
+        int n_bc = 0, n_x = 0;
+        float dv[4], dn[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int t = t0 + 4 * lane + i;
-                dv[i] = t < Tlen ? __ldg(dtb + (size_t)t * H) : 0.f;
+        for (int i = 0; i < 4; ++i) dn[i] = (4 * lane + i < Tlen) ? __ldg(dtb + (size_t)(4 * lane + i) * H) : 0.f;
+#pragma unroll 1
+        for (int c = 0; c < nchunks; ++c) {
+            const int t0 = c * Q, s = c & 1, sx = c % X_SLOTS, d = c & (DEC_DEPTH - 1);
+            if (lane == 0) {
+                if (tc::mbar_wait(bars + B_BCE + s, ((c >> 1) & 1) ^ 1, abort_flag)) {
+                    uint64_t *fb = bars + B_BCF + s;
+                    tc::mbar_arrive_expect_tx(fb, 4 * TILE_16K);
+                    tc::tma_load_3d(smem + OFF_B + (s * 2) * TILE_16K, &tmap_b, fb, g * NS, t0, b);
+                    tc::tma_load_3d(smem + OFF_B + (s * 2 + 1) * TILE_16K, &tmap_b, fb, g * NS + 64, t0, b);
+                    tc::tma_load_3d(smem + OFF_C + (s * 2) * TILE_16K, &tmap_c, fb, g * NS, t0, b);
+                    tc::tma_load_3d(smem + OFF_C + (s * 2 + 1) * TILE_16K, &tmap_c, fb, g * NS + 64, t0, b);
+                    ++n_bc;
+                    if (tc::mbar_wait(bars + B_XE + sx, ((c / X_SLOTS) & 1) ^ 1, abort_flag)) {
+                        tc::mbar_arrive_expect_tx(bars + B_XF + sx, TILE_16K);
+                        tc::tma_load_3d(smem + OFF_X + sx * TILE_16K, &tmap_x, bars + B_XF + sx, h * P, t0, b);
+                        ++n_x;
+                    } else {
+                        ok = false;
+                    }
+                } else {
+                    ok = false;
+                }
             }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {             // this chunk's dt was fetched one iteration ago
+                dv[i] = dn[i];
+                const int t = (c + 1) * Q + 4 * lane + i;
+                dn[i] = t < Tlen ? __ldg(dtb + (size_t)t * H) : 0.f;
+            }
+            if (!tc::mbar_wait(bars + B_DECE + d, ((c >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
+            float l[4];
             l[0] = dv[0] * Ah2;
 #pragma unroll
             for (int i = 1; i < 4; ++i) l[i] = fmaf(dv[i], Ah2, l[i - 1]);
@@ -210,7 +162,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const float l_endb = __shfl_sync(0xffffffffu, incl, lane | 7);       // end of this 32-token block
             const float l_end = __shfl_sync(0xffffffffu, incl, 31);
             // blk[bt][bj] = exp(l_start(bt) - l_endblock(bj)), bj < bt; lanes 0..15 hold (bt, bj) = (lane/4, lane%4)
-            const float bs = __shfl_sync(0xffffffffu, excl, (lane >> 2 & 3) * 8);
+            const float bs = __shfl_sync(0xffffffffu, excl, ((lane >> 2) & 3) * 8);
             const float be = __shfl_sync(0xffffffffu, incl, (lane & 3) * 8 + 7);
             float *dec = decs + d * DEC_FLOATS;
             float4 v_ls, v_colf, v_xw, v_rowf, v_erow;
@@ -234,12 +186,88 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             if (lane == 0) dec[D_EEND] = tc::ex2(l_end);
             warp_arrive(bars + B_DECF + d, lane);
         }
-        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
-    } else if (warp < 4) {
+        if (!ok && lane == 0) {
+            atomicCAS(status, 0, STR_ERR_TIMEOUT);
+            for (int back = 1; back <= 2 && back <= n_bc; ++back) {      // let issued copies land
+                const int j = n_bc - back;
+                tc::mbar_wait(bars + B_BCF + (j & 1), (j >> 1) & 1, abort_flag + 1);
+            }
+            for (int back = 1; back <= X_SLOTS && back <= n_x; ++back) {
+                const int j = n_x - back;
+                tc::mbar_wait(bars + B_XF + j % X_SLOTS, (j / X_SLOTS) & 1, abort_flag + 1);
+            }
+        }
+    } else if (warp == 13) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t id_cb = tc::make_idesc_bf16(128, 128, 0, 0);   // C (K-major) x B (K-major)
+            const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major / tensor-memory A x MN-major B
+            const uint32_t id_nn = tc::make_idesc_bf16(128, 64, 1, 1);    // MN-major A x MN-major B
+            const uint32_t sbase = tc::smem_u32(smem);
+            // descriptors of the first K-slice of every operand; K-slice ks of a K-major operand sits
+            // (ks / 4) * 16 KB + (ks % 4) * 32 bytes further on, of an MN-major operand ks * 2 KB further on
+            const uint64_t dk_c0 = tc::desc_kmajor_sw128(sbase + OFF_C, 0), dk_b0 = tc::desc_kmajor_sw128(sbase + OFF_B, 0);
+            const uint64_t dm_b0 = tc::make_smem_desc(sbase + OFF_B, TILE_16K, 1024, tc::SWZ_128B);
+            const uint64_t dm_xs = tc::make_smem_desc(sbase + OFF_XS, TILE_16K, 1024, tc::SWZ_128B);
+            const uint64_t dm_sb = tc::make_smem_desc(sbase + OFF_SB, TILE_16K, 1024, tc::SWZ_128B);
+            const uint64_t dm_x0 = tc::make_smem_desc(sbase + OFF_X, TILE_16K, 1024, tc::SWZ_128B);
+            bool ok = true;
+#pragma unroll 1
+            for (int c = 0; c <= nchunks && ok; ++c) {
+                const int s = c & 1;
+                if (c >= 2) {        // the epilogue has read the Y accumulators of chunk c-2
+                    if (!tc::mbar_wait(bars + B_YE, (c - 2) & 1, abort_flag)) { ok = false; break; }
+                }
+                if (c < nchunks) {
+                    const uint64_t dk_c = desc_add(dk_c0, (uint32_t)s * 2 * TILE_16K), dk_b = desc_add(dk_b0, (uint32_t)s * 2 * TILE_16K);
+                    if (!tc::mbar_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)      // CB_c = C B^T
+                        tc::mma_ss(tmem + TM_CB + (uint32_t)s * 128, desc_add(dk_c, (ks >> 2) * TILE_16K + (ks & 3) * 32),
+                                   desc_add(dk_b, (ks >> 2) * TILE_16K + (ks & 3) * 32), id_cb, ks != 0);
+                    tc::mma_commit(bars + B_CBF + s);
+                    if (c > 0) {
+                        if (!tc::mbar_wait(bars + B_SF, (c - 1) & 1, abort_flag)) { ok = false; break; }
+                        tc::tc_fence_after();
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)  // Y_inter_c = C S_{c-1}^T
+                            tc::mma_ss(tmem + TM_YO + (uint32_t)s * 64, desc_add(dk_c, (ks >> 2) * TILE_16K + (ks & 3) * 32),
+                                       desc_add(dm_sb, ks * 2048), id_kn, ks != 0);
+                    }
+                    if (!tc::mbar_wait(bars + B_XSF, c & 1, abort_flag)) { ok = false; break; }
+                    if (c > 0 && !tc::mbar_wait(bars + B_DSE, (c - 1) & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint64_t dm_b = desc_add(dm_b0, (uint32_t)s * 2 * TILE_16K);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)      // dS_c^T = B^T Xs
+                        tc::mma_ss(tmem + TM_DS, desc_add(dm_b, ks * 2048), desc_add(dm_xs, ks * 2048), id_nn, ks != 0);
+                    tc::mma_commit(bars + B_DSF);
+                    tc::mma_commit(bars + B_BCE + s);
+                }
+                if (c >= 1) {
+                    const int cp = c - 1, sp = cp & 1;
+                    if (!tc::mbar_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint64_t dm_x = desc_add(dm_x0, (uint32_t)(cp % X_SLOTS) * TILE_16K);
+                    const uint32_t tW = tmem + TM_CB + (uint32_t)sp * 128;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)      // Y_intra_{c-1} = W X; K-slices 4-7 of W start at column 64
+                        tc::mma_ts(tmem + TM_YI, tW + (uint32_t)((ks >> 2) * 64 + (ks & 3) * 8), desc_add(dm_x, ks * 2048), id_kn,
+                                   ks != 0);
+                    tc::mma_commit(bars + B_YF);
+                    tc::mma_commit(bars + B_XE + cp % X_SLOTS);
+                }
+            }
+            if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+        }
+    } else if (warp < 4 || warp >= 14) {
         // ------------------------------------------------------------------ W_c = CB_c o decay
-        const int quad = warp, row = quad * 32 + lane;
+        const int quad = warp & 3, half = warp >= 14 ? 1 : 0;
+        const int row = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         bool ok = true;
+#pragma unroll 1
         for (int c = 0; c < nchunks; ++c) {
             const int d = c & (DEC_DEPTH - 1), s = c & 1;
             const float *dec = decs + d * DEC_FLOATS;
@@ -247,23 +275,24 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const float l_t = dec[D_LS + row], rf = dec[D_ROWF + row];
             if (!tc::mbar_wait(bars + B_CBF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
-            const uint32_t tW = tmem + lane_base + TM_CB + (uint32_t)s * 128;
-#pragma unroll
-            for (int bj = 0; bj < 4; ++bj) {
-                uint32_t packed[16];
+            const uint32_t tW = tmem + lane_base + TM_CB + (uint32_t)(s * 128 + half * 64);
+#pragma unroll 1
+            for (int k = 0; k < 4; ++k) {             // 16-column pieces of this warp's 64 columns
+                const int col0 = half * 64 + k * 16, bj = col0 >> 5;
+                uint32_t packed[8];
                 if (bj > quad) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) packed[i] = 0u;
+                    for (int i = 0; i < 8; ++i) packed[i] = 0u;
                 } else {
-                    uint32_t v[32];
-                    tc::tmem_ld32(tW + (uint32_t)(bj * 32), v);
+                    uint32_t v[16];
+                    tc::tmem_ld16(tW + (uint32_t)(k * 16), v);
                     tc::tmem_ld_wait();
                     if (bj == quad) {
 #pragma unroll
-                        for (int i4 = 0; i4 < 8; ++i4) {
-                            const float4 lj = *(const float4 *)(dec + D_LS + bj * 32 + 4 * i4);
-                            const float4 dj = *(const float4 *)(dec + D_DT + bj * 32 + 4 * i4);
-                            const int j0 = bj * 32 + 4 * i4;
+                        for (int i4 = 0; i4 < 4; ++i4) {
+                            const float4 lj = *(const float4 *)(dec + D_LS + col0 + 4 * i4);
+                            const float4 dj = *(const float4 *)(dec + D_DT + col0 + 4 * i4);
+                            const int j0 = col0 + 4 * i4;
                             const float f0 = (j0 <= row) ? tc::ex2(l_t - lj.x) * dj.x : 0.f;
                             const float f1 = (j0 + 1 <= row) ? tc::ex2(l_t - lj.y) * dj.y : 0.f;
                             const float f2 = (j0 + 2 <= row) ? tc::ex2(l_t - lj.z) * dj.z : 0.f;
@@ -274,16 +303,23 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     } else {
                         const float f = rf * dec[D_BLK + quad * 4 + bj];
 #pragma unroll
-                        for (int i4 = 0; i4 < 8; ++i4) {
-                            const float4 cf = *(const float4 *)(dec + D_COLF + bj * 32 + 4 * i4);
+                        for (int i4 = 0; i4 < 4; ++i4) {
+                            const float4 cf = *(const float4 *)(dec + D_COLF + col0 + 4 * i4);
                             packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * (f * cf.x), __uint_as_float(v[4 * i4 + 1]) * (f * cf.y));
                             packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * (f * cf.z), __uint_as_float(v[4 * i4 + 3]) * (f * cf.w));
                         }
                     }
                 }
-                // bf16 pairs of columns [32 bj, 32 bj + 32) go to 32-bit columns [16 bj, 16 bj + 16): only over
-                // accumulator columns this thread has already read
-                tc::tmem_st16(tW + (uint32_t)(bj * 16), packed);
+                // the 8 bf16 pairs of piece k go to 32-bit columns [8k, 8k+8) of this half: accumulator columns
+                // of pieces <= k, which this thread has already read
+                tc::tmem_st8(tW + (uint32_t)(k * 8), packed);
+            }
+            if (quad < 2) {                           // columns 64..127 of row blocks 0 and 1 lie above the diagonal
+                uint32_t zero[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) zero[i] = 0u;
+                tc::tmem_st16(tW + 64, zero);
+                tc::tmem_st16(tW + 80, zero);
             }
             tc::tmem_st_wait();
             tc::tc_fence_before();
@@ -292,25 +328,72 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
     } else if (warp < 8) {
-        // ------------------------------------------------------------------ Xs_c and the state update
+        // ------------------------------------------------------------------ state update
         const int quad = warp & 3, row = quad * 32 + lane;        // row = state index n
-        const int tid_g = threadIdx.x - 128;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         float S[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) S[i] = 0.f;
         bool ok = true;
+#pragma unroll 1
         for (int c = 0; c < nchunks; ++c) {
-            const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
-            const float *dec = decs + d * DEC_FLOATS;
+            const int d = c & (DEC_DEPTH - 1);
             if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
-            if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
-            // Xs = exp(l_end - l_j) dt_j x_j, same swizzled layout as the X tile (the Xs buffer is free:
-            // this warp has already seen dS_{c-1} complete)
-            {
+            const float eend = decs[d * DEC_FLOATS + D_EEND];
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
+            if (!tc::mbar_wait(bars + B_DSF, c & 1, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after();
+            uint8_t *srow = smem + OFF_SB + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem + lane_base + TM_DS + (uint32_t)(hf * 32), v);
+                tc::tmem_ld_wait();
+                if (hf == 1) {                        // both halves of dS_c are in registers: the accumulator is free
+                    tc::tc_fence_before();
+                    warp_arrive(bars + B_DSE, lane);
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) S[hf * 32 + i] = fmaf(eend, S[hf * 32 + i], __uint_as_float(v[i]));
+                // bf16 copy of S^T for the next chunk's Y_inter (dS_c complete implies Y_inter_c complete, so
+                // the previous copy is no longer being read)
+#pragma unroll
+                for (int ci = 0; ci < 4; ++ci) {
+                    const int q4 = hf * 4 + ci;
+                    *(uint4 *)(srow + ((q4 ^ (row & 7)) << 4)) =
+                        make_uint4(tc::pack_bf16x2(S[8 * q4], S[8 * q4 + 1]), tc::pack_bf16x2(S[8 * q4 + 2], S[8 * q4 + 3]),
+                                   tc::pack_bf16x2(S[8 * q4 + 4], S[8 * q4 + 5]), tc::pack_bf16x2(S[8 * q4 + 6], S[8 * q4 + 7]));
+                }
+            }
+            tc::fence_proxy_async();
+            warp_arrive(bars + B_SF, lane);
+        }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+        if (ok && final_state) {
+            float *fs = final_state + ((size_t)b * H + h) * P * NS;
+#pragma unroll
+            for (int i = 0; i < 64; ++i) fs[(size_t)i * NS + row] = S[i];
+        }
+    } else if (warp < 12) {
+        // ------------------------------------------------------------------ Xs_{c+1}, then y of chunk c
+        const int quad = warp & 3, row = quad * 32 + lane;
+        const int tid_g = threadIdx.x - 256;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        __nv_bfloat16 *yb = y + ((size_t)b * Tlen * H + h) * P;
+        bool ok = true;
+#pragma unroll 1
+        for (int c = 0; c <= nchunks; ++c) {
+            if (c < nchunks) {
+                // Xs_c = exp(l_end - l_j) dt_j x_j, same swizzled layout as the X tile
+                const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
+                const float *dec = decs + d * DEC_FLOATS;
+                if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
+                if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
+                if (c > 0 && !tc::mbar_wait(bars + B_DSF, (c - 1) & 1, abort_flag)) { ok = false; break; }   // Xs buffer free
                 const uint4 *src = (const uint4 *)(smem + OFF_X + sx * TILE_16K);
                 uint4 *dst = (uint4 *)(smem + OFF_XS);
-#pragma unroll
+#pragma unroll 2
                 for (int i = 0; i < 8; ++i) {
                     const int u = tid_g + 128 * i;
                     const float sc = dec[D_XW + (u >> 3)];
@@ -321,82 +404,41 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         wv[j] = tc::pack_bf16x2(__uint_as_float(wv[j] << 16) * sc, __uint_as_float(wv[j] & 0xFFFF0000u) * sc);
                     dst[u] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
                 }
+                tc::fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
             }
-            tc::fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
-            const float eend = dec[D_EEND];
-            if (!tc::mbar_wait(bars + B_DSF, c & 1, abort_flag)) { ok = false; break; }
-            tc::tc_fence_after();
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                uint32_t v[32];
-                tc::tmem_ld32(tmem + lane_base + TM_DS + (uint32_t)(hf * 32), v);
-                tc::tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) S[hf * 32 + i] = fmaf(eend, S[hf * 32 + i], __uint_as_float(v[i]));
-            }
-            tc::tc_fence_before();
-            warp_arrive(bars + B_DSE, lane);
-            // bf16 copy of S^T for the next chunk's Y_inter (dS_c complete implies Y_inter_c complete, so the
-            // previous copy is no longer being read)
-            {
-                uint8_t *srow = smem + OFF_SB + (row >> 3) * 1024 + (row & 7) * 128;
-#pragma unroll
-                for (int ci = 0; ci < 8; ++ci)
-                    *(uint4 *)(srow + ((ci ^ (row & 7)) << 4)) =
-                        make_uint4(tc::pack_bf16x2(S[8 * ci], S[8 * ci + 1]), tc::pack_bf16x2(S[8 * ci + 2], S[8 * ci + 3]),
-                                   tc::pack_bf16x2(S[8 * ci + 4], S[8 * ci + 5]), tc::pack_bf16x2(S[8 * ci + 6], S[8 * ci + 7]));
-            }
-            tc::fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) { tc::mbar_arrive(bars + B_SF); tc::mbar_arrive(bars + B_DECE + d); }
-        }
-        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
-        if (ok && final_state) {
-            float *fs = final_state + ((size_t)b * H + h) * P * NS;
-#pragma unroll
-            for (int i = 0; i < 64; ++i) fs[(size_t)i * NS + row] = S[i];
-        }
-    } else if (warp < 12) {
-        // ------------------------------------------------------------------ epilogue: y_t = Y_intra + exp(l_t) Y_inter
-        const int quad = warp & 3, row = quad * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        __nv_bfloat16 *yb = y + ((size_t)b * Tlen * H + h) * P;
-        bool ok = true;
-        for (int c = 0; c < nchunks; ++c) {
-            const int d = c & (DEC_DEPTH - 1), t0 = c * Q;
-            if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
-            const float er = decs[d * DEC_FLOATS + D_EROW + row];
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
-            if (!tc::mbar_wait(bars + B_YF, c & 1, abort_flag)) { ok = false; break; }
-            tc::tc_fence_after();
-            float out[64];
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                uint32_t yi[32];
-                tc::tmem_ld32(tmem + lane_base + TM_YI + (uint32_t)(hf * 32), yi);
-                if (c > 0) {
-                    uint32_t yo[32];
-                    tc::tmem_ld32(tmem + lane_base + TM_YO + (uint32_t)((c & 1) * 64 + hf * 32), yo);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) out[hf * 32 + i] = fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yi[i]));
-                } else {
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) out[hf * 32 + i] = __uint_as_float(yi[i]);
-                }
-            }
-            tc::tc_fence_before();
-            warp_arrive(bars + B_YE, lane);
-            if (t0 + row < Tlen) {
+            if (c >= 1) {
+                const int cp = c - 1, d = cp & (DEC_DEPTH - 1), t0 = cp * Q;
+                const float er = decs[d * DEC_FLOATS + D_EROW + row];      // DECF of chunk cp was seen one iteration ago
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
+                if (!tc::mbar_wait(bars + B_YF, cp & 1, abort_flag)) { ok = false; break; }
+                tc::tc_fence_after();
                 uint4 *dst = (uint4 *)(yb + (size_t)(t0 + row) * H * P);
 #pragma unroll
-                for (int ci = 0; ci < 8; ++ci)
-                    dst[ci] = make_uint4(tc::pack_bf16x2(out[8 * ci], out[8 * ci + 1]), tc::pack_bf16x2(out[8 * ci + 2], out[8 * ci + 3]),
-                                         tc::pack_bf16x2(out[8 * ci + 4], out[8 * ci + 5]), tc::pack_bf16x2(out[8 * ci + 6], out[8 * ci + 7]));
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t yi[32], yo[32];
+                    tc::tmem_ld32(tmem + lane_base + TM_YI + (uint32_t)(hf * 32), yi);
+                    if (cp > 0) tc::tmem_ld32(tmem + lane_base + TM_YO + (uint32_t)((cp & 1) * 64 + hf * 32), yo);
+                    tc::tmem_ld_wait();
+                    if (hf == 1) {                    // both accumulators are in registers
+                        tc::tc_fence_before();
+                        warp_arrive(bars + B_YE, lane);
+                    }
+                    if (cp > 0) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) yi[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yi[i])));
+                    }
+                    if (t0 + row < Tlen) {
+#pragma unroll
+                        for (int ci = 0; ci < 4; ++ci)
+                            dst[hf * 4 + ci] = make_uint4(tc::pack_bf16x2(__uint_as_float(yi[8 * ci]), __uint_as_float(yi[8 * ci + 1])),
+                                                          tc::pack_bf16x2(__uint_as_float(yi[8 * ci + 2]), __uint_as_float(yi[8 * ci + 3])),
+                                                          tc::pack_bf16x2(__uint_as_float(yi[8 * ci + 4]), __uint_as_float(yi[8 * ci + 5])),
+                                                          tc::pack_bf16x2(__uint_as_float(yi[8 * ci + 6]), __uint_as_float(yi[8 * ci + 7])));
+                    }
+                }
             }
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
