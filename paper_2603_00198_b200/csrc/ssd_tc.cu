@@ -24,7 +24,7 @@
 //   warps 8-11         Xs_{c+1}, then the epilogue of chunk c (one thread per token row)
 //   warp 12            TMA producer (lane 0): B,C ring of 2, X ring of 3 (128-byte swizzle); then, all lanes,
 //                      the decay vectors of the chunk (cumulative sum, exponentials) into a ring of 4
-//   warp 13            MMA issuer; iteration c issues  CB_c, Y_inter_c, dS_c, Y_intra_{c-1}
+//   warp 13            MMA issuer; iteration c issues  CB_c, Y_intra_{c-1}, Y_inter_c, dS_c
 // Loops are kept rolled where registers allow: the instruction footprint of all roles together has to
 // stay inside the instruction cache, or every role slows down together.
 // Tensor memory: CB/W 2 x 128 columns | Y_inter 2 x 64 | Y_intra 64 | dS 64.  W's K-slices 0-3 (keys
@@ -64,9 +64,16 @@ __device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane) {
     if (lane == 0) tc::mbar_arrive(bar);
 }
 
+// Whole-warp wait: every lane polls, then the lanes agree on the outcome.
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile int *abort) {
+    return __all_sync(0xffffffffu, tc::mbar_wait(bar, parity, abort));
+}
+
 // Descriptor arithmetic: the 14-bit start-address field holds (shared address >> 4); every operand of
 // this kernel lies below 256 KB, so adding a byte offset >> 4 to the descriptor never carries out of it.
 __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
+// Byte offset of K-slice ks (16 elements) inside a K-major operand stored as two 64-column, 16 KB halves.
+__device__ __forceinline__ uint32_t kmajor_off(int ks) { return (uint32_t)(ks >> 2) * TILE_16K + (uint32_t)(ks & 3) * 32; }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_b,
@@ -165,23 +172,22 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const float bs = __shfl_sync(0xffffffffu, excl, ((lane >> 2) & 3) * 8);
             const float be = __shfl_sync(0xffffffffu, incl, (lane & 3) * 8 + 7);
             float *dec = decs + d * DEC_FLOATS;
-            float4 v_ls, v_colf, v_xw, v_rowf, v_erow;
-            float *p_ls = &v_ls.x, *p_colf = &v_colf.x, *p_xw = &v_xw.x, *p_rowf = &v_rowf.x, *p_erow = &v_erow.x;
+            float o_ls[4], o_colf[4], o_xw[4], o_rowf[4], o_erow[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const float li = excl + l[i];
-                p_ls[i] = li;
-                p_colf[i] = tc::ex2(l_endb - li) * dv[i];
-                p_xw[i] = tc::ex2(l_end - li) * dv[i];
-                p_rowf[i] = tc::ex2(li - l_start);
-                p_erow[i] = tc::ex2(li);
+                o_ls[i] = li;
+                o_colf[i] = tc::ex2(l_endb - li) * dv[i];
+                o_xw[i] = tc::ex2(l_end - li) * dv[i];
+                o_rowf[i] = tc::ex2(li - l_start);
+                o_erow[i] = tc::ex2(li);
             }
-            *(float4 *)(dec + D_LS + 4 * lane) = v_ls;
+            *(float4 *)(dec + D_LS + 4 * lane) = make_float4(o_ls[0], o_ls[1], o_ls[2], o_ls[3]);
             *(float4 *)(dec + D_DT + 4 * lane) = make_float4(dv[0], dv[1], dv[2], dv[3]);
-            *(float4 *)(dec + D_COLF + 4 * lane) = v_colf;
-            *(float4 *)(dec + D_XW + 4 * lane) = v_xw;
-            *(float4 *)(dec + D_ROWF + 4 * lane) = v_rowf;
-            *(float4 *)(dec + D_EROW + 4 * lane) = v_erow;
+            *(float4 *)(dec + D_COLF + 4 * lane) = make_float4(o_colf[0], o_colf[1], o_colf[2], o_colf[3]);
+            *(float4 *)(dec + D_XW + 4 * lane) = make_float4(o_xw[0], o_xw[1], o_xw[2], o_xw[3]);
+            *(float4 *)(dec + D_ROWF + 4 * lane) = make_float4(o_rowf[0], o_rowf[1], o_rowf[2], o_rowf[3]);
+            *(float4 *)(dec + D_EROW + 4 * lane) = make_float4(o_erow[0], o_erow[1], o_erow[2], o_erow[3]);
             if (lane < 16) dec[D_BLK + lane] = ((lane & 3) < (lane >> 2)) ? tc::ex2(bs - be) : 0.f;
             if (lane == 0) dec[D_EEND] = tc::ex2(l_end);
             warp_arrive(bars + B_DECF + d, lane);
@@ -199,68 +205,84 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         }
     } else if (warp == 13) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t id_cb = tc::make_idesc_bf16(128, 128, 0, 0);   // C (K-major) x B (K-major)
-            const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major / tensor-memory A x MN-major B
-            const uint32_t id_nn = tc::make_idesc_bf16(128, 64, 1, 1);    // MN-major A x MN-major B
-            const uint32_t sbase = tc::smem_u32(smem);
-            // descriptors of the first K-slice of every operand; K-slice ks of a K-major operand sits
-            // (ks / 4) * 16 KB + (ks % 4) * 32 bytes further on, of an MN-major operand ks * 2 KB further on
-            const uint64_t dk_c0 = tc::desc_kmajor_sw128(sbase + OFF_C, 0), dk_b0 = tc::desc_kmajor_sw128(sbase + OFF_B, 0);
-            const uint64_t dm_b0 = tc::make_smem_desc(sbase + OFF_B, TILE_16K, 1024, tc::SWZ_128B);
-            const uint64_t dm_xs = tc::make_smem_desc(sbase + OFF_XS, TILE_16K, 1024, tc::SWZ_128B);
-            const uint64_t dm_sb = tc::make_smem_desc(sbase + OFF_SB, TILE_16K, 1024, tc::SWZ_128B);
-            const uint64_t dm_x0 = tc::make_smem_desc(sbase + OFF_X, TILE_16K, 1024, tc::SWZ_128B);
-            bool ok = true;
+        // The whole warp runs the loop (so descriptors and addresses stay warp-uniform); one elected lane
+        // issues.  Product order per iteration: CB_c, Y_intra_{c-1}, Y_inter_c, dS_c.
+        const uint32_t id_cb = tc::make_idesc_bf16(128, 128, 0, 0);   // C (K-major) x B (K-major)
+        const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major / tensor-memory A x MN-major B
+        const uint32_t id_nn = tc::make_idesc_bf16(128, 64, 1, 1);    // MN-major A x MN-major B
+        const uint32_t sbase = tc::smem_u32(smem);
+        // descriptors of the first K-slice of every operand; K-slice ks of a K-major operand sits
+        // (ks / 4) * 16 KB + (ks % 4) * 32 bytes further on, of an MN-major operand ks * 2 KB further on
+        const uint64_t dk_c0 = tc::desc_kmajor_sw128(sbase + OFF_C, 0), dk_b0 = tc::desc_kmajor_sw128(sbase + OFF_B, 0);
+        const uint64_t dm_b0 = tc::make_smem_desc(sbase + OFF_B, TILE_16K, 1024, tc::SWZ_128B);
+        const uint64_t dm_xs = tc::make_smem_desc(sbase + OFF_XS, TILE_16K, 1024, tc::SWZ_128B);
+        const uint64_t dm_sb = tc::make_smem_desc(sbase + OFF_SB, TILE_16K, 1024, tc::SWZ_128B);
+        const uint64_t dm_x0 = tc::make_smem_desc(sbase + OFF_X, TILE_16K, 1024, tc::SWZ_128B);
+        bool ok = true;
 #pragma unroll 1
-            for (int c = 0; c <= nchunks && ok; ++c) {
-                const int s = c & 1;
-                if (c >= 2) {        // the epilogue has read the Y accumulators of chunk c-2
-                    if (!tc::mbar_wait(bars + B_YE, (c - 2) & 1, abort_flag)) { ok = false; break; }
-                }
-                if (c < nchunks) {
-                    const uint64_t dk_c = desc_add(dk_c0, (uint32_t)s * 2 * TILE_16K), dk_b = desc_add(dk_b0, (uint32_t)s * 2 * TILE_16K);
-                    if (!tc::mbar_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-#pragma unroll
+        for (int c = 0; c <= nchunks && ok; ++c) {
+            const int s = c & 1;
+            const uint64_t dk_c = desc_add(dk_c0, (uint32_t)s * 2 * TILE_16K), dk_b = desc_add(dk_b0, (uint32_t)s * 2 * TILE_16K);
+            if (c < nchunks) {
+                ok = warp_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc::tc_fence_after();
+                if (tc::elect_one()) {
+#pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks)      // CB_c = C B^T
-                        tc::mma_ss(tmem + TM_CB + (uint32_t)s * 128, desc_add(dk_c, (ks >> 2) * TILE_16K + (ks & 3) * 32),
-                                   desc_add(dk_b, (ks >> 2) * TILE_16K + (ks & 3) * 32), id_cb, ks != 0);
+                        tc::mma_ss(tmem + TM_CB + (uint32_t)s * 128, desc_add(dk_c, kmajor_off(ks)), desc_add(dk_b, kmajor_off(ks)),
+                                   id_cb, ks != 0);
                     tc::mma_commit(bars + B_CBF + s);
-                    if (c > 0) {
-                        if (!tc::mbar_wait(bars + B_SF, (c - 1) & 1, abort_flag)) { ok = false; break; }
-                        tc::tc_fence_after();
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)  // Y_inter_c = C S_{c-1}^T
-                            tc::mma_ss(tmem + TM_YO + (uint32_t)s * 64, desc_add(dk_c, (ks >> 2) * TILE_16K + (ks & 3) * 32),
-                                       desc_add(dm_sb, ks * 2048), id_kn, ks != 0);
-                    }
-                    if (!tc::mbar_wait(bars + B_XSF, c & 1, abort_flag)) { ok = false; break; }
-                    if (c > 0 && !tc::mbar_wait(bars + B_DSE, (c - 1) & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-                    const uint64_t dm_b = desc_add(dm_b0, (uint32_t)s * 2 * TILE_16K);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)      // dS_c^T = B^T Xs
-                        tc::mma_ss(tmem + TM_DS, desc_add(dm_b, ks * 2048), desc_add(dm_xs, ks * 2048), id_nn, ks != 0);
-                    tc::mma_commit(bars + B_DSF);
-                    tc::mma_commit(bars + B_BCE + s);
                 }
-                if (c >= 1) {
-                    const int cp = c - 1, sp = cp & 1;
-                    if (!tc::mbar_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-                    const uint64_t dm_x = desc_add(dm_x0, (uint32_t)(cp % X_SLOTS) * TILE_16K);
-                    const uint32_t tW = tmem + TM_CB + (uint32_t)sp * 128;
-#pragma unroll
+                __syncwarp();
+            }
+            if (c >= 1) {
+                const int cp = c - 1, sp = cp & 1;
+                // the epilogue has read the Y accumulators of chunk c-2; W_{c-1} is in tensor memory
+                ok = (c < 2 || warp_wait(bars + B_YE, (c - 2) & 1, abort_flag)) &&
+                     warp_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc::tc_fence_after();
+                const uint64_t dm_x = desc_add(dm_x0, (uint32_t)(cp % X_SLOTS) * TILE_16K);
+                const uint32_t tW = tmem + TM_CB + (uint32_t)sp * 128;
+                if (tc::elect_one()) {
+#pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks)      // Y_intra_{c-1} = W X; K-slices 4-7 of W start at column 64
                         tc::mma_ts(tmem + TM_YI, tW + (uint32_t)((ks >> 2) * 64 + (ks & 3) * 8), desc_add(dm_x, ks * 2048), id_kn,
                                    ks != 0);
                     tc::mma_commit(bars + B_YF);
                     tc::mma_commit(bars + B_XE + cp % X_SLOTS);
                 }
+                __syncwarp();
             }
-            if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+            if (c < nchunks) {
+                if (c > 0) {
+                    ok = warp_wait(bars + B_SF, (c - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    if (tc::elect_one()) {
+#pragma unroll 1
+                        for (int ks = 0; ks < 8; ++ks)  // Y_inter_c = C S_{c-1}^T
+                            tc::mma_ss(tmem + TM_YO + (uint32_t)s * 64, desc_add(dk_c, kmajor_off(ks)), desc_add(dm_sb, ks * 2048), id_kn,
+                                       ks != 0);
+                    }
+                    __syncwarp();
+                }
+                ok = warp_wait(bars + B_XSF, c & 1, abort_flag) && (c == 0 || warp_wait(bars + B_DSE, (c - 1) & 1, abort_flag));
+                if (!ok) break;
+                tc::tc_fence_after();
+                const uint64_t dm_b = desc_add(dm_b0, (uint32_t)s * 2 * TILE_16K);
+                if (tc::elect_one()) {
+#pragma unroll 1
+                    for (int ks = 0; ks < 8; ++ks)      // dS_c^T = B^T Xs
+                        tc::mma_ss(tmem + TM_DS, desc_add(dm_b, ks * 2048), desc_add(dm_xs, ks * 2048), id_nn, ks != 0);
+                    tc::mma_commit(bars + B_DSF);
+                    tc::mma_commit(bars + B_BCE + s);
+                }
+                __syncwarp();
+            }
         }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
     } else if (warp < 4 || warp >= 14) {
         // ------------------------------------------------------------------ W_c = CB_c o decay
         const int quad = warp & 3, half = warp >= 14 ? 1 : 0;
@@ -276,42 +298,43 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             if (!tc::mbar_wait(bars + B_CBF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
             const uint32_t tW = tmem + lane_base + TM_CB + (uint32_t)(s * 128 + half * 64);
+            uint32_t v[16], vn[16];
+            tc::tmem_ld16(tW, vn);
 #pragma unroll 1
             for (int k = 0; k < 4; ++k) {             // 16-column pieces of this warp's 64 columns
                 const int col0 = half * 64 + k * 16, bj = col0 >> 5;
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = vn[i];
+                if (k < 3) tc::tmem_ld16(tW + (uint32_t)((k + 1) * 16), vn);     // in flight while piece k is worked on
                 uint32_t packed[8];
                 if (bj > quad) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) packed[i] = 0u;
+                } else if (bj == quad) {
+#pragma unroll
+                    for (int i4 = 0; i4 < 4; ++i4) {
+                        const float4 lj = *(const float4 *)(dec + D_LS + col0 + 4 * i4);
+                        const float4 dj = *(const float4 *)(dec + D_DT + col0 + 4 * i4);
+                        const int j0 = col0 + 4 * i4;
+                        const float f0 = (j0 <= row) ? tc::ex2(l_t - lj.x) * dj.x : 0.f;
+                        const float f1 = (j0 + 1 <= row) ? tc::ex2(l_t - lj.y) * dj.y : 0.f;
+                        const float f2 = (j0 + 2 <= row) ? tc::ex2(l_t - lj.z) * dj.z : 0.f;
+                        const float f3 = (j0 + 3 <= row) ? tc::ex2(l_t - lj.w) * dj.w : 0.f;
+                        packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * f0, __uint_as_float(v[4 * i4 + 1]) * f1);
+                        packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * f2, __uint_as_float(v[4 * i4 + 3]) * f3);
+                    }
                 } else {
-                    uint32_t v[16];
-                    tc::tmem_ld16(tW + (uint32_t)(k * 16), v);
-                    tc::tmem_ld_wait();
-                    if (bj == quad) {
+                    const float f = rf * dec[D_BLK + quad * 4 + bj];
 #pragma unroll
-                        for (int i4 = 0; i4 < 4; ++i4) {
-                            const float4 lj = *(const float4 *)(dec + D_LS + col0 + 4 * i4);
-                            const float4 dj = *(const float4 *)(dec + D_DT + col0 + 4 * i4);
-                            const int j0 = col0 + 4 * i4;
-                            const float f0 = (j0 <= row) ? tc::ex2(l_t - lj.x) * dj.x : 0.f;
-                            const float f1 = (j0 + 1 <= row) ? tc::ex2(l_t - lj.y) * dj.y : 0.f;
-                            const float f2 = (j0 + 2 <= row) ? tc::ex2(l_t - lj.z) * dj.z : 0.f;
-                            const float f3 = (j0 + 3 <= row) ? tc::ex2(l_t - lj.w) * dj.w : 0.f;
-                            packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * f0, __uint_as_float(v[4 * i4 + 1]) * f1);
-                            packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * f2, __uint_as_float(v[4 * i4 + 3]) * f3);
-                        }
-                    } else {
-                        const float f = rf * dec[D_BLK + quad * 4 + bj];
-#pragma unroll
-                        for (int i4 = 0; i4 < 4; ++i4) {
-                            const float4 cf = *(const float4 *)(dec + D_COLF + col0 + 4 * i4);
-                            packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * (f * cf.x), __uint_as_float(v[4 * i4 + 1]) * (f * cf.y));
-                            packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * (f * cf.z), __uint_as_float(v[4 * i4 + 3]) * (f * cf.w));
-                        }
+                    for (int i4 = 0; i4 < 4; ++i4) {
+                        const float4 cf = *(const float4 *)(dec + D_COLF + col0 + 4 * i4);
+                        packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * (f * cf.x), __uint_as_float(v[4 * i4 + 1]) * (f * cf.y));
+                        packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * (f * cf.z), __uint_as_float(v[4 * i4 + 3]) * (f * cf.w));
                     }
                 }
-                // the 8 bf16 pairs of piece k go to 32-bit columns [8k, 8k+8) of this half: accumulator columns
-                // of pieces <= k, which this thread has already read
+                // the 8 bf16 pairs of piece k go to 32-bit columns [8k, 8k+8) of this half: accumulator columns of
+                // pieces k/2 <= k, in registers by now; the load in flight reads piece k+1, columns >= 16(k+1)
                 tc::tmem_st8(tW + (uint32_t)(k * 8), packed);
             }
             if (quad < 2) {                           // columns 64..127 of row blocks 0 and 1 lie above the diagonal
@@ -393,7 +416,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (c > 0 && !tc::mbar_wait(bars + B_DSF, (c - 1) & 1, abort_flag)) { ok = false; break; }   // Xs buffer free
                 const uint4 *src = (const uint4 *)(smem + OFF_X + sx * TILE_16K);
                 uint4 *dst = (uint4 *)(smem + OFF_XS);
-#pragma unroll 2
+#pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int u = tid_g + 128 * i;
                     const float sc = dec[D_XW + (u >> 3)];
@@ -416,28 +439,40 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (!tc::mbar_wait(bars + B_YF, cp & 1, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after();
                 uint4 *dst = (uint4 *)(yb + (size_t)(t0 + row) * H * P);
+                const bool valid = t0 + row < Tlen;
+                uint32_t ya[32], yb2[32], yo[32];
+                tc::tmem_ld32(tmem + lane_base + TM_YI, ya);
+                if (cp > 0) tc::tmem_ld32(tmem + lane_base + TM_YO + (uint32_t)((cp & 1) * 64), yo);
+                tc::tmem_ld_wait();
+                if (cp > 0) {
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    uint32_t yi[32], yo[32];
-                    tc::tmem_ld32(tmem + lane_base + TM_YI + (uint32_t)(hf * 32), yi);
-                    if (cp > 0) tc::tmem_ld32(tmem + lane_base + TM_YO + (uint32_t)((cp & 1) * 64 + hf * 32), yo);
-                    tc::tmem_ld_wait();
-                    if (hf == 1) {                    // both accumulators are in registers
-                        tc::tc_fence_before();
-                        warp_arrive(bars + B_YE, lane);
-                    }
-                    if (cp > 0) {
+                    for (int i = 0; i < 32; ++i) ya[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(ya[i])));
+                }
+                // second half in flight while the first is narrowed and stored
+                tc::tmem_ld32(tmem + lane_base + TM_YI + 32, yb2);
+                if (cp > 0) tc::tmem_ld32(tmem + lane_base + TM_YO + (uint32_t)((cp & 1) * 64 + 32), yo);
+                if (valid) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) yi[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yi[i])));
-                    }
-                    if (t0 + row < Tlen) {
+                    for (int ci = 0; ci < 4; ++ci)
+                        dst[ci] = make_uint4(tc::pack_bf16x2(__uint_as_float(ya[8 * ci]), __uint_as_float(ya[8 * ci + 1])),
+                                             tc::pack_bf16x2(__uint_as_float(ya[8 * ci + 2]), __uint_as_float(ya[8 * ci + 3])),
+                                             tc::pack_bf16x2(__uint_as_float(ya[8 * ci + 4]), __uint_as_float(ya[8 * ci + 5])),
+                                             tc::pack_bf16x2(__uint_as_float(ya[8 * ci + 6]), __uint_as_float(ya[8 * ci + 7])));
+                }
+                tc::tmem_ld_wait();
+                tc::tc_fence_before();               // both accumulators are in registers
+                warp_arrive(bars + B_YE, lane);
+                if (cp > 0) {
 #pragma unroll
-                        for (int ci = 0; ci < 4; ++ci)
-                            dst[hf * 4 + ci] = make_uint4(tc::pack_bf16x2(__uint_as_float(yi[8 * ci]), __uint_as_float(yi[8 * ci + 1])),
-                                                          tc::pack_bf16x2(__uint_as_float(yi[8 * ci + 2]), __uint_as_float(yi[8 * ci + 3])),
-                                                          tc::pack_bf16x2(__uint_as_float(yi[8 * ci + 4]), __uint_as_float(yi[8 * ci + 5])),
-                                                          tc::pack_bf16x2(__uint_as_float(yi[8 * ci + 6]), __uint_as_float(yi[8 * ci + 7])));
-                    }
+                    for (int i = 0; i < 32; ++i) yb2[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yb2[i])));
+                }
+                if (valid) {
+#pragma unroll
+                    for (int ci = 0; ci < 4; ++ci)
+                        dst[4 + ci] = make_uint4(tc::pack_bf16x2(__uint_as_float(yb2[8 * ci]), __uint_as_float(yb2[8 * ci + 1])),
+                                                 tc::pack_bf16x2(__uint_as_float(yb2[8 * ci + 2]), __uint_as_float(yb2[8 * ci + 3])),
+                                                 tc::pack_bf16x2(__uint_as_float(yb2[8 * ci + 4]), __uint_as_float(yb2[8 * ci + 5])),
+                                                 tc::pack_bf16x2(__uint_as_float(yb2[8 * ci + 6]), __uint_as_float(yb2[8 * ci + 7])));
                 }
             }
         }

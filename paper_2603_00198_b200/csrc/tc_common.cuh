@@ -38,25 +38,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after ~2 s of wall time or as soon as another role raised *abort.
-// Returns false on give-up; the caller records STR_ERR_TIMEOUT and leaves its loops.
-// The polling loop is kept out of line so that the many wait sites of a warp-specialised kernel
-// cost one probe and one call each instead of a copy of the loop (instruction-cache footprint).
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, volatile int *abort) {
-    const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 255u) == 0) {
-            if (*abort) return false;
-            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort = 1; return false; }
-        }
-    }
-}
+// Bounded wait.  Each failed probe parks the warp for a hardware-defined slice of time, so the limit is
+// a count of probes (millions: far beyond any legitimate wait inside these kernels, which last
+// microseconds).  Gives up at once when another role of the CTA has raised *abort.  Returns false on
+// give-up; the caller records STR_ERR_TIMEOUT and leaves its loops.  Kept to a handful of
+// instructions and never unrolled: warp-specialised kernels have dozens of wait sites and their
+// combined footprint has to stay inside the instruction cache.
+constexpr uint32_t WAIT_PROBE_LIMIT = 1u << 22;
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort);
+    uint32_t probes = 0;
+#pragma unroll 1
+    while (!mbar_try_wait(bar, parity)) {
+        if (++probes > WAIT_PROBE_LIMIT || *abort) { *abort = 1; return false; }
+    }
+    return true;
 }
 
 // ---- TMA ------------------------------------------------------------------------------------
@@ -76,6 +71,19 @@ __device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *m
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_u32(smem_dst)), "l"((uint64_t)m), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+
+// One lane of a converged warp (the lowest active one).  Used to predicate single-thread instructions
+// (tcgen05.mma, tcgen05.commit) while the whole warp runs the surrounding loop, so that addresses and
+// descriptors stay warp-uniform values.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
 }
 
 // ---- tcgen05 --------------------------------------------------------------------------------
