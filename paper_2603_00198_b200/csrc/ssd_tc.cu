@@ -34,6 +34,20 @@
 #include "dispatch.cuh"
 #include "tc_common.cuh"
 
+// Optional device-side timeline (compile with -DSTR_SSD_TRACE): lane 0 of selected warps of one CTA
+// stores the SM clock at a few points of chunks 16..31.  Compiled out of the library build.
+#ifdef STR_SSD_TRACE
+__device__ long long g_ssd_trace[8 * 16 * 8];
+#define SSD_TR(role, c, pt)                                                                              \
+    do {                                                                                                 \
+        if (blockIdx.x == 5 && blockIdx.y == 0 && (c) >= 16 && (c) < 32 && lane == 0)                    \
+            g_ssd_trace[((role) * 16 + ((c) - 16)) * 8 + (pt)] = clock64();                              \
+    } while (0)
+extern "C" int str_ssd_trace_fetch(long long *host) { return (int)cudaMemcpyFromSymbol(host, g_ssd_trace, sizeof(g_ssd_trace)); }
+#else
+#define SSD_TR(role, c, pt) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int Q = 128, P = 64, NS = 128;
@@ -127,6 +141,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const int t0 = c * Q, s = c & 1, sx = c % X_SLOTS, d = c & (DEC_DEPTH - 1);
             if (lane == 0) {
                 if (tc::mbar_wait(bars + B_BCE + s, ((c >> 1) & 1) ^ 1, abort_flag)) {
+                    SSD_TR(0, c, 0);
                     uint64_t *fb = bars + B_BCF + s;
                     tc::mbar_arrive_expect_tx(fb, 4 * TILE_16K);
                     tc::tma_load_3d(smem + OFF_B + (s * 2) * TILE_16K, &tmap_b, fb, g * NS, t0, b);
@@ -135,6 +150,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     tc::tma_load_3d(smem + OFF_C + (s * 2 + 1) * TILE_16K, &tmap_c, fb, g * NS + 64, t0, b);
                     ++n_bc;
                     if (tc::mbar_wait(bars + B_XE + sx, ((c / X_SLOTS) & 1) ^ 1, abort_flag)) {
+                        SSD_TR(0, c, 1);
                         tc::mbar_arrive_expect_tx(bars + B_XF + sx, TILE_16K);
                         tc::tma_load_3d(smem + OFF_X + sx * TILE_16K, &tmap_x, bars + B_XF + sx, h * P, t0, b);
                         ++n_x;
@@ -154,6 +170,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 dn[i] = t < Tlen ? __ldg(dtb + (size_t)t * H) : 0.f;
             }
             if (!tc::mbar_wait(bars + B_DECE + d, ((c >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
+            SSD_TR(0, c, 2);
             float l[4];
             l[0] = dv[0] * Ah2;
 #pragma unroll
@@ -191,6 +208,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             if (lane < 16) dec[D_BLK + lane] = ((lane & 3) < (lane >> 2)) ? tc::ex2(bs - be) : 0.f;
             if (lane == 0) dec[D_EEND] = tc::ex2(l_end);
             warp_arrive(bars + B_DECF + d, lane);
+            SSD_TR(0, c, 3);
         }
         if (!ok && lane == 0) {
             atomicCAS(status, 0, STR_ERR_TIMEOUT);
@@ -294,8 +312,10 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const int d = c & (DEC_DEPTH - 1), s = c & 1;
             const float *dec = decs + d * DEC_FLOATS;
             if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
+            if (warp == 3) SSD_TR(2, c, 0); else if (warp == 15) SSD_TR(3, c, 0); else if (warp == 0) SSD_TR(4, c, 0);
             const float l_t = dec[D_LS + row], rf = dec[D_ROWF + row];
             if (!tc::mbar_wait(bars + B_CBF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
+            if (warp == 3) SSD_TR(2, c, 1); else if (warp == 15) SSD_TR(3, c, 1); else if (warp == 0) SSD_TR(4, c, 1);
             tc::tc_fence_after();
             const uint32_t tW = tmem + lane_base + TM_CB + (uint32_t)(s * 128 + half * 64);
             uint32_t v[16], vn[16];
@@ -346,6 +366,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             }
             tc::tmem_st_wait();
             tc::tc_fence_before();
+            if (warp == 3) SSD_TR(2, c, 2); else if (warp == 15) SSD_TR(3, c, 2); else if (warp == 0) SSD_TR(4, c, 2);
             warp_arrive(bars + B_WF + s, lane);
             if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
         }
@@ -365,7 +386,9 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const float eend = decs[d * DEC_FLOATS + D_EEND];
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
+            if (quad == 0) SSD_TR(5, c, 0);
             if (!tc::mbar_wait(bars + B_DSF, c & 1, abort_flag)) { ok = false; break; }
+            if (quad == 0) SSD_TR(5, c, 1);
             tc::tc_fence_after();
             uint8_t *srow = smem + OFF_SB + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
@@ -391,6 +414,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             }
             tc::fence_proxy_async();
             warp_arrive(bars + B_SF, lane);
+            if (quad == 0) SSD_TR(5, c, 2);
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         if (ok && final_state) {
@@ -407,6 +431,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         bool ok = true;
 #pragma unroll 1
         for (int c = 0; c <= nchunks; ++c) {
+            if (quad == 0) SSD_TR(6, c, 0);
             if (c < nchunks) {
                 // Xs_c = exp(l_end - l_j) dt_j x_j, same swizzled layout as the X tile
                 const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
@@ -414,6 +439,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
                 if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
                 if (c > 0 && !tc::mbar_wait(bars + B_DSF, (c - 1) & 1, abort_flag)) { ok = false; break; }   // Xs buffer free
+                if (quad == 0) SSD_TR(6, c, 1);
                 const uint4 *src = (const uint4 *)(smem + OFF_X + sx * TILE_16K);
                 uint4 *dst = (uint4 *)(smem + OFF_XS);
 #pragma unroll
@@ -430,6 +456,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
+                if (quad == 0) SSD_TR(6, c, 2);
             }
             if (c >= 1) {
                 const int cp = c - 1, d = cp & (DEC_DEPTH - 1), t0 = cp * Q;
@@ -437,6 +464,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
                 if (!tc::mbar_wait(bars + B_YF, cp & 1, abort_flag)) { ok = false; break; }
+                if (quad == 0) SSD_TR(6, c, 3);
                 tc::tc_fence_after();
                 uint4 *dst = (uint4 *)(yb + (size_t)(t0 + row) * H * P);
                 const bool valid = t0 + row < Tlen;
@@ -462,6 +490,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc::tmem_ld_wait();
                 tc::tc_fence_before();               // both accumulators are in registers
                 warp_arrive(bars + B_YE, lane);
+                if (quad == 0) SSD_TR(6, c, 4);
                 if (cp > 0) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) yb2[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yb2[i])));
