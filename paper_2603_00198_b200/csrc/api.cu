@@ -53,6 +53,8 @@ extern "C" int str_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, 
         return STR_ERR_INVALID_ARG;
     if (n_vis == 0) return STR_OK;
     if (!scores_out) return STR_ERR_INVALID_ARG;
+    if (!str_force_simt() && ctx->encode_tiled && str_mamba_importance_tc_supported(s, n_vis, n_text, B, C))
+        return str_mamba_importance_tc(ctx, s, n_vis, n_text, B, C, dt, scores_out, (cudaStream_t)stream);
     return str_mamba_importance_simt(ctx, s, n_vis, n_text, B, C, dt, scores_out, (cudaStream_t)stream);
 }
 

@@ -27,3 +27,6 @@ int str_ssd_tc(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float 
 bool str_attn_prefill_tc_supported(const str_attn_shape *s, const void *q, const void *k, const void *v, const void *o);
 int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v, float scale,
                         void *o, cudaStream_t st);
+bool str_mamba_importance_tc_supported(const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C);
+int str_mamba_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C,
+                            const float *dt, float *scores, cudaStream_t st);

@@ -26,6 +26,13 @@ MAMBA_CASES = [
     ("bf16", 1000, 100, 16, 64, 4, 2),       # ragged tiles, batch
     ("f32", 70, 3, 4, 32, 2, 1),
     ("bf16", 5, 1, 2, 16, 1, 1),
+    # d_state 128 in bf16 runs on the tensor cores: text counts that need padding to 16, more than 128 text
+    # rows, ragged token tiles, a single token, batch
+    ("bf16", 1000, 100, 16, 128, 4, 2),
+    ("bf16", 300, 1, 8, 128, 8, 1),
+    ("bf16", 777, 200, 32, 128, 2, 1),
+    ("bf16", 1, 16, 4, 128, 1, 3),
+    ("bf16", 129, 256, 8, 128, 2, 1),
 ]
 
 
