@@ -62,7 +62,8 @@ extern "C" int str_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, 
 extern "C" size_t str_attn_importance_workspace_size(const str_attn_score_shape *s, int n_vis, int n_text) {
     (void)n_vis;
     if (!s || s->Bz <= 0 || s->Hq <= 0 || n_text <= 0) return 0;
-    return align_up((size_t)2 * s->Bz * s->Hq * n_text * sizeof(float), 256);
+    // row maxima and sums per (sequence, head, key segment, text query), plus their merged form
+    return align_up((size_t)2 * s->Bz * s->Hq * n_text * (STR_ATTN_SCORE_MAX_SEGMENTS + 1) * sizeof(float), 256);
 }
 
 extern "C" int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
@@ -76,6 +77,9 @@ extern "C" int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, 
     if (n_vis == 0) return STR_OK;
     if (!scores_out || !workspace) return STR_ERR_INVALID_ARG;
     if (workspace_bytes < str_attn_importance_workspace_size(s, n_vis, n_text)) return STR_ERR_WORKSPACE_TOO_SMALL;
+    if (!str_force_simt() && ctx->encode_tiled && str_attn_importance_tc_supported(s, n_vis, n_text, q, k))
+        return str_attn_importance_tc(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, (float *)workspace,
+                                      (cudaStream_t)stream);
     float *row_max = (float *)workspace;
     float *row_sum = row_max + (size_t)s->Bz * s->Hq * n_text;
     return str_attn_importance_simt(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, row_max, row_sum,

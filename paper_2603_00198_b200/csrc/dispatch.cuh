@@ -30,3 +30,8 @@ int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, const void *q, co
 bool str_mamba_importance_tc_supported(const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C);
 int str_mamba_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C,
                             const float *dt, float *scores, cudaStream_t st);
+// Key segments the tensor-core attention score may split its first pass into (sizes the workspace).
+#define STR_ATTN_SCORE_MAX_SEGMENTS 8
+bool str_attn_importance_tc_supported(const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k);
+int str_attn_importance_tc(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k,
+                           float scale, float *scores, float *workspace, cudaStream_t st);

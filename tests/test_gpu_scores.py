@@ -56,6 +56,13 @@ ATTN_CASES = [
     ("bf16", 300, 5, 6, 2, 32, 1),
     ("f32", 64, 1, 2, 2, 16, 1),
     ("bf16", 3, 2, 4, 1, 128, 1),
+    # head_dim 128 in bf16 runs on the tensor cores: padded text counts, more than 128 text rows, ragged key
+    # tiles (last 256-key step and last 128-key tile partly beyond the visual keys), no GQA, batch
+    ("bf16", 1000, 100, 8, 2, 128, 2),
+    ("bf16", 777, 200, 4, 4, 128, 1),
+    ("bf16", 129, 256, 2, 1, 128, 1),
+    ("bf16", 5000, 1, 8, 8, 128, 1),
+    ("bf16", 256, 16, 4, 2, 128, 3),
 ]
 
 
