@@ -1,12 +1,18 @@
 // str_topk_select: per-sequence radix select of the k largest fp32 scores, emitted in
 // ascending index order (temporal order preserved; ties go to the lower index).
 //
-// One CTA per sequence.  Four 8-bit MSB-first passes over the order-preserving integer image
+// Two kernels: rows of up to 131072 scores are shared by a thread-block cluster that keeps the keys in
+// registers (second half of this file); longer rows take one CTA per sequence that re-reads the scores
+// every pass.  Both: four 8-bit MSB-first passes over the order-preserving integer image
 // of the scores narrow down the k-th largest key; per-warp private histograms with
 // warp-aggregated increments keep shared-memory atomics uncontended even when every score
 // shares its top byte.  A last ordered pass emits the survivors: each warp owns a contiguous
 // index segment, so a single block-level exclusive scan of 32 warp counts orders the output.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -120,6 +126,154 @@ topk_select_kernel(int n, int k, const float *__restrict__ scores, int32_t *__re
     }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Cluster version for rows of up to CL_MAX_N scores: a thread-block cluster of up to 8 CTAs shares one row.
+// Every thread keeps a contiguous run of KPT keys in registers, so the scores are read from memory once.
+// Per radix pass each CTA builds a 256-bin histogram of its live keys in shared memory; after one cluster
+// barrier every CTA sums the histograms of the whole cluster through distributed shared memory and takes
+// the same decision (histograms are double-buffered, so one barrier per pass is enough).  The ordered emit
+// uses a block scan of per-thread (greater, equal) counts plus the totals of the lower-ranked CTAs.
+constexpr int CL_THREADS = 1024, CL_MAX_CTAS = 8, CL_MAX_KPT = 16;
+constexpr int CL_MAX_N = CL_THREADS * CL_MAX_CTAS * CL_MAX_KPT;      // 131072
+
+template <int KPT>
+__global__ void __launch_bounds__(CL_THREADS)
+topk_cluster_kernel(int n, int k, const float *__restrict__ scores, int32_t *__restrict__ kept) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank(), ncta = (int)cluster.num_blocks();
+    __shared__ uint32_t hist[2][256];
+    __shared__ uint32_t total[256];
+    __shared__ uint32_t sh_prefix, sh_need;
+    __shared__ uint32_t warp_gt[32], warp_eq[32];
+    __shared__ uint32_t cta_tot[2];
+
+    const float *s = scores + (size_t)blockIdx.y * n;
+    int32_t *out = kept + (size_t)blockIdx.y * k;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per_cta = KPT * CL_THREADS;
+    const int base = rank * per_cta + tid * KPT;                     // first index of this thread's run
+
+    uint32_t key[KPT];
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) key[j] = (base + j < n) ? score_key(__ldg(s + base + j)) : 0u;
+
+    uint32_t prefix = 0, mask = 0, need = (uint32_t)k;
+    int pass = 0;
+    for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
+        uint32_t *h = hist[pass & 1];
+        if (tid < 256) h[tid] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const bool live = (base + j < n) && ((key[j] & mask) == prefix);
+            const uint32_t bin = (key[j] >> shift) & 255u;
+            const uint32_t live_mask = __ballot_sync(0xffffffffu, live);
+            if (live) {       // warp-aggregated increment: lanes with the same bin elect one leader
+                const uint32_t peers = __match_any_sync(live_mask, bin);
+                if (lane == __ffs(peers) - 1) atomicAdd(&h[bin], (uint32_t)__popc(peers));
+            }
+            __syncwarp();
+        }
+        cluster.sync();
+        if (tid < 256) {
+            uint32_t t = 0;
+            for (int r = 0; r < ncta; ++r) t += cluster.map_shared_rank(h, r)[tid];
+            total[tid] = t;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane L owns bins 255-8L .. 248-8L (descending); find the bin holding the need-th largest
+            uint32_t c[8], lane_sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { c[j] = total[255 - 8 * lane - j]; lane_sum += c[j]; }
+            uint32_t incl = lane_sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const uint32_t before = incl - lane_sum;
+            if (before < need && need <= incl) {
+                uint32_t run = before;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (run < need && need <= run + c[j]) {
+                        sh_prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
+                        sh_need = need - run;
+                    }
+                    run += c[j];
+                }
+            }
+        }
+        __syncthreads();
+        prefix = sh_prefix;
+        need = sh_need;
+        mask |= 255u << shift;
+    }
+    // prefix = key of the k-th largest score; keep every key > prefix plus the first `need` (in index order)
+    // of the keys == prefix
+    uint32_t gt = 0, eq = 0;
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const bool in = base + j < n;
+        gt += (in && key[j] > prefix) ? 1u : 0u;
+        eq += (in && key[j] == prefix) ? 1u : 0u;
+    }
+    uint32_t gt_incl = gt, eq_incl = eq;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t a = __shfl_up_sync(0xffffffffu, gt_incl, o), b2 = __shfl_up_sync(0xffffffffu, eq_incl, o);
+        if (lane >= o) { gt_incl += a; eq_incl += b2; }
+    }
+    if (lane == 31) { warp_gt[warp] = gt_incl; warp_eq[warp] = eq_incl; }
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t a = warp_gt[lane], b2 = warp_eq[lane], ai = a, bi = b2;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t x = __shfl_up_sync(0xffffffffu, ai, o), y = __shfl_up_sync(0xffffffffu, bi, o);
+            if (lane >= o) { ai += x; bi += y; }
+        }
+        warp_gt[lane] = ai - a;                                      // exclusive prefix over warps
+        warp_eq[lane] = bi - b2;
+        if (lane == 31) { cta_tot[0] = ai; cta_tot[1] = bi; }
+    }
+    cluster.sync();
+    uint32_t gt_before = warp_gt[warp] + (gt_incl - gt), eq_before = warp_eq[warp] + (eq_incl - eq);
+    for (int r = 0; r < rank; ++r) {
+        const uint32_t *t = cluster.map_shared_rank(cta_tot, r);
+        gt_before += t[0];
+        eq_before += t[1];
+    }
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const bool in = base + j < n;
+        const bool is_gt = in && key[j] > prefix, is_eq = in && key[j] == prefix;
+        if (is_gt || (is_eq && eq_before < need)) out[gt_before + min(eq_before, need)] = base + j;
+        gt_before += is_gt ? 1u : 0u;
+        eq_before += is_eq ? 1u : 0u;
+    }
+    cluster.sync();           // no CTA leaves while another may still read its shared memory
+}
+
+template <int KPT>
+cudaError_t launch_cluster(int ncta, int Bz, int n, int k, const float *scores, int32_t *kept, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ncta, Bz, 1);
+    cfg.blockDim = dim3(CL_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ncta;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, topk_cluster_kernel<KPT>, n, k, scores, kept);
+}
+
 }  // namespace
 
 extern "C" size_t str_topk_select_workspace_size(int, int, int) { return 0; }
@@ -130,6 +284,21 @@ extern "C" int str_topk_select(str_ctx *ctx, int Bz, int n_vis, int k, const flo
     if (!ctx || Bz <= 0 || n_vis < 0 || k < 0 || k > n_vis) return STR_ERR_INVALID_ARG;
     if (k == 0) return STR_OK;
     if (!scores || !kept_idx_out) return STR_ERR_INVALID_ARG;
-    topk_select_kernel<<<Bz, TOPK_THREADS, 0, (cudaStream_t)stream>>>(n_vis, k, scores, kept_idx_out);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n_vis <= CL_MAX_N) {
+        // smallest cluster (power of two, at most 8 CTAs) and run length that cover the row
+        int ncta = 1;
+        while (ncta < CL_MAX_CTAS && ncta * CL_THREADS * 4 < n_vis) ncta *= 2;
+        const int per_thread = ceil_div(n_vis, ncta * CL_THREADS);
+        cudaError_t e;
+        if (per_thread <= 1) e = launch_cluster<1>(ncta, Bz, n_vis, k, scores, kept_idx_out, st);
+        else if (per_thread <= 2) e = launch_cluster<2>(ncta, Bz, n_vis, k, scores, kept_idx_out, st);
+        else if (per_thread <= 4) e = launch_cluster<4>(ncta, Bz, n_vis, k, scores, kept_idx_out, st);
+        else if (per_thread <= 8) e = launch_cluster<8>(ncta, Bz, n_vis, k, scores, kept_idx_out, st);
+        else e = launch_cluster<16>(ncta, Bz, n_vis, k, scores, kept_idx_out, st);
+        ctx->launches += 1;
+        return e == cudaSuccess ? STR_OK : STR_ERR_CUDA;
+    }
+    topk_select_kernel<<<Bz, TOPK_THREADS, 0, st>>>(n_vis, k, scores, kept_idx_out);
     return str_launch_ok(ctx);
 }
