@@ -20,7 +20,7 @@ Pin status (tests/test_oracle_*.py, all CPU):
                          pinned  (the paper's printed compression percentages)
   sigmoid_schedule       parity unpinned: the printed percentages of the sigmoid rows are
                          not reproduced to the printed digit by any indexing of the formula
-  rmsnorm, causal_conv1d_silu, rope, attention_forward, mamba2_block, attn_block, stack_prefill
+  rmsnorm, causal_conv1d_silu, rope, attention_forward, attention_rows, mamba2_block, attn_block, stack_prefill
                          parity unpinned by the paper (it does not define the block around the
                          recurrence); pinned only to textbook definitions, library routines
                          and brute force on tiny inputs
@@ -340,6 +340,22 @@ def attention_forward(q, k, v, scale, slab=512):
             w = np.exp(logits)
             w /= w.sum(axis=1, keepdims=True)
             o[s:e, h] = w @ v[:e, kv]
+    return o
+
+
+def attention_rows(q, k, v, scale, rows):
+    """The same definition for a few query rows only: o_t for t in ``rows``, shape [len(rows), Hq, d].
+    Used where the sequence is too long to evaluate every row on the CPU."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    o = np.zeros((len(rows), Hq, d))
+    for i, t in enumerate(rows):
+        for h in range(Hq):
+            kv = h // (Hq // Hkv)
+            logits = (k[:t + 1, kv] @ q[t, h]) * scale
+            w = np.exp(logits - logits.max())
+            o[i, h] = (w / w.sum()) @ v[:t + 1, kv]
     return o
 
 

@@ -1,0 +1,131 @@
+"""GPU parity at the benchmark's full sizes (the 32768+128-token stack shapes), in the launch
+configurations the benchmark times.  The oracle cannot evaluate every output at these sizes in
+seconds, so it evaluates sampled outputs one by one (whole heads of the scan, sampled tokens of the
+scores, sampled rows of the products) and the rest is checked through properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_00198_b200 import binding, inputs
+from util_gpu import assert_kept_matches, dev, host, max_rel_err, score_rel_err
+
+pytestmark = pytest.mark.gpu
+MS, AT = inputs.MAMBA_8B, inputs.ATTN_8B
+N_VIS, M = 32768, 128
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.check_status()
+    c.close()
+
+
+def test_scan_full_length_sampled_heads(ctx):
+    T, H, p, n, G = N_VIS + M, MS["H"], MS["p"], MS["n"], MS["G"]
+    d = inputs.ssd_inputs(81, T, H, p, n, G, "bf16")
+    y, fs = binding.str_mamba2_prefill(ctx, dev(d["x"], "bf16"), dev(d["dt"]), dev(d["A"]), dev(d["B"], "bf16"),
+                                       dev(d["C"], "bf16"), Q=MS["Q"], want_final_state=True)
+    ctx.check_status()
+    y, fs = y.float().cpu().numpy(), fs.cpu().numpy()
+    assert np.all(np.isfinite(y))
+    hpg = H // G
+    for h in (0, 37, 127):                       # whole heads: the sequential recurrence over all 32896 tokens
+        g = h // hpg
+        ry, rs = oracle.mamba2_recurrence(d["x"][0][:, h:h + 1], d["dt"][0][:, h:h + 1], d["A"][h:h + 1],
+                                          d["B"][0][:, g:g + 1], d["C"][0][:, g:g + 1])
+        assert max_rel_err(y[0][:, h], ry[:, 0]) <= 2e-2, h
+        assert max_rel_err(fs[0][h], rs[0]) <= 1e-2, h
+
+
+@pytest.mark.parametrize("n_vis", [32768, 65536])
+def test_mamba_importance_full_length_sampled_tokens(ctx, n_vis):
+    H, n, G = MS["H"], MS["n"], MS["G"]
+    T = n_vis + M
+    g = inputs.rng(82, n_vis)
+    Bm = inputs.to_grid(g.standard_normal((1, T, G, n), dtype=np.float32), "bf16")
+    Cm = inputs.to_grid(g.standard_normal((1, T, G, n), dtype=np.float32), "bf16")
+    dt = g.uniform(1e-3, 1e-1, size=(1, T, H)).astype(np.float32)
+    got = binding.str_mamba_importance(ctx, dev(Bm, "bf16"), dev(Cm, "bf16"), dev(dt), n_vis, M).cpu().numpy()[0]
+    ctx.check_status()
+    assert got.shape == (n_vis,) and np.all(np.isfinite(got)) and np.all(got > 0)
+    # a token's score depends on its own row and on the text rows only: evaluate sampled tokens
+    sample = np.unique(np.concatenate([g.choice(n_vis, size=500, replace=False), [0, 127, 128, n_vis - 129, n_vis - 1]]))
+    rows = np.concatenate([sample, np.arange(n_vis, T)])
+    ref = oracle.mamba_importance(Bm[0][rows], Cm[0][rows], dt[0][rows], len(sample), M)
+    assert score_rel_err(got[sample], ref) <= 1e-3
+
+
+def test_gemm_full_size_sampled_entries(ctx):
+    Mrows, K = N_VIS + M, MS["D"]
+    N = 2 * MS["H"] * MS["p"] + 2 * MS["G"] * MS["n"] + MS["H"]            # in_proj width 18560
+    g = inputs.rng(83, 1)
+    a = inputs.to_grid(g.standard_normal((Mrows, K), dtype=np.float32), "bf16")
+    w = inputs.to_grid(g.standard_normal((N, K), dtype=np.float32) / np.sqrt(K), "bf16")
+    out = binding.str_gemm(ctx, dev(a, "bf16"), dev(w, "bf16"))
+    ctx.check_status()
+    rows = np.unique(np.concatenate([g.choice(Mrows, size=40, replace=False), [0, 127, 128, Mrows - 1]]))
+    ref = a[rows].astype(np.float64) @ w.astype(np.float64).T               # full output rows
+    got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+    assert max_rel_err(got, ref) <= 2e-2
+
+
+def test_attention_forward_full_length_sampled_rows(ctx):
+    T, Hq, Hkv, d = 16384 + M, AT["Hq"], AT["Hkv"], AT["d"]               # the stack's attention layers see 16512 tokens
+    g = inputs.rng(84, 1)
+    q = inputs.to_grid(g.standard_normal((1, T, Hq, d), dtype=np.float32), "bf16")
+    k = inputs.to_grid(g.standard_normal((1, T, Hkv, d), dtype=np.float32), "bf16")
+    v = inputs.to_grid(g.standard_normal((1, T, Hkv, d), dtype=np.float32), "bf16")
+    scale = 1.0 / np.sqrt(d)
+    o = binding.str_attn_prefill(ctx, dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16"), scale)
+    ctx.check_status()
+    rows = [0, 1, 127, 128, 255, 256, 5000, 12345, T - 129, T - 1]
+    ref = oracle.attention_rows(q[0], k[0], v[0], scale, rows)
+    got = o[0][torch.tensor(rows).cuda()].float().cpu().numpy()
+    assert max_rel_err(got, ref) <= 2e-2
+
+
+def test_compaction_full_size_is_bit_exact(ctx):
+    D, k = MS["D"], N_VIS // 2
+    T = N_VIS + M
+    h = inputs.hidden_inputs(85, T, D, "bf16")
+    g = inputs.rng(85, 9)
+    ids = np.arange(T, dtype=np.int32)[None]
+    kept = np.sort(g.choice(N_VIS, size=k, replace=False)).astype(np.int32)[None]
+    ho, po, io = binding.str_compact(ctx, dev(h, "bf16"), dev(ids), dev(ids), dev(kept), M)
+    rh, rp, ri = oracle.compact(h[0], ids[0], ids[0], kept[0], M)
+    assert np.array_equal(io[0].cpu().numpy(), ri) and np.array_equal(po[0].cpu().numpy(), rp)
+    assert np.array_equal(ho[0].float().cpu().numpy(), rh)
+
+
+def test_stack_full_size_properties(ctx):
+    """The 12-layer stack exactly as the benchmark runs it: schedule, ordering and bookkeeping properties
+    that hold at any size, plus the first reducing layer's selection against the oracle's selection rule
+    applied to the scores the GPU produced."""
+    cfg = inputs.CONFIGS["C3"]
+    n_vis, n_text = cfg["n_vis"], cfg["n_text"]
+    K = binding.str_schedule_keep_counts(cfg["alpha_bp"], n_vis, cfg["min_keep"])
+    assert K == oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis, cfg["min_keep"])
+    assert K == [32768] * 4 + [16384] * 4 + [8192] * 4
+    layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], "f32")
+    st = binding.Stack(ctx, layers, "bf16", 1, n_vis, n_text, K, Q=cfg["mamba"]["Q"])
+    del layers
+    h0 = inputs.hidden_inputs(cfg["seed"], n_vis + n_text, cfg["mamba"]["D"], "bf16")
+    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, "bf16"), want_trace=True)
+    ctx.check_status()
+    assert out.shape == (1, K[-1] + n_text, cfg["mamba"]["D"]) and bool(torch.isfinite(out.float()).all())
+    gi = idx[0].cpu().numpy()
+    assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-n_text:], np.arange(n_vis, n_vis + n_text))
+    assert np.array_equal(pos[0].cpu().numpy(), gi)
+    assert [t["layer"] for t in tr] == [4, 8] and [t["n_in"] for t in tr] == [32768, 16384]
+    # selection at each reducing layer = the oracle's rule on the same scores (bit-exact), and the survivors of
+    # the second cut are a subset of the first cut's
+    kept1 = tr[0]["kept"][0].cpu().numpy()
+    s1 = tr[0]["scores"][0].cpu().numpy()
+    assert np.all(s1 > 0) and np.array_equal(kept1, oracle.topk_select(s1, K[4]))
+    kept2 = tr[1]["kept"][0].cpu().numpy()
+    s2 = tr[1]["scores"][0].cpu().numpy()
+    assert np.array_equal(kept2, oracle.topk_select(s2, K[8]))
+    assert np.array_equal(gi[:K[-1]], kept1[kept2])

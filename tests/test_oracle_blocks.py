@@ -68,6 +68,19 @@ def test_attention_forward_brute_force_and_special_cases():
     np.testing.assert_allclose(o0[:, 0], np.cumsum(v[:, 0], axis=0) / np.arange(1, T + 1)[:, None], rtol=1e-12)
 
 
+def test_attention_rows_is_the_same_definition_row_by_row():
+    r = np.random.default_rng(6)
+    T, Hq, Hkv, d = 23, 6, 3, 5
+    q, k, v = r.normal(size=(T, Hq, d)), r.normal(size=(T, Hkv, d)), r.normal(size=(T, Hkv, d))
+    rows = [0, 1, 7, 22]
+    o = oracle.attention_rows(q, k, v, 0.9, rows)
+    np.testing.assert_allclose(o, oracle.attention_forward(q, k, v, 0.9)[rows], atol=1e-13)
+    for i, t in enumerate(rows):                 # a library softmax over the allowed keys
+        for h in range(Hq):
+            w = softmax((k[:t + 1, h // 2] @ q[t, h]) * 0.9)
+            np.testing.assert_allclose(o[i, h], w @ v[:t + 1, h // 2], atol=1e-13)
+
+
 def test_stack_identity_schedule_and_text_rows_last():
     from paper_2603_00198_b200 import inputs
     ms = dict(D=32, H=4, p=8, n=8, G=2, Q=16, conv=4)
