@@ -195,6 +195,22 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of per-rank timings over all ranks (every rank gets the result).  The path does
+    not shard, so this reduction of the measured times is the only collective the benchmark makes."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_tokens_per_s(tokens_per_rank, world, ms_step_max):
+    """Whole-job throughput of `world` independent replicas: all ranks' tokens over the slowest rank's time."""
+    return tokens_per_rank * world / (ms_step_max * 1e-3)
+
+
 # ------------------------------------------------------------------ GPU arm
 def run_ours(args):
     import torch
@@ -265,19 +281,15 @@ def run_ours(args):
     ms_e2e = e0.elapsed_time(e1)
     same = bool((out_pin.cuda() == out).all()) and bool((idx_pin.cuda() == idx).all())
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     ms_step = ms_total / args.steps
-    tokens = Bz * T0 * world
-    value = tokens / (ms_step * 1e-3)
-    e2e_value = tokens / (ms_e2e / e2e_steps * 1e-3)
+    value = aggregate_tokens_per_s(Bz * T0, world, ms_step)
+    e2e_value = aggregate_tokens_per_s(Bz * T0, world, ms_e2e / e2e_steps)
     pk = peaks()
     work = work_model(cfg, K)
     kernels = {}
