@@ -37,6 +37,9 @@
 // Optional device-side timeline (compile with -DSTR_SSD_TRACE): lane 0 of selected warps of one CTA
 // stores the SM clock at a few points of chunks 16..31.  Compiled out of the library build.
 #ifdef STR_SSD_TRACE
+#ifndef STR_SSD_TRACE_QUAD
+#define STR_SSD_TRACE_QUAD 0
+#endif
 __device__ long long g_ssd_trace[8 * 16 * 8];
 #define SSD_TR(role, c, pt)                                                                              \
     do {                                                                                                 \
@@ -44,8 +47,10 @@ __device__ long long g_ssd_trace[8 * 16 * 8];
             g_ssd_trace[((role) * 16 + ((c) - 16)) * 8 + (pt)] = clock64();                              \
     } while (0)
 extern "C" int str_ssd_trace_fetch(long long *host) { return (int)cudaMemcpyFromSymbol(host, g_ssd_trace, sizeof(g_ssd_trace)); }
+#define SSD_TRQ STR_SSD_TRACE_QUAD
 #else
 #define SSD_TR(role, c, pt) do { } while (0)
+#define SSD_TRQ 0
 #endif
 
 namespace {
@@ -241,9 +246,11 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         for (int c = 0; c <= nchunks && ok; ++c) {
             const int s = c & 1;
             const uint64_t dk_c = desc_add(dk_c0, (uint32_t)s * 2 * TILE_16K), dk_b = desc_add(dk_b0, (uint32_t)s * 2 * TILE_16K);
+            SSD_TR(1, c, 0);
             if (c < nchunks) {
                 ok = warp_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag);
                 if (!ok) break;
+                SSD_TR(1, c, 1);
                 tc::tc_fence_after();
                 if (tc::elect_one()) {
 #pragma unroll 1
@@ -253,6 +260,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     tc::mma_commit(bars + B_CBF + s);
                 }
                 __syncwarp();
+                SSD_TR(1, c, 2);
             }
             if (c >= 1) {
                 const int cp = c - 1, sp = cp & 1;
@@ -260,6 +268,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 ok = (c < 2 || warp_wait(bars + B_YE, (c - 2) & 1, abort_flag)) &&
                      warp_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag);
                 if (!ok) break;
+                SSD_TR(1, c, 3);
                 tc::tc_fence_after();
                 const uint64_t dm_x = desc_add(dm_x0, (uint32_t)(cp % X_SLOTS) * TILE_16K);
                 const uint32_t tW = tmem + TM_CB + (uint32_t)sp * 128;
@@ -272,11 +281,13 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     tc::mma_commit(bars + B_XE + cp % X_SLOTS);
                 }
                 __syncwarp();
+                SSD_TR(1, c, 4);
             }
             if (c < nchunks) {
                 if (c > 0) {
                     ok = warp_wait(bars + B_SF, (c - 1) & 1, abort_flag);
                     if (!ok) break;
+                    SSD_TR(1, c, 5);
                     tc::tc_fence_after();
                     if (tc::elect_one()) {
 #pragma unroll 1
@@ -288,6 +299,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 }
                 ok = warp_wait(bars + B_XSF, c & 1, abort_flag) && (c == 0 || warp_wait(bars + B_DSE, (c - 1) & 1, abort_flag));
                 if (!ok) break;
+                SSD_TR(1, c, 6);
                 tc::tc_fence_after();
                 const uint64_t dm_b = desc_add(dm_b0, (uint32_t)s * 2 * TILE_16K);
                 if (tc::elect_one()) {
@@ -298,6 +310,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     tc::mma_commit(bars + B_BCE + s);
                 }
                 __syncwarp();
+                SSD_TR(1, c, 7);
             }
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
@@ -386,9 +399,9 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const float eend = decs[d * DEC_FLOATS + D_EEND];
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
-            if (quad == 0) SSD_TR(5, c, 0);
+            if (quad == SSD_TRQ) SSD_TR(5, c, 0);
             if (!tc::mbar_wait(bars + B_DSF, c & 1, abort_flag)) { ok = false; break; }
-            if (quad == 0) SSD_TR(5, c, 1);
+            if (quad == SSD_TRQ) SSD_TR(5, c, 1);
             tc::tc_fence_after();
             uint8_t *srow = smem + OFF_SB + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
@@ -414,7 +427,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             }
             tc::fence_proxy_async();
             warp_arrive(bars + B_SF, lane);
-            if (quad == 0) SSD_TR(5, c, 2);
+            if (quad == SSD_TRQ) SSD_TR(5, c, 2);
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         if (ok && final_state) {
@@ -431,7 +444,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         bool ok = true;
 #pragma unroll 1
         for (int c = 0; c <= nchunks; ++c) {
-            if (quad == 0) SSD_TR(6, c, 0);
+            if (quad == SSD_TRQ) SSD_TR(6, c, 0);
             if (c < nchunks) {
                 // Xs_c = exp(l_end - l_j) dt_j x_j, same swizzled layout as the X tile
                 const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
@@ -439,7 +452,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
                 if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
                 if (c > 0 && !tc::mbar_wait(bars + B_DSF, (c - 1) & 1, abort_flag)) { ok = false; break; }   // Xs buffer free
-                if (quad == 0) SSD_TR(6, c, 1);
+                if (quad == SSD_TRQ) SSD_TR(6, c, 1);
                 const uint4 *src = (const uint4 *)(smem + OFF_X + sx * TILE_16K);
                 uint4 *dst = (uint4 *)(smem + OFF_XS);
 #pragma unroll
@@ -456,7 +469,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
-                if (quad == 0) SSD_TR(6, c, 2);
+                if (quad == SSD_TRQ) SSD_TR(6, c, 2);
             }
             if (c >= 1) {
                 const int cp = c - 1, d = cp & (DEC_DEPTH - 1), t0 = cp * Q;
@@ -464,7 +477,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
                 if (!tc::mbar_wait(bars + B_YF, cp & 1, abort_flag)) { ok = false; break; }
-                if (quad == 0) SSD_TR(6, c, 3);
+                if (quad == SSD_TRQ) SSD_TR(6, c, 3);
                 tc::tc_fence_after();
                 uint4 *dst = (uint4 *)(yb + (size_t)(t0 + row) * H * P);
                 const bool valid = t0 + row < Tlen;
@@ -490,7 +503,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc::tmem_ld_wait();
                 tc::tc_fence_before();               // both accumulators are in registers
                 warp_arrive(bars + B_YE, lane);
-                if (quad == 0) SSD_TR(6, c, 4);
+                if (quad == SSD_TRQ) SSD_TR(6, c, 4);
                 if (cp > 0) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) yb2[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yb2[i])));

@@ -45,7 +45,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // instructions and never unrolled: warp-specialised kernels have dozens of wait sites and their
 // combined footprint has to stay inside the instruction cache.
 constexpr uint32_t WAIT_PROBE_LIMIT = 1u << 22;
+// Non-blocking probe: has the phase with this parity completed?
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort) {
+    if (mbar_test_wait(bar, parity)) return true;        // the common case in a pipeline that runs ahead
     uint32_t probes = 0;
 #pragma unroll 1
     while (!mbar_try_wait(bar, parity)) {
