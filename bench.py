@@ -46,6 +46,11 @@ def workload(args):
         cfg["n_vis"] = args.n_vis
     if args.final_bp:
         cfg["alpha_bp"] = inputs.sweep_alpha_bp(args.final_bp, len(cfg["pattern"]))
+    if args.schedule == "sigmoid":
+        # all-layer sigmoid retention (the paper's appendix: k = 20, start 1.0, end 0.125, midpoint x0): every
+        # layer cuts a little, so the attention layers select inside the stack as well
+        from paper_2603_00198_b200 import binding
+        cfg["alpha_bp"] = binding.str_sigmoid_schedule_bp(len(cfg["pattern"]), 20.0, args.x0, 1.0, 0.125)
     cfg["batch"] = args.batch
     return cfg
 
@@ -335,7 +340,8 @@ def run_ours(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": "C3 12-layer hybrid stack [M,M,M,M,M,A]x2, %d visual + %d text tokens, batch %d, "
-                               "schedule %s" % (n_vis, M, Bz, "/".join(str(a // 100) for a in cfg["alpha_bp"][::4])),
+                               "schedule %s" % (n_vis, M, Bz, "/".join(str(a // 100) for a in (cfg["alpha_bp"][::4] if args.schedule == "step"
+                                                                                  else cfg["alpha_bp"]))),
                    "keep_counts": K, "l2": "inputs larger than L2 (hidden %d MB, workspace %d MB)"
                                            % (h_dev.numel() * 2 >> 20, stack.ws_bytes >> 20),
                    "multi_gpu": "replicas only (the path does not shard)"},
@@ -466,6 +472,8 @@ def main():
     ap.add_argument("--final-bp", type=int, default=0, help="final keep budget in basis points (sweep)")
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the CPU oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--schedule", default="step", choices=["step", "sigmoid"], help="retention schedule of the stack")
+    ap.add_argument("--x0", type=float, default=0.11, help="midpoint of the sigmoid schedule (0.11 / 0.24 / 0.41)")
     ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | attn_score | attn_fwd | "
                                                 "topk | compact | gemm")
     args = ap.parse_args()

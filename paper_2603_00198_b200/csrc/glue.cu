@@ -58,9 +58,9 @@ mamba_conv_split_kernel(int Tlen, int H, int p, int n, int G, int W, const T *__
     const int conv_dim = d_inner + 2 * gn;
     const int ld = 2 * d_inner + 2 * gn + H;
     const int cols = conv_dim + H;                       // conv channels, then the H dt columns
-    const size_t row = blockIdx.y;                       // b * Tlen + t
+    const size_t row = blockIdx.x;                       // b * Tlen + t (grid.x: no 65535 limit)
     const int t = (int)(row % Tlen);
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = blockIdx.y * blockDim.x + threadIdx.x;
     if (c >= cols) return;
     const T *base = zxbcdt + row * ld;
     if (c >= conv_dim) {
@@ -86,8 +86,8 @@ rope_split_kernel(int Hq, int Hkv, int d, double log2_theta, const int32_t *__re
                   const T *__restrict__ qkv, T *__restrict__ q_out, T *__restrict__ k_out, T *__restrict__ v_out) {
     const int half = d / 2;
     const int ld = (Hq + 2 * Hkv) * d;
-    const size_t row = blockIdx.y;
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t row = blockIdx.x;                       // grid.x: no 65535 limit
+    const int e = blockIdx.y * blockDim.x + threadIdx.x;
     const int n_rot = (Hq + Hkv) * half;
     const int n_v = Hkv * d;
     const T *base = qkv + row * ld;
@@ -118,6 +118,14 @@ __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
         f[2 * j] = __uint_as_float(w[j] << 16);
         f[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
     }
+}
+// SiLU for results that are stored as bf16: exp2 and reciprocal on the special-function unit (relative
+// error about 2^-21, far below the 2^-9 of the storage rounding) instead of the exact exp and division.
+__device__ __forceinline__ float silu_fast(float v) {
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-1.4426950408889634f * v));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+    return v * r;
 }
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -192,7 +200,7 @@ gated_rmsnorm_bf16_vec_kernel(int d_inner, int ld_z, float eps, const __nv_bfloa
         unpack8(zv[i], fz);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            g[i][j] = fy[j] * silu_f(fz[j]);
+            g[i][j] = fy[j] * silu_fast(fz[j]);
             ss = fmaf(g[i][j], g[i][j], ss);
         }
     }
@@ -223,10 +231,10 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
     const int conv_dim = d_inner + 2 * gn;
     const int ld = 2 * d_inner + 2 * gn + H;
     const int tiles = (Tlen + CONV_TT - 1) / CONV_TT;
-    const int b = blockIdx.y / tiles, t0 = (blockIdx.y % tiles) * CONV_TT;
+    const int b = blockIdx.x / tiles, t0 = (blockIdx.x % tiles) * CONV_TT;
     const int t1 = min(Tlen, t0 + CONV_TT);
     const size_t row0 = (size_t)b * Tlen;
-    if (blockIdx.x == gridDim.x - 1) {
+    if (blockIdx.y == gridDim.y - 1) {
         for (int e = threadIdx.x; e < (t1 - t0) * H; e += blockDim.x) {
             const int t = t0 + e / H, h = e % H;
             dt_out[(row0 + t) * H + h] =
@@ -234,7 +242,7 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
         }
         return;
     }
-    const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    const int c0 = (blockIdx.y * blockDim.x + threadIdx.x) * 8;
     if (c0 >= conv_dim) return;
     float w[8][4], bias[8];
 #pragma unroll
@@ -273,7 +281,7 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
                 acc = fmaf(w[j][1], h2[j], acc);
                 acc = fmaf(w[j][2], h1[j], acc);
                 acc = fmaf(w[j][3], cur[j], acc);
-                o[j] = silu_f(acc);
+                o[j] = silu_fast(acc);
                 h3[j] = h2[j]; h2[j] = h1[j]; h1[j] = cur[j];
             }
             if (tb + u < t1) *reinterpret_cast<uint4 *>(dst + (row0 + tb + u) * dst_ld) = pack8(o);
@@ -331,21 +339,17 @@ extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int 
         return STR_ERR_INVALID_ARG;
     if ((long long)Bz * T > 2147483647LL) return STR_ERR_UNSUPPORTED_SHAPE;
     const int cols = H * p + 2 * G * n + H;
-    dim3 grid(ceil_div(cols, 256), Bz * T);
+    dim3 grid(Bz * T, ceil_div(cols, 256));
     cudaStream_t st = (cudaStream_t)stream;
     const int d_inner_ = H * p, gn_ = G * n;
     if (dtype == STR_BF16 && W == 4 && d_inner_ % 8 == 0 && gn_ % 8 == 0 && H % 8 == 0 &&
         (((uintptr_t)zxbcdt | (uintptr_t)x_out | (uintptr_t)B_out | (uintptr_t)C_out | (uintptr_t)conv_w) & 15) == 0) {
         const int tiles = ceil_div(T, CONV_TT);
-        if ((long long)Bz * tiles > 65535) {
-            // grid.y limit: fall through to the generic kernel below
-        } else {
-            dim3 vgrid(ceil_div((d_inner_ + 2 * gn_) / 8, 256) + 1, Bz * tiles);
-            mamba_conv_split_bf16_vec_kernel<<<vgrid, 256, 0, st>>>(
-                T, H, p, n, G, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
-                (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out);
-            return str_launch_ok(ctx);
-        }
+        dim3 vgrid(Bz * tiles, ceil_div((d_inner_ + 2 * gn_) / 8, 256) + 1);
+        mamba_conv_split_bf16_vec_kernel<<<vgrid, 256, 0, st>>>(
+            T, H, p, n, G, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
+            (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out);
+        return str_launch_ok(ctx);
     }
     if (dtype == STR_BF16)
         mamba_conv_split_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
@@ -367,7 +371,7 @@ extern "C" int str_rope_split(str_ctx *ctx, int dtype, int Bz, int T, int Hq, in
         return STR_ERR_INVALID_ARG;
     if ((long long)Bz * T > 2147483647LL) return STR_ERR_UNSUPPORTED_SHAPE;
     const int work = (Hq + Hkv) * (d / 2) + Hkv * d;
-    dim3 grid(ceil_div(work, 256), Bz * T);
+    dim3 grid(Bz * T, ceil_div(work, 256));
     cudaStream_t st = (cudaStream_t)stream;
     const double l2t = log2((double)theta);
     if (dtype == STR_BF16)

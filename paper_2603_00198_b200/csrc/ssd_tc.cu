@@ -20,8 +20,8 @@
 // dS_c -> Xs_{c+1} -> dS_{c+1}  (single Xs buffer):
 //   warps 0-3, 14, 15  W_c from CB_c (one thread per token row and 64-column half; the upper halves of
 //                      row blocks 0 and 1 are all zero and are written by warps 0 and 1)
-//   warps 4-7          state update (one thread per state row n, 64 fp32 registers of state)
-//   warps 8-11         Xs_{c+1}, then the epilogue of chunk c (one thread per token row)
+//   warps 4-7          state update (one thread per state row n, 64 fp32 registers of state), then half of Xs_{c+1}
+//   warps 8-11         the other half of Xs_{c+1}, then the epilogue of chunk c (one thread per token row)
 //   warp 12            TMA producer (lane 0): B,C ring of 2, X ring of 3 (128-byte swizzle); then, all lanes,
 //                      the decay vectors of the chunk (cumulative sum, exponentials) into a ring of 4
 //   warp 13            MMA issuer; iteration c issues  CB_c, Y_intra_{c-1}, Y_inter_c, dS_c
@@ -94,6 +94,24 @@ __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { retur
 // Byte offset of K-slice ks (16 elements) inside a K-major operand stored as two 64-column, 16 KB halves.
 __device__ __forceinline__ uint32_t kmajor_off(int ks) { return (uint32_t)(ks >> 2) * TILE_16K + (uint32_t)(ks & 3) * 32; }
 
+// Half of Xs_c = exp(l_end - l_j) dt_j x_j (same swizzled layout as the X tile): 128 threads, four 16-byte
+// units each; `part` 0 and 1 are done by two different warp groups.
+__device__ __forceinline__ void scale_x_half(const uint8_t *x_tile, uint8_t *xs_tile, const float *dec_xw, int tid_g, int part) {
+    const uint4 *src = (const uint4 *)x_tile;
+    uint4 *dst = (uint4 *)xs_tile;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int u = tid_g + 128 * (4 * part + i);
+        const float sc = dec_xw[u >> 3];
+        const uint4 v = src[u];
+        uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            wv[j] = tc::pack_bf16x2(__uint_as_float(wv[j] << 16) * sc, __uint_as_float(wv[j] & 0xFFFF0000u) * sc);
+        dst[u] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    }
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_b,
               const __grid_constant__ CUtensorMap tmap_c, int Tlen, int H, int G, const float *__restrict__ dt,
@@ -114,13 +132,13 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     }
     if (*(volatile int *)status != 0) return;         // an earlier CTA failed: leave at once
     if (threadIdx.x == 0) {
-        for (int i = 0; i < X_SLOTS; ++i) { tc::mbar_init(bars + B_XF + i, 1); tc::mbar_init(bars + B_XE + i, 5); }
+        for (int i = 0; i < X_SLOTS; ++i) { tc::mbar_init(bars + B_XF + i, 1); tc::mbar_init(bars + B_XE + i, 9); }
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(bars + B_BCF + i, 1); tc::mbar_init(bars + B_BCE + i, 1);
             tc::mbar_init(bars + B_CBF + i, 1); tc::mbar_init(bars + B_WF + i, W_WARPS);
         }
         for (int i = 0; i < DEC_DEPTH; ++i) { tc::mbar_init(bars + B_DECF + i, 1); tc::mbar_init(bars + B_DECE + i, DEC_READERS); }
-        tc::mbar_init(bars + B_XSF, 4); tc::mbar_init(bars + B_DSF, 1); tc::mbar_init(bars + B_DSE, 4);
+        tc::mbar_init(bars + B_XSF, 8); tc::mbar_init(bars + B_DSF, 1); tc::mbar_init(bars + B_DSE, 4);
         tc::mbar_init(bars + B_SF, 4); tc::mbar_init(bars + B_YF, 1); tc::mbar_init(bars + B_YE, 4);
         abort_flag[0] = 0; abort_flag[1] = 0;
         tc::fence_mbar_init();
@@ -388,12 +406,26 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // ------------------------------------------------------------------ state update
         const int quad = warp & 3, row = quad * 32 + lane;        // row = state index n
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const int tid_s = threadIdx.x - 128;
         float S[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) S[i] = 0.f;
         bool ok = true;
+        // this group's half of Xs_c (the other half is the epilogue group's); chunk 0 before the loop, chunk c+1
+        // right after the state update of chunk c (the Xs buffer is free once dS_c has completed)
+        auto xs_half = [&](int c) -> bool {
+            const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
+            if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) return false;
+            if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) return false;
+            scale_x_half(smem + OFF_X + sx * TILE_16K, smem + OFF_XS, decs + d * DEC_FLOATS + D_XW, tid_s, 0);
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
+            return true;
+        };
+        ok = xs_half(0);
 #pragma unroll 1
-        for (int c = 0; c < nchunks; ++c) {
+        for (int c = 0; c < nchunks && ok; ++c) {
             const int d = c & (DEC_DEPTH - 1);
             if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
             const float eend = decs[d * DEC_FLOATS + D_EEND];
@@ -428,6 +460,8 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             tc::fence_proxy_async();
             warp_arrive(bars + B_SF, lane);
             if (quad == SSD_TRQ) SSD_TR(5, c, 2);
+            if (c + 1 < nchunks && !xs_half(c + 1)) { ok = false; break; }
+            if (quad == SSD_TRQ) SSD_TR(5, c, 3);
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         if (ok && final_state) {
@@ -453,19 +487,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
                 if (c > 0 && !tc::mbar_wait(bars + B_DSF, (c - 1) & 1, abort_flag)) { ok = false; break; }   // Xs buffer free
                 if (quad == SSD_TRQ) SSD_TR(6, c, 1);
-                const uint4 *src = (const uint4 *)(smem + OFF_X + sx * TILE_16K);
-                uint4 *dst = (uint4 *)(smem + OFF_XS);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int u = tid_g + 128 * i;
-                    const float sc = dec[D_XW + (u >> 3)];
-                    const uint4 v = src[u];
-                    uint32_t wv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        wv[j] = tc::pack_bf16x2(__uint_as_float(wv[j] << 16) * sc, __uint_as_float(wv[j] & 0xFFFF0000u) * sc);
-                    dst[u] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
-                }
+                scale_x_half(smem + OFF_X + sx * TILE_16K, smem + OFF_XS, dec + D_XW, tid_g, 1);
                 tc::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }

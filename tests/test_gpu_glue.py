@@ -45,7 +45,8 @@ def test_rmsnorm(ctx, dtype, rows, D):
 
 @pytest.mark.parametrize("dtype,Bz,T,H,p,n,G", [("bf16", 1, 300, 16, 64, 128, 2), ("f32", 2, 70, 8, 32, 16, 1),
                                                 ("bf16", 3, 70, 8, 64, 64, 1), ("bf16", 2, 33, 4, 16, 32, 2),
-                                                ("bf16", 1, 2, 8, 64, 128, 8)])
+                                                ("bf16", 1, 2, 8, 64, 128, 8), ("bf16", 2, 33000, 8, 8, 8, 1),
+                                                ("f32", 1, 66000, 2, 4, 4, 1)])
 def test_conv_split_and_gated_norm(ctx, dtype, Bz, T, H, p, n, G):
     d_inner, gn = H * p, G * n
     ld = 2 * d_inner + 2 * gn + H
@@ -69,7 +70,9 @@ def test_conv_split_and_gated_norm(ctx, dtype, Bz, T, H, p, n, G):
     assert max_rel_err(got, ref) <= TOL[dtype]
 
 
-@pytest.mark.parametrize("dtype,Bz,T,Hq,Hkv,d", [("bf16", 1, 200, 8, 2, 128), ("f32", 2, 50, 4, 4, 32)])
+# the last case has more than 65535 rows (batch 4 of the 16512-token attention layers has 66048)
+@pytest.mark.parametrize("dtype,Bz,T,Hq,Hkv,d", [("bf16", 1, 200, 8, 2, 128), ("f32", 2, 50, 4, 4, 32),
+                                                   ("bf16", 2, 35000, 2, 1, 16)])
 def test_rope_split(ctx, dtype, Bz, T, Hq, Hkv, d):
     g = inputs.rng(54, T)
     qkv = inputs.to_grid(g.standard_normal((Bz * T, (Hq + 2 * Hkv) * d), dtype=np.float32), dtype)

@@ -115,3 +115,35 @@ def test_host_buffer_entry_point_matches_device_entry_point(ctx):
     iout = torch.empty((1, K[-1] + M), dtype=torch.int32).pin_memory()
     binding.str_stack_prefill_host(st, hin, hout, iout)
     assert bool((hout == out.cpu()).all()) and bool((iout == idx.cpu()).all())
+
+
+def test_all_layer_sigmoid_schedule(ctx):
+    """Every layer cuts a little (the paper's all-layer sigmoid schedule): Mamba and attention layers both
+    select inside the stack, with token counts that are not multiples of any tile."""
+    n_vis, M = 1000, 12
+    pattern = "MMAMMA"
+    layers = inputs.stack_params(65, pattern, MS, AS, "bf16")
+    h0 = inputs.hidden_inputs(65, n_vis + M, 128, "bf16")
+    alpha = binding.str_sigmoid_schedule_bp(len(pattern), 20.0, 0.24, 1.0, 0.125)
+    assert alpha == [int(round(a * 10000)) for a in oracle.sigmoid_schedule(len(pattern), 20.0, 0.24, 1.0, 0.125)]
+    K = binding.str_schedule_keep_counts(alpha, n_vis, 16)
+    assert K == oracle.schedule_keep_counts(alpha, n_vis, 16)
+    reducing = [l for l, (a, b) in enumerate(zip([n_vis] + K, K)) if b < a]
+    assert len(reducing) >= 5 and 2 in reducing                      # Mamba and attention layers both cut
+    st = binding.Stack(ctx, layers, "bf16", 1, n_vis, M, K)
+    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, "bf16"), want_trace=True)
+    assert [t["layer"] for t in tr] == reducing and out.shape == (1, K[-1] + M, 128)
+    ref, rpos, ridx, trace = oracle.stack_prefill(h0[0], M, layers, K, oracle.round_to_bf16)
+    gi = idx[0].cpu().numpy()
+    assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], np.arange(n_vis, n_vis + M))
+    # layer 0 sees identical tokens on both sides: its selection must match up to near-ties
+    assert_kept_matches(tr[0]["kept"][0].cpu().numpy(), trace[0]["kept"], trace[0]["scores"], tol=5e-3)
+    # every later selection is the oracle's rule applied to the scores the GPU produced
+    for t in tr:
+        assert np.array_equal(t["kept"][0].cpu().numpy(), oracle.topk_select(t["scores"][0].cpu().numpy(), K[t["layer"]]))
+    common, a, c = np.intersect1d(gi, ridx, return_indices=True)
+    assert len(common) >= 0.9 * len(ridx)
+    # six cuts in a row: a near-tie swap at any of them changes the context of every later row, so only the
+    # bulk of the surviving rows is compared, loosely
+    row_err = np.abs(host(out)[0][a] - ref[c]).max(axis=1) / np.abs(ref).max()
+    assert np.median(row_err) <= 5e-2
