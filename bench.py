@@ -69,17 +69,18 @@ def work_model(cfg, keep_counts):
     n_cur = cfg["n_vis"]
     for kind, K in zip(cfg["pattern"], keep_counts):
         T = n_cur + M
+        To = min(K, n_cur) + M          # a reducing layer projects only the rows it keeps
         if kind == "M":
-            w["gemm"]["flops"] += 2.0 * Bz * T * D * dip + 2.0 * Bz * T * d_inner * D
-            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dip) + D * dip) + 2.0 * (Bz * T * (d_inner + 2 * D) + d_inner * D)
+            w["gemm"]["flops"] += 2.0 * Bz * T * D * dip + 2.0 * Bz * To * d_inner * D
+            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dip) + D * dip) + 2.0 * (Bz * To * (d_inner + 2 * D) + d_inner * D)
             w["ssd_scan"]["flops"] += Bz * T * (G * 2 * n * (Q + 1) / 2 + H * (2 * p * (Q + 1) / 2 + 4 * n * p))
             w["ssd_scan"]["bytes"] += Bz * T * (2 * (2 * H * p + 2 * G * n) + 4 * H)
             if K < n_cur:
                 w["mamba_score"]["flops"] += Bz * n_cur * 2.0 * M * n * G
                 w["mamba_score"]["bytes"] += Bz * n_cur * (2 * G * n + 4 * H + 4)
         else:
-            w["gemm"]["flops"] += 2.0 * Bz * T * D * dqkv + 2.0 * Bz * T * Hq * d * D
-            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dqkv) + D * dqkv) + 2.0 * (Bz * T * (Hq * d + 2 * D) + Hq * d * D)
+            w["gemm"]["flops"] += 2.0 * Bz * T * D * dqkv + 2.0 * Bz * To * Hq * d * D
+            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dqkv) + D * dqkv) + 2.0 * (Bz * To * (Hq * d + 2 * D) + Hq * d * D)
             w["attn_fwd"]["flops"] += Bz * Hq * 4.0 * d * T * (T + 1) / 2
             w["attn_fwd"]["bytes"] += Bz * T * 2.0 * (2 * Hq * d + 2 * Hkv * d)
             if K < n_cur:
@@ -88,6 +89,8 @@ def work_model(cfg, keep_counts):
         if K < n_cur:
             w["topk"]["bytes"] += Bz * (4.0 * n_cur + 4.0 * K)
             w["compact"]["bytes"] += Bz * 2.0 * (K + M) * (2 * D + 8)
+            if kind == "A":
+                w["compact"]["bytes"] += Bz * 2.0 * (K + M) * 2 * Hq * d     # the survivors' attention outputs
             n_cur = K
     return w
 

@@ -35,3 +35,5 @@ int str_mamba_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int n_vi
 bool str_attn_importance_tc_supported(const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k);
 int str_attn_importance_tc(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k,
                            float scale, float *scores, float *workspace, cudaStream_t st);
+int str_gated_rmsnorm_gather(str_ctx *ctx, int dtype, int Bz, int T_in, int n_vis, int n_text, int k, int d_inner, int ld_z,
+                             float eps, const void *y, const void *z, const int32_t *kept, void *out, void *stream);

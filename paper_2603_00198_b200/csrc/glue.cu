@@ -29,13 +29,25 @@ rmsnorm_kernel(int D, float eps, const T *__restrict__ in, T *__restrict__ out) 
     for (int c = threadIdx.x; c < D; c += blockDim.x) stf(o + c, ldf(r + c) * inv);
 }
 
+// Source row of output row r when the rows are gathered on the fly (the same map as str_compact: per
+// sequence the k kept visual rows, then the text rows); the identity when kept == nullptr.
+struct RowGather { const int32_t *kept; int T_in, n_vis, k, T_out; };
+__device__ __forceinline__ size_t gather_src_row(const RowGather &g, size_t r) {
+    if (!g.kept) return r;
+    const size_t b = r / g.T_out;
+    const int j = (int)(r - b * g.T_out);
+    const int src = j < g.k ? __ldg(g.kept + b * g.k + j) : g.n_vis + (j - g.k);
+    return b * g.T_in + src;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 gated_rmsnorm_kernel(int d_inner, int ld_z, float eps, const T *__restrict__ y, const T *__restrict__ z,
-                     T *__restrict__ out) {
+                     T *__restrict__ out, RowGather rg) {
     __shared__ float red[32];
-    const T *yr = y + (size_t)blockIdx.x * d_inner;
-    const T *zr = z + (size_t)blockIdx.x * ld_z;
+    const size_t srow = gather_src_row(rg, blockIdx.x);
+    const T *yr = y + srow * d_inner;
+    const T *zr = z + srow * ld_z;
     T *o = out + (size_t)blockIdx.x * d_inner;
     float ss = 0.f;
     for (int c = threadIdx.x; c < d_inner; c += blockDim.x) {
@@ -178,11 +190,12 @@ rmsnorm_bf16_vec_kernel(int rows, int D, float eps, const __nv_bfloat16 *__restr
 template <int VPT>
 __global__ void __launch_bounds__(256)
 gated_rmsnorm_bf16_vec_kernel(int d_inner, int ld_z, float eps, const __nv_bfloat16 *__restrict__ y,
-                              const __nv_bfloat16 *__restrict__ z, __nv_bfloat16 *__restrict__ out) {
+                              const __nv_bfloat16 *__restrict__ z, __nv_bfloat16 *__restrict__ out, RowGather rg) {
     __shared__ float red[32];
     const int nvec = d_inner >> 3;
-    const uint4 *yr = reinterpret_cast<const uint4 *>(y + (size_t)blockIdx.x * d_inner);
-    const uint4 *zr = reinterpret_cast<const uint4 *>(z + (size_t)blockIdx.x * ld_z);
+    const size_t srow = gather_src_row(rg, blockIdx.x);
+    const uint4 *yr = reinterpret_cast<const uint4 *>(y + srow * d_inner);
+    const uint4 *zr = reinterpret_cast<const uint4 *>(z + srow * ld_z);
     uint4 *o = reinterpret_cast<uint4 *>(out + (size_t)blockIdx.x * d_inner);
     uint4 yv[VPT], zv[VPT];
 #pragma unroll
@@ -309,24 +322,44 @@ extern "C" int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, 
     return str_launch_ok(ctx);
 }
 
+static int launch_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps, const void *y,
+                                const void *z, void *out, RowGather rg, cudaStream_t st) {
+    if (dtype == STR_BF16 && d_inner % 8 == 0 && ld_z % 8 == 0 && d_inner <= 256 * 8 * 4 &&
+        (((uintptr_t)y | (uintptr_t)z | (uintptr_t)out) & 15) == 0)
+        gated_rmsnorm_bf16_vec_kernel<4><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const __nv_bfloat16 *)y,
+                                                                (const __nv_bfloat16 *)z, (__nv_bfloat16 *)out, rg);
+    else if (dtype == STR_BF16)
+        gated_rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const __nv_bfloat16 *)y,
+                                                                 (const __nv_bfloat16 *)z, (__nv_bfloat16 *)out, rg);
+    else
+        gated_rmsnorm_kernel<float><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const float *)y, (const float *)z,
+                                                         (float *)out, rg);
+    return str_launch_ok(ctx);
+}
+
 extern "C" int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps,
                                  const void *y, const void *z, void *out, void *stream) {
     StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
     if (!ctx || !y || !z || !out || rows < 0 || d_inner <= 0 || ld_z < d_inner || !STR_DTYPE_OK(dtype))
         return STR_ERR_INVALID_ARG;
     if (rows == 0) return STR_OK;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (dtype == STR_BF16 && d_inner % 8 == 0 && ld_z % 8 == 0 && d_inner <= 256 * 8 * 4 &&
-        (((uintptr_t)y | (uintptr_t)z | (uintptr_t)out) & 15) == 0)
-        gated_rmsnorm_bf16_vec_kernel<4><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const __nv_bfloat16 *)y,
-                                                                (const __nv_bfloat16 *)z, (__nv_bfloat16 *)out);
-    else if (dtype == STR_BF16)
-        gated_rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const __nv_bfloat16 *)y,
-                                                                 (const __nv_bfloat16 *)z, (__nv_bfloat16 *)out);
-    else
-        gated_rmsnorm_kernel<float><<<rows, 256, 0, st>>>(d_inner, ld_z, eps, (const float *)y, (const float *)z,
-                                                         (float *)out);
-    return str_launch_ok(ctx);
+    return launch_gated_rmsnorm(ctx, dtype, rows, d_inner, ld_z, eps, y, z, out, RowGather{nullptr, 0, 0, 0, 0},
+                                (cudaStream_t)stream);
+}
+
+// Internal (stack driver): the same operation on gathered rows.  Output row (b, j) takes y and z from input row
+// kept[b][j] for j < k and from text row n_vis + (j - k) after that, so the rows a reducing layer is about to
+// drop are never normalised or projected.
+int str_gated_rmsnorm_gather(str_ctx *ctx, int dtype, int Bz, int T_in, int n_vis, int n_text, int k, int d_inner, int ld_z,
+                             float eps, const void *y, const void *z, const int32_t *kept, void *out, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
+    if (!ctx || !y || !z || !out || !kept || Bz <= 0 || k < 0 || k > n_vis || T_in != n_vis + n_text || d_inner <= 0 ||
+        ld_z < d_inner || !STR_DTYPE_OK(dtype))
+        return STR_ERR_INVALID_ARG;
+    const int rows = Bz * (k + n_text);
+    if (rows == 0) return STR_OK;
+    return launch_gated_rmsnorm(ctx, dtype, rows, d_inner, ld_z, eps, y, z, out, RowGather{kept, T_in, n_vis, k, k + n_text},
+                                (cudaStream_t)stream);
 }
 
 extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, int n, int G, int W,

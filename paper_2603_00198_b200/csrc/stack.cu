@@ -148,6 +148,13 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
         void *mix_out = (last && !reduce) ? hidden_out : hid[hsel];
 
         STR_TRY(str_rmsnorm(ctx, dtype, rows, D, d->norm_eps, cur, normed, stream));
+        // A reducing layer selects BEFORE the mixer's epilogue: the score only needs the projections, so the rows
+        // about to be dropped skip the gate / norm / output projection (their inputs still feed the scan state
+        // and the attention keys).  The surviving rows come out bit-identical to computing every row first.
+        void *dst = !reduce ? mix_out : (last ? hidden_out : hid[hsel]);
+        int32_t *pdst = (last && positions_out) ? positions_out : pos[1 - psel];
+        int32_t *idst = (last && idx_map_out) ? idx_map_out : idx[1 - psel];
+        const int rows_out = reduce ? Bz * (K + M) : rows;
         if (L.kind == STR_LAYER_MAMBA) {
             const int d_inner = d->H * d->p, gn = d->G * d->n, dip = 2 * d_inner + 2 * gn + d->H;
             STR_TRY(str_gemm(ctx, dtype, rows, dip, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
@@ -160,8 +167,18 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
                 str_ssm_score_shape ss = {Bz, T, d->H, d->n, d->G, dtype};
                 STR_TRY(str_mamba_importance(ctx, &ss, n_cur, M, bufB, bufC, dt, scores, sub, r.sub_bytes, stream));
             }
-            STR_TRY(str_gated_rmsnorm(ctx, dtype, rows, d_inner, dip, d->norm_eps, bufY, proj, bufA, stream));
-            STR_TRY(str_gemm(ctx, dtype, rows, D, d_inner, bufA, L.w_out, cur, mix_out, sub, r.sub_bytes, stream));
+            if (reduce) {
+                STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));
+                // residual rows, positions and the index map of the survivors (normed is free after in_proj)
+                STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, cur, pos[psel], idx[psel], kept, normed, pdst, idst,
+                                    stream));
+                STR_TRY(str_gated_rmsnorm_gather(ctx, dtype, Bz, T, n_cur, M, K, d_inner, dip, d->norm_eps, bufY, proj, kept,
+                                                 bufA, stream));
+                STR_TRY(str_gemm(ctx, dtype, rows_out, D, d_inner, bufA, L.w_out, normed, dst, sub, r.sub_bytes, stream));
+            } else {
+                STR_TRY(str_gated_rmsnorm(ctx, dtype, rows, d_inner, dip, d->norm_eps, bufY, proj, bufA, stream));
+                STR_TRY(str_gemm(ctx, dtype, rows, D, d_inner, bufA, L.w_out, cur, dst, sub, r.sub_bytes, stream));
+            }
         } else {
             const int qd = d->Hq * d->d, kd = d->Hkv * d->d;
             STR_TRY(str_gemm(ctx, dtype, rows, qd + 2 * kd, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
@@ -174,28 +191,27 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
                 str_attn_score_shape ss = {Bz, T, d->Hq, d->Hkv, d->d, dtype};
                 STR_TRY(str_attn_importance(ctx, &ss, n_cur, M, bufA, bufB, scale, scores, sub, r.sub_bytes, stream));
             }
-            STR_TRY(str_gemm(ctx, dtype, rows, D, qd, bufY, L.w_out, cur, mix_out, sub, r.sub_bytes, stream));
+            if (reduce) {
+                STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));
+                STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, cur, pos[psel], idx[psel], kept, normed, pdst, idst,
+                                    stream));
+                // the attention outputs of the survivors (q is no longer needed: its buffer takes them)
+                STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, qd, dtype, bufY, nullptr, nullptr, kept, bufA, nullptr, nullptr,
+                                    stream));
+                STR_TRY(str_gemm(ctx, dtype, rows_out, D, qd, bufA, L.w_out, normed, dst, sub, r.sub_bytes, stream));
+            } else {
+                STR_TRY(str_gemm(ctx, dtype, rows, D, qd, bufY, L.w_out, cur, dst, sub, r.sub_bytes, stream));
+            }
         }
+        cur = dst;
+        if (dst == hid[0]) hsel = 1;
+        else if (dst == hid[1]) hsel = 0;
         if (reduce) {
-            STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));
-            void *dst = last ? hidden_out : hid[1 - hsel];
-            int32_t *pdst = (last && positions_out) ? positions_out : pos[1 - psel];
-            int32_t *idst = (last && idx_map_out) ? idx_map_out : idx[1 - psel];
-            STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, mix_out, pos[psel], idx[psel], kept, dst, pdst,
-                                idst, stream));
-            cur = dst;
-            hsel = (dst == hid[0]) ? 1 : 0;
             psel = 1 - psel;
             kept_off += (size_t)Bz * K;
             score_off += (size_t)Bz * n_cur;
             n_cur = K;
-            if (last) {
-                // positions/idx already written where the caller wants them
-                return STR_OK;
-            }
-        } else {
-            cur = mix_out;
-            hsel = 1 - hsel;
+            if (last) return STR_OK;          // positions / index map already written where the caller wants them
         }
     }
     // last layer did not reduce: hidden_out holds the result; hand back the carried ids
