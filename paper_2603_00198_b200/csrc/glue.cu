@@ -229,12 +229,18 @@ gated_rmsnorm_bf16_vec_kernel(int d_inner, int ld_z, float eps, const __nv_bfloa
     }
 }
 
-// Mamba-2 pre-scan step, width-4 conv: one thread owns 8 consecutive conv channels and walks CONV_TT
+// Mamba-2 pre-scan step, width-4 conv: one thread owns 4 consecutive conv channels and walks CONV_TT
 // consecutive tokens with the three previous inputs held in registers, so every input element is
-// read once (plus a 3-token halo per tile) and every output written once, all as 16-byte vectors.
-// The last block column handles the dt columns.
-constexpr int CONV_TT = 32;
-__global__ void __launch_bounds__(256)
+// read once (plus a 3-token halo per tile) and every output written once, as 8-byte vectors (a warp
+// covers 256 contiguous bytes of a row).  Eight loads are in flight per thread and three CTAs fit an
+// SM, which is what it takes to keep HBM busy from a kernel this short.  The last block row handles the
+// dt columns.
+constexpr int CONV_TT = 32, CONV_CPT = 4, CONV_UNROLL = 8;
+__device__ __forceinline__ void unpack4(const uint2 &v, float (&f)[4]) {
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+}
+__global__ void __launch_bounds__(256, 3)
 mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __nv_bfloat16 *__restrict__ zxbcdt,
                                  const float *__restrict__ conv_w, const float *__restrict__ conv_b,
                                  const float *__restrict__ dt_bias, __nv_bfloat16 *__restrict__ x_out,
@@ -255,11 +261,11 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
         }
         return;
     }
-    const int c0 = (blockIdx.y * blockDim.x + threadIdx.x) * 8;
+    const int c0 = (blockIdx.y * blockDim.x + threadIdx.x) * CONV_CPT;
     if (c0 >= conv_dim) return;
-    float w[8][4], bias[8];
+    float w[CONV_CPT][4], bias[CONV_CPT];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < CONV_CPT; ++j) {
         const float4 wv = __ldg(reinterpret_cast<const float4 *>(conv_w) + c0 + j);
         w[j][0] = wv.x; w[j][1] = wv.y; w[j][2] = wv.z; w[j][3] = wv.w;
         bias[j] = __ldg(conv_b + c0 + j);
@@ -270,25 +276,25 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
     else if (c0 < d_inner + gn) { dst = B_out + (c0 - d_inner); dst_ld = gn; }
     else { dst = C_out + (c0 - d_inner - gn); dst_ld = gn; }
     const __nv_bfloat16 *src = zxbcdt + d_inner + c0;
-    float h3[8], h2[8], h1[8];     // inputs of tokens t-3, t-2, t-1
+    float h3[CONV_CPT], h2[CONV_CPT], h1[CONV_CPT];     // inputs of tokens t-3, t-2, t-1
     {
-        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-        unpack8(t0 >= 3 ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + t0 - 3) * ld)) : zero, h3);
-        unpack8(t0 >= 2 ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + t0 - 2) * ld)) : zero, h2);
-        unpack8(t0 >= 1 ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + t0 - 1) * ld)) : zero, h1);
+        const uint2 zero = make_uint2(0u, 0u);
+        unpack4(t0 >= 3 ? __ldg(reinterpret_cast<const uint2 *>(src + (row0 + t0 - 3) * ld)) : zero, h3);
+        unpack4(t0 >= 2 ? __ldg(reinterpret_cast<const uint2 *>(src + (row0 + t0 - 2) * ld)) : zero, h2);
+        unpack4(t0 >= 1 ? __ldg(reinterpret_cast<const uint2 *>(src + (row0 + t0 - 1) * ld)) : zero, h1);
     }
-    for (int tb = t0; tb < t1; tb += 4) {
-        uint4 raw[4];
+#pragma unroll 1
+    for (int tb = t0; tb < t1; tb += CONV_UNROLL) {
+        uint2 raw[CONV_UNROLL];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-            raw[u] = (tb + u < t1) ? __ldg(reinterpret_cast<const uint4 *>(src + (row0 + tb + u) * ld))
-                                   : make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < CONV_UNROLL; ++u)
+            raw[u] = (tb + u < t1) ? __ldg(reinterpret_cast<const uint2 *>(src + (row0 + tb + u) * ld)) : make_uint2(0u, 0u);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            float cur[8], o[8];
-            unpack8(raw[u], cur);
+        for (int u = 0; u < CONV_UNROLL; ++u) {
+            float cur[CONV_CPT], o[CONV_CPT];
+            unpack4(raw[u], cur);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < CONV_CPT; ++j) {
                 float acc = bias[j];
                 acc = fmaf(w[j][0], h3[j], acc);
                 acc = fmaf(w[j][1], h2[j], acc);
@@ -297,7 +303,8 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
                 o[j] = silu_fast(acc);
                 h3[j] = h2[j]; h2[j] = h1[j]; h1[j] = cur[j];
             }
-            if (tb + u < t1) *reinterpret_cast<uint4 *>(dst + (row0 + tb + u) * dst_ld) = pack8(o);
+            if (tb + u < t1)
+                *reinterpret_cast<uint2 *>(dst + (row0 + tb + u) * dst_ld) = make_uint2(pack2(o[0], o[1]), pack2(o[2], o[3]));
         }
     }
 }
@@ -378,7 +385,7 @@ extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int 
     if (dtype == STR_BF16 && W == 4 && d_inner_ % 8 == 0 && gn_ % 8 == 0 && H % 8 == 0 &&
         (((uintptr_t)zxbcdt | (uintptr_t)x_out | (uintptr_t)B_out | (uintptr_t)C_out | (uintptr_t)conv_w) & 15) == 0) {
         const int tiles = ceil_div(T, CONV_TT);
-        dim3 vgrid(Bz * tiles, ceil_div((d_inner_ + 2 * gn_) / 8, 256) + 1);
+        dim3 vgrid(Bz * tiles, ceil_div((d_inner_ + 2 * gn_) / CONV_CPT, 256) + 1);
         mamba_conv_split_bf16_vec_kernel<<<vgrid, 256, 0, st>>>(
             T, H, p, n, G, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
             (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out);
