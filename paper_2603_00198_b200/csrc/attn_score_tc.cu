@@ -435,16 +435,9 @@ int str_attn_importance_tc(str_ctx *ctx, const str_attn_score_shape *s, int n_vi
     while (stages > 2 && fixed2 + (size_t)stages * cs::K_TILE > (size_t)ctx->max_smem_optin) --stages;
     const size_t smem2 = fixed2 + (size_t)stages * cs::K_TILE;
     if (smem2 > (size_t)ctx->max_smem_optin || rs::SMEM_BYTES > (size_t)ctx->max_smem_optin) return STR_ERR_UNSUPPORTED_SHAPE;
-    static bool attr1 = false;
-    static size_t attr2 = 0;
-    if (!attr1) {
-        STR_CUDA_OK(cudaFuncSetAttribute(attn_rowstats_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs::SMEM_BYTES));
-        attr1 = true;
-    }
-    if (smem2 > attr2) {
-        STR_CUDA_OK(cudaFuncSetAttribute(attn_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
-        attr2 = smem2;
-    }
+    rc = str_ensure_smem(ctx, STR_SMEM_ATTN_ROWSTATS, attn_rowstats_tc_kernel, rs::SMEM_BYTES);
+    if (rc == STR_OK) rc = str_ensure_smem(ctx, STR_SMEM_ATTN_COLSUM, attn_colsum_tc_kernel, smem2);
+    if (rc != STR_OK) return rc;
     dim3 g1(nseg, s->Hq * m_tiles, s->Bz);
     attn_rowstats_tc_kernel<<<g1, NUM_THREADS, rs::SMEM_BYTES, st>>>(tq128, tk256, s->Hq, s->Hkv, n_vis, n_text, m_tiles, scale_log2,
                                                                       ws_max, ws_sum, ctx->status_dev);

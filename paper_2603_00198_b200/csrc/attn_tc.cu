@@ -290,11 +290,8 @@ int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, const void *q, co
     if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tk, k, (uint64_t)s->Hkv * HD, (uint64_t)s->T, (uint64_t)s->Bz, BKV);
     if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tv, v, (uint64_t)s->Hkv * HD, (uint64_t)s->T, (uint64_t)s->Bz, BKV);
     if (rc != STR_OK) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        STR_CUDA_OK(cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-        attr_set = true;
-    }
+    rc = str_ensure_smem(ctx, STR_SMEM_ATTN_FWD, attn_fwd_tc_kernel, SMEM_BYTES);
+    if (rc != STR_OK) return rc;
     dim3 grid(ceil_div(s->T, 2 * BQ), s->Hq, s->Bz);
     attn_fwd_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, s->T, s->Hq, s->Hkv,
                                                              scale * 1.4426950408889634f, (__nv_bfloat16 *)o,

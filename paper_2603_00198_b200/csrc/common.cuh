@@ -22,6 +22,7 @@ struct str_ctx {
     int *status_dev;          // device status word: 0 or the first STR_ERR_* a kernel recorded
     void *encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), or nullptr
     long long launches;       // host-side count of kernels launched through this context
+    size_t smem_attr[8];      // dynamic shared memory already opted into on this device, per tensor-core kernel
     bool prof_on;             // record an event pair per leaf call
     std::vector<str_prof_span> prof_spans;
     std::vector<cudaEvent_t> prof_free;
@@ -53,6 +54,20 @@ struct StrProfScope {
 static inline int str_launch_ok(str_ctx *ctx, int n = 1) {
     ctx->launches += n;
     return cudaGetLastError() == cudaSuccess ? STR_OK : STR_ERR_CUDA;
+}
+
+// Opt a kernel into `bytes` of dynamic shared memory once per context (the attribute belongs to the device the
+// context was created on, so it is tracked per context, not per process).
+enum { STR_SMEM_GEMM = 0, STR_SMEM_SSD, STR_SMEM_ATTN_FWD, STR_SMEM_MAMBA_SCORE, STR_SMEM_ATTN_ROWSTATS, STR_SMEM_ATTN_COLSUM };
+template <typename F>
+static inline int str_ensure_smem(str_ctx *ctx, int slot, F kernel, size_t bytes) {
+    // The attribute belongs to the device's copy of the kernel, not to this context: every context raises it to
+    // the same value (the device's opt-in maximum), so contexts that share a device never lower it for each other.
+    if (bytes > (size_t)ctx->max_smem_optin) return STR_ERR_UNSUPPORTED_SHAPE;
+    if (ctx->smem_attr[slot]) return STR_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin) != cudaSuccess) return STR_ERR_CUDA;
+    ctx->smem_attr[slot] = (size_t)ctx->max_smem_optin;
+    return STR_OK;
 }
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

@@ -15,6 +15,7 @@ extern "C" int str_create(int device, str_ctx **out) {
     c->device = device;
     c->launches = 0;
     c->prof_on = false;
+    for (size_t &v : c->smem_attr) v = 0;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return STR_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;

@@ -185,11 +185,8 @@ int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w,
     if (rc != STR_OK) return rc;
     rc = str_make_tmap_2d_bf16(ctx, &tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN, BK, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != STR_OK) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        STR_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-        attr_set = true;
-    }
+    rc = str_ensure_smem(ctx, STR_SMEM_GEMM, gemm_tc_kernel, SMEM_BYTES);
+    if (rc != STR_OK) return rc;
     const int tiles = ceil_div(M, BM) * ceil_div(N, BN);
     const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tw, M, N, K, (const __nv_bfloat16 *)residual,

@@ -228,11 +228,8 @@ int str_mamba_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int n_vi
     int rc = str_make_tmap_3d_bf16_sw128(ctx, &tb, B, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz, TI);
     if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tcm, C, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz, (uint32_t)n_pad);
     if (rc != STR_OK) return rc;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        STR_CUDA_OK(cudaFuncSetAttribute(mamba_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_smem = smem;
-    }
+    rc = str_ensure_smem(ctx, STR_SMEM_MAMBA_SCORE, mamba_score_tc_kernel, smem);
+    if (rc != STR_OK) return rc;
     const int tiles = ceil_div(n_vis, TI);
     const int per_seq = ceil_div(ctx->sm_count, s->Bz);
     dim3 grid(tiles < per_seq ? tiles : per_seq, s->Bz);

@@ -563,11 +563,8 @@ int str_ssd_tc(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float 
     if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tb, B, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz, Q);
     if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tcm, C, (uint64_t)s->G * NS, (uint64_t)s->T, (uint64_t)s->Bz, Q);
     if (rc != STR_OK) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        STR_CUDA_OK(cudaFuncSetAttribute(ssd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-        attr_set = true;
-    }
+    rc = str_ensure_smem(ctx, STR_SMEM_SSD, ssd_tc_kernel, SMEM_BYTES);
+    if (rc != STR_OK) return rc;
     dim3 grid(s->H, s->Bz);
     ssd_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tx, tb, tcm, s->T, s->H, s->G, dt, A, (__nv_bfloat16 *)y,
                                                         final_state, ctx->status_dev);
