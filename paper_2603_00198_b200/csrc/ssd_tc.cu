@@ -20,10 +20,12 @@
 // dS_c -> Xs_{c+1} -> dS_{c+1}  (single Xs buffer):
 //   warps 0-3, 14, 15  W_c from CB_c (one thread per token row and 64-column half; the upper halves of
 //                      row blocks 0 and 1 are all zero and are written by warps 0 and 1)
-//   warps 4-7          state update (one thread per state row n, 64 fp32 registers of state), then half of Xs_{c+1}
+//   warps 4-7          state update (one thread per state row n, 64 fp32 registers of state), then half of Xs_{c+1};
+//                      lane 0 of warp 4 is the TMA producer (B,C ring of 2, X ring of 3, 128-byte swizzle): seeing
+//                      dS_c complete is what frees the slots of chunk c+2, so there are no slot-release barriers
 //   warps 8-11         the other half of Xs_{c+1}, then the epilogue of chunk c (one thread per token row)
-//   warp 12            TMA producer (lane 0): B,C ring of 2, X ring of 3 (128-byte swizzle); then, all lanes,
-//                      the decay vectors of the chunk (cumulative sum, exponentials) into a ring of 4
+//   warp 12            the decay vectors of each chunk (cumulative sum, exponentials) into a ring of 4; depends on
+//                      dt only and runs up to three chunks ahead of its readers
 //   warp 13            MMA issuer; iteration c issues  CB_c, Y_intra_{c-1}, Y_inter_c, dS_c
 // Loops are kept rolled where registers allow: the instruction footprint of all roles together has to
 // stay inside the instruction cache, or every role slows down together.
@@ -68,7 +70,7 @@ constexpr int OFF_BARS = OFF_DEC + DEC_DEPTH * DEC_FLOATS * 4;
 // decay vectors of one chunk (floats): log2-domain cumulative decay, dt, column / state / row factors
 constexpr int D_LS = 0, D_DT = 128, D_COLF = 256, D_XW = 384, D_ROWF = 512, D_EROW = 640, D_BLK = 768, D_EEND = 784;
 enum {
-    B_XF = 0, B_XE = 3, B_BCF = 6, B_BCE = 8, B_DECF = 10, B_DECE = 14, B_CBF = 18, B_WF = 20, B_XSF = 22, B_DSF, B_DSE,
+    B_XF = 0, B_BCF = 3, B_DECF = 5, B_DECE = 9, B_CBF = 13, B_WF = 15, B_XSF = 17, B_DSF, B_DSE,
     B_SF, B_YF, B_YE, B_COUNT
 };
 constexpr size_t SMEM_BYTES = (size_t)OFF_BARS + B_COUNT * 8 + 32;
@@ -122,7 +124,12 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     uint32_t *tmem_slot = (uint32_t *)(bars + B_COUNT);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Role numbers (the `warp` used below) are decoupled from hardware warp numbers: when several warps of a
+    // scheduler are ready it favours the lower-numbered one, so the MMA issuer and the decay warp, which need
+    // few issue slots but need them promptly, take hardware warps 0 and 1 and the instruction-heavy W roles
+    // the highest numbers.  Roles that touch tensor memory keep role % 4 == hardware warp % 4 (lane quadrant).
+    const int hw_warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = hw_warp < 2 ? 13 - hw_warp : hw_warp < 4 ? hw_warp + 12 : hw_warp < 12 ? hw_warp : hw_warp - 12;
     const int h = blockIdx.x, b = blockIdx.y, g = h / (H / G);
     const int nchunks = (Tlen + Q - 1) / Q;
 
@@ -132,9 +139,9 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     }
     if (*(volatile int *)status != 0) return;         // an earlier CTA failed: leave at once
     if (threadIdx.x == 0) {
-        for (int i = 0; i < X_SLOTS; ++i) { tc::mbar_init(bars + B_XF + i, 1); tc::mbar_init(bars + B_XE + i, 9); }
+        for (int i = 0; i < X_SLOTS; ++i) tc::mbar_init(bars + B_XF + i, 1);
         for (int i = 0; i < 2; ++i) {
-            tc::mbar_init(bars + B_BCF + i, 1); tc::mbar_init(bars + B_BCE + i, 1);
+            tc::mbar_init(bars + B_BCF + i, 1);
             tc::mbar_init(bars + B_CBF + i, 1); tc::mbar_init(bars + B_WF + i, W_WARPS);
         }
         for (int i = 0; i < DEC_DEPTH; ++i) { tc::mbar_init(bars + B_DECF + i, 1); tc::mbar_init(bars + B_DECE + i, DEC_READERS); }
@@ -151,41 +158,16 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 12) {
-        // ------------------------------------------------------------------ TMA producer + decay vectors
+        // ------------------------------------------------------------------ decay vectors
         const float Ah2 = A[h] * LOG2E;
         const float *dtb = dt + (size_t)b * Tlen * H + h;
         bool ok = true;
-        int n_bc = 0, n_x = 0;
         float dv[4], dn[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) dn[i] = (4 * lane + i < Tlen) ? __ldg(dtb + (size_t)(4 * lane + i) * H) : 0.f;
 #pragma unroll 1
         for (int c = 0; c < nchunks; ++c) {
-            const int t0 = c * Q, s = c & 1, sx = c % X_SLOTS, d = c & (DEC_DEPTH - 1);
-            if (lane == 0) {
-                if (tc::mbar_wait(bars + B_BCE + s, ((c >> 1) & 1) ^ 1, abort_flag)) {
-                    SSD_TR(0, c, 0);
-                    uint64_t *fb = bars + B_BCF + s;
-                    tc::mbar_arrive_expect_tx(fb, 4 * TILE_16K);
-                    tc::tma_load_3d(smem + OFF_B + (s * 2) * TILE_16K, &tmap_b, fb, g * NS, t0, b);
-                    tc::tma_load_3d(smem + OFF_B + (s * 2 + 1) * TILE_16K, &tmap_b, fb, g * NS + 64, t0, b);
-                    tc::tma_load_3d(smem + OFF_C + (s * 2) * TILE_16K, &tmap_c, fb, g * NS, t0, b);
-                    tc::tma_load_3d(smem + OFF_C + (s * 2 + 1) * TILE_16K, &tmap_c, fb, g * NS + 64, t0, b);
-                    ++n_bc;
-                    if (tc::mbar_wait(bars + B_XE + sx, ((c / X_SLOTS) & 1) ^ 1, abort_flag)) {
-                        SSD_TR(0, c, 1);
-                        tc::mbar_arrive_expect_tx(bars + B_XF + sx, TILE_16K);
-                        tc::tma_load_3d(smem + OFF_X + sx * TILE_16K, &tmap_x, bars + B_XF + sx, h * P, t0, b);
-                        ++n_x;
-                    } else {
-                        ok = false;
-                    }
-                } else {
-                    ok = false;
-                }
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
+            const int d = c & (DEC_DEPTH - 1);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {             // this chunk's dt was fetched one iteration ago
                 dv[i] = dn[i];
@@ -205,6 +187,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (lane >= o) incl += v;
             }
             const float excl = incl - l[3];
+            SSD_TR(0, c, 4);
             const float l_start = __shfl_sync(0xffffffffu, excl, lane & ~7);     // start of this 32-token block
             const float l_endb = __shfl_sync(0xffffffffu, incl, lane | 7);       // end of this 32-token block
             const float l_end = __shfl_sync(0xffffffffu, incl, 31);
@@ -222,6 +205,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 o_rowf[i] = tc::ex2(li - l_start);
                 o_erow[i] = tc::ex2(li);
             }
+            SSD_TR(0, c, 5);
             *(float4 *)(dec + D_LS + 4 * lane) = make_float4(o_ls[0], o_ls[1], o_ls[2], o_ls[3]);
             *(float4 *)(dec + D_DT + 4 * lane) = make_float4(dv[0], dv[1], dv[2], dv[3]);
             *(float4 *)(dec + D_COLF + 4 * lane) = make_float4(o_colf[0], o_colf[1], o_colf[2], o_colf[3]);
@@ -230,20 +214,11 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             *(float4 *)(dec + D_EROW + 4 * lane) = make_float4(o_erow[0], o_erow[1], o_erow[2], o_erow[3]);
             if (lane < 16) dec[D_BLK + lane] = ((lane & 3) < (lane >> 2)) ? tc::ex2(bs - be) : 0.f;
             if (lane == 0) dec[D_EEND] = tc::ex2(l_end);
+            SSD_TR(0, c, 6);
             warp_arrive(bars + B_DECF + d, lane);
             SSD_TR(0, c, 3);
         }
-        if (!ok && lane == 0) {
-            atomicCAS(status, 0, STR_ERR_TIMEOUT);
-            for (int back = 1; back <= 2 && back <= n_bc; ++back) {      // let issued copies land
-                const int j = n_bc - back;
-                tc::mbar_wait(bars + B_BCF + (j & 1), (j >> 1) & 1, abort_flag + 1);
-            }
-            for (int back = 1; back <= X_SLOTS && back <= n_x; ++back) {
-                const int j = n_x - back;
-                tc::mbar_wait(bars + B_XF + j % X_SLOTS, (j / X_SLOTS) & 1, abort_flag + 1);
-            }
-        }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
     } else if (warp == 13) {
         // ------------------------------------------------------------------ MMA issuer
         // The whole warp runs the loop (so descriptors and addresses stay warp-uniform); one elected lane
@@ -283,8 +258,11 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             if (c >= 1) {
                 const int cp = c - 1, sp = cp & 1;
                 // the epilogue has read the Y accumulators of chunk c-2; W_{c-1} is in tensor memory
-                ok = (c < 2 || warp_wait(bars + B_YE, (c - 2) & 1, abort_flag)) &&
-                     warp_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag);
+                SSD_TR(7, c, 0);
+                ok = c < 2 || warp_wait(bars + B_YE, (c - 2) & 1, abort_flag);
+                SSD_TR(7, c, 1);
+                ok = ok && warp_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag);
+                SSD_TR(7, c, 2);
                 if (!ok) break;
                 SSD_TR(1, c, 3);
                 tc::tc_fence_after();
@@ -296,7 +274,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         tc::mma_ts(tmem + TM_YI, tW + (uint32_t)((ks >> 2) * 64 + (ks & 3) * 8), desc_add(dm_x, ks * 2048), id_kn,
                                    ks != 0);
                     tc::mma_commit(bars + B_YF);
-                    tc::mma_commit(bars + B_XE + cp % X_SLOTS);
                 }
                 __syncwarp();
                 SSD_TR(1, c, 4);
@@ -325,7 +302,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     for (int ks = 0; ks < 8; ++ks)      // dS_c^T = B^T Xs
                         tc::mma_ss(tmem + TM_DS, desc_add(dm_b, ks * 2048), desc_add(dm_xs, ks * 2048), id_nn, ks != 0);
                     tc::mma_commit(bars + B_DSF);
-                    tc::mma_commit(bars + B_BCE + s);
                 }
                 __syncwarp();
                 SSD_TR(1, c, 7);
@@ -420,9 +396,31 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             scale_x_half(smem + OFF_X + sx * TILE_16K, smem + OFF_XS, decs + d * DEC_FLOATS + D_XW, tid_s, 0);
             tc::fence_proxy_async();
             __syncwarp();
-            if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
+            if (lane == 0) tc::mbar_arrive(bars + B_XSF);
             return true;
         };
+        // Lane 0 of the first state warp is the TMA producer.  The operands of chunk c+2 go into the slots of chunk
+        // c (B, C: ring of 2) and chunk c-1 (X: ring of 3) once dS_c is seen complete: the tensor pipe runs in
+        // order, so CB_c, Y_inter_c, Y_intra_{c-1} and dS_{c-1} (issued after all of Xs_{c-1} was written, i.e.
+        // after every read of X_{c-1}) are complete too.  No slot-release barriers are needed.
+        const bool loader = warp == 4 && lane == 0;
+        int n_loaded = 0;
+        auto load_chunk = [&](int c) {
+            const int t0 = c * Q, s = c & 1, sx = c % X_SLOTS;
+            uint64_t *fb = bars + B_BCF + s;
+            tc::mbar_arrive_expect_tx(fb, 4 * TILE_16K);
+            tc::tma_load_3d(smem + OFF_B + (s * 2) * TILE_16K, &tmap_b, fb, g * NS, t0, b);
+            tc::tma_load_3d(smem + OFF_B + (s * 2 + 1) * TILE_16K, &tmap_b, fb, g * NS + 64, t0, b);
+            tc::tma_load_3d(smem + OFF_C + (s * 2) * TILE_16K, &tmap_c, fb, g * NS, t0, b);
+            tc::tma_load_3d(smem + OFF_C + (s * 2 + 1) * TILE_16K, &tmap_c, fb, g * NS + 64, t0, b);
+            tc::mbar_arrive_expect_tx(bars + B_XF + sx, TILE_16K);
+            tc::tma_load_3d(smem + OFF_X + sx * TILE_16K, &tmap_x, bars + B_XF + sx, h * P, t0, b);
+            ++n_loaded;
+        };
+        if (loader) {
+            load_chunk(0);
+            if (nchunks > 1) load_chunk(1);
+        }
         ok = xs_half(0);
 #pragma unroll 1
         for (int c = 0; c < nchunks && ok; ++c) {
@@ -459,11 +457,19 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             }
             tc::fence_proxy_async();
             warp_arrive(bars + B_SF, lane);
+            if (loader && c + 2 < nchunks) load_chunk(c + 2);
             if (quad == SSD_TRQ) SSD_TR(5, c, 2);
             if (c + 1 < nchunks && !xs_half(c + 1)) { ok = false; break; }
             if (quad == SSD_TRQ) SSD_TR(5, c, 3);
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+        if (!ok && loader) {                          // let copies already issued land before the CTA goes away
+            for (int back = 1; back <= 2 && back <= n_loaded; ++back) {
+                const int j = n_loaded - back;
+                tc::mbar_wait(bars + B_BCF + (j & 1), (j >> 1) & 1, abort_flag + 1);
+                tc::mbar_wait(bars + B_XF + j % X_SLOTS, (j / X_SLOTS) & 1, abort_flag + 1);
+            }
+        }
         if (ok && final_state) {
             float *fs = final_state + ((size_t)b * H + h) * P * NS;
 #pragma unroll
@@ -490,7 +496,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 scale_x_half(smem + OFF_X + sx * TILE_16K, smem + OFF_XS, dec + D_XW, tid_g, 1);
                 tc::fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) { tc::mbar_arrive(bars + B_XSF); tc::mbar_arrive(bars + B_XE + sx); }
+                if (lane == 0) tc::mbar_arrive(bars + B_XSF);
                 if (quad == SSD_TRQ) SSD_TR(6, c, 2);
             }
             if (c >= 1) {
