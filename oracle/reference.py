@@ -193,6 +193,31 @@ def mamba_importance(B, C, dt, n_vis, n_text):
     return s / (n_text * G)
 
 
+def mamba_importance_full_dynamic(B, C, dt, A, n_vis, n_text):
+    """The "Full Mamba Dynamic" score (Section 3.1, "Why the Full Mamba Dynamic Fails"): |w_{t,i}| of Eq. 1,
+    i.e. content alignment times the cumulative decay between visual token i and text position t,
+
+        s_i = 1/(M H) sum_{m,h} | (prod_{u=i+1..t_m} Abar_u^(h)) (Delta_i^(h) b_i^(g(h)))^T c_{t_m}^(g(h)) |,
+
+    t_m = n_vis + m the m-th text row.  The paper names the per-pair quantity |w_{t,j}| and does not spell
+    out the aggregation; the mean over the M text positions and the H heads is taken by analogy with Eq. 2
+    (the decay is per head, so heads replace groups).  The decay product is written as the exponential of
+    a difference of cumulative sums of Delta_u A_h.  B,C [T,G,n], dt [T,H], A [H] (< 0).  Returns s [n_vis].
+    """
+    B, C, dt, A = _f64(B), _f64(C), _f64(dt), _f64(A)
+    T, G, n = B.shape
+    H = dt.shape[1]
+    assert n_vis + n_text == T and H % G == 0
+    L = np.cumsum(dt * A[None, :], axis=0)                        # [T, H]: log of prod_{u<=t} Abar_u
+    s = np.zeros(n_vis)
+    for h in range(H):
+        g = h // (H // G)
+        align = (dt[:n_vis, h, None] * B[:n_vis, g, :]) @ C[n_vis:, g, :].T      # [n_vis, M]
+        decay = np.exp(L[None, n_vis:, h] - L[:n_vis, None, h])                  # [n_vis, M], all exponents <= 0
+        s += np.abs(decay * align).sum(axis=1)
+    return s / (n_text * H)
+
+
 def attn_importance(q, k, n_vis, n_text, scale):
     """s_i = 1/(M Hq) sum_{m,h} softmax_i( q_m^(h) . k_i^(kv(h)) * scale ), text -> visual.
 

@@ -109,3 +109,68 @@ def test_attn_score_peaks_on_the_aligned_key():
     q[3, 0, 0] = 40.0
     s = oracle.attn_importance(q, k, 3, 1, 1.0)
     assert s.argmax() == 1 and s[1] > 0.999999
+
+
+# ---- "Full Mamba Dynamic" score: |w_{t,i}| of Eq. 1, averaged over text positions and heads ----
+
+def _ssm_dyn(seed, n_vis, M, H, G, n):
+    B, C, dt = _ssm(seed, n_vis, M, H, G, n)
+    A = -np.exp(np.random.default_rng(seed + 100).uniform(0.0, np.log(16.0), size=H))
+    return B, C, dt, A
+
+
+def test_full_dynamic_score_equals_unrolled_weights_of_eq1():
+    # the pure-loop Eq. 1 weights (product of Abar written out factor by factor) of every head
+    n_vis, M, H, G, n = 6, 3, 4, 2, 5
+    B, C, dt, A = _ssm_dyn(20, n_vis, M, H, G, n)
+    s = oracle.mamba_importance_full_dynamic(B, C, dt, A, n_vis, M)
+    ref = np.zeros(n_vis)
+    for h in range(H):
+        w = oracle.mamba2_unrolled_weights(dt, A, B, C, h)          # [T, T], rows = output positions
+        ref += np.abs(w[n_vis:, :n_vis]).sum(axis=0)
+    np.testing.assert_allclose(s, ref / (M * H), rtol=1e-12)
+
+
+def test_full_dynamic_score_is_the_response_of_the_recurrence_to_one_token():
+    # w_{t,i} is what token i contributes to y_t: feed the sequential recurrence (the C loop) a one-hot x
+    n_vis, M, H, G, n = 5, 2, 4, 2, 3
+    B, C, dt, A = _ssm_dyn(21, n_vis, M, H, G, n)
+    s = oracle.mamba_importance_full_dynamic(B, C, dt, A, n_vis, M)
+    ref = np.zeros(n_vis)
+    for i in range(n_vis):
+        x = np.zeros((n_vis + M, H, 1))
+        x[i] = 1.0
+        y, _ = oracle.mamba2_recurrence(x, dt, A, B, C)
+        ref[i] = np.abs(y[n_vis:, :, 0]).sum()
+    np.testing.assert_allclose(s, ref / (M * H), rtol=1e-11)
+
+
+def test_full_dynamic_score_without_decay_is_eq2():
+    # A = 0 makes every Abar one: what is left is the content alignment, i.e. Eq. 2 (per-head form = group form)
+    n_vis, M, H, G, n = 11, 4, 6, 3, 4
+    B, C, dt, _ = _ssm_dyn(22, n_vis, M, H, G, n)
+    s = oracle.mamba_importance_full_dynamic(B, C, dt, np.zeros(H), n_vis, M)
+    np.testing.assert_allclose(s, oracle.mamba_importance(B, C, dt, n_vis, M), rtol=1e-12)
+
+
+def test_full_dynamic_score_closed_form_constant_decay():
+    # one head, one text row, dt = const: decay between token i and the text row is exp(A dt (n_vis - i))
+    n_vis, n = 8, 3
+    r = np.random.default_rng(23)
+    B, C = r.normal(size=(n_vis + 1, 1, n)), r.normal(size=(n_vis + 1, 1, n))
+    dt, A = np.full((n_vis + 1, 1), 0.25), np.array([-2.0])
+    s = oracle.mamba_importance_full_dynamic(B, C, dt, A, n_vis, 1)
+    i = np.arange(n_vis)
+    ref = np.exp(-0.5 * (n_vis - i)) * 0.25 * np.abs(B[:n_vis, 0] @ C[n_vis, 0])
+    np.testing.assert_allclose(s, ref, rtol=1e-13)
+
+
+def test_full_dynamic_score_suppresses_early_tokens():
+    # the paper's failure mode: with equal content alignment the score decays monotonically with distance
+    n_vis, M, H = 40, 2, 2
+    B = np.ones((n_vis + M, 1, 4)); C = np.ones((n_vis + M, 1, 4))
+    dt = np.full((n_vis + M, H), 0.05); A = np.array([-1.0, -8.0])
+    s = oracle.mamba_importance_full_dynamic(B, C, dt, A, n_vis, M)
+    assert np.all(np.diff(s) > 0) and s[0] < 0.2 * s[-1]
+    flat = oracle.mamba_importance(B, C, dt, n_vis, M)
+    np.testing.assert_allclose(flat, flat[0], rtol=1e-13)            # Eq. 2 does not see position at all
