@@ -396,6 +396,17 @@ def run_micro(args):
         fn = lambda: binding.str_mamba_importance(ctx, Bm, Cm, dt, n_vis, M)
         flops = Bz * n_vis * 2.0 * M * n * G
         nbytes = Bz * n_vis * (2 * G * n + 4 * H + 4)
+    elif name == "mamba_dyn_score":
+        # Full Mamba Dynamic (Eq. 1 weights): reads B of the visual rows and dt of every row, writes and re-reads
+        # the bf16 high/low decay weights (64 columns per group), two products per tile
+        H, n, G = ms_["H"], ms_["n"], ms_["G"]
+        Bm = torch.randn(Bz, T, G, n, device=dev).to(bf)
+        Cm = torch.randn(Bz, T, G, n, device=dev).to(bf)
+        dt = torch.empty(Bz, T, H, device=dev).uniform_(1e-3, 1e-1)
+        A = -torch.exp(torch.empty(H, device=dev).uniform_(0.0, float(np.log(16.0))))
+        fn = lambda: binding.str_mamba_importance_dynamic(ctx, Bm, Cm, dt, A, n_vis, M)
+        flops = Bz * n_vis * 2.0 * M * (n + 3 * H // G) * G
+        nbytes = Bz * n_vis * (2 * G * n + 2 * 4 * H + 2 * 2 * G * 64 + 4)
     elif name == "attn_score":
         Hq, Hkv, d = at_["Hq"], at_["Hkv"], at_["d"]
         q = torch.randn(Bz, T, Hq, d, device=dev).to(bf)
@@ -477,7 +488,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--schedule", default="step", choices=["step", "sigmoid"], help="retention schedule of the stack")
     ap.add_argument("--x0", type=float, default=0.11, help="midpoint of the sigmoid schedule (0.11 / 0.24 / 0.41)")
-    ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | attn_score | attn_fwd | "
+    ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | mamba_dyn_score | attn_score | attn_fwd | "
                                                 "topk | compact | gemm")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

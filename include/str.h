@@ -85,6 +85,19 @@ int str_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, 
                          const void *B, const void *C, const float *dt, float *scores_out,
                          void *workspace, size_t workspace_bytes, void *stream);
 
+/* (2a', score variant)  "Full Mamba Dynamic", Section 3.1 (the paragraph on why it fails) and Eq. 1: the
+ * magnitude of the exact weight w_{t,i} with which visual token i enters the output at text position t,
+ *   s_i = 1/(M H) sum_{m,h} | (prod_{u=i+1..t_m} Abar_u^(h)) (dt[i,h] b_i^(g(h)))^T c_{t_m}^(g(h)) |,
+ * Abar_u^(h) = exp(dt[u,h] A[h]), t_m = n_vis + m.  The paper uses it as the ablation against Eq. 2 (its
+ * scoring-ablation table); the mean over text positions and heads is this library's reading.
+ *   B, C device [Bz,T,G,n] dtype; dt device [Bz,T,H] fp32 (post-softplus); A device [H] fp32 (< 0);
+ *   scores_out device [Bz,n_vis] fp32 (tokens far from the text underflow to 0: that is the score's nature).
+ * Workspace (caller-owned, size from the query) holds the per-token decay weights.  Errors as (2a). */
+size_t str_mamba_importance_dynamic_workspace_size(const str_ssm_score_shape *s, int n_vis, int n_text);
+int str_mamba_importance_dynamic(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text,
+                                 const void *B, const void *C, const float *dt, const float *A,
+                                 float *scores_out, void *workspace, size_t workspace_bytes, void *stream);
+
 /* (2b) Attention importance, Section 3.1 "Attention Layers":
  *   s_i = 1/(M Hq) sum_{m,h} softmax_i( q_m^(h) . k_i^(kv(h)) * softmax_scale ),
  * softmax over the n_vis visual keys, m over the last n_text query rows, kv(h) = h/(Hq/Hkv).

@@ -59,6 +59,7 @@ EXPORTS = [
     "str_profile_enable", "str_profile_collect",
     "str_mamba2_prefill_workspace_size", "str_mamba2_prefill",
     "str_mamba_importance_workspace_size", "str_mamba_importance",
+    "str_mamba_importance_dynamic_workspace_size", "str_mamba_importance_dynamic",
     "str_attn_importance_workspace_size", "str_attn_importance", "str_attn_importance_static",
     "str_topk_select_workspace_size", "str_topk_select", "str_compact",
     "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
@@ -188,6 +189,19 @@ def str_mamba_importance(ctx, B, C, dt, n_vis, n_text):
     ws = ctx.workspace(nb)
     _check(lib().str_mamba_importance(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(B), _p(C), _p(dt),
                                       _p(out), _p(ws), c_size_t(ws.numel()), _stream()), "str_mamba_importance")
+    return out
+
+
+def str_mamba_importance_dynamic(ctx, B, C, dt, A, n_vis, n_text):
+    Bz, T, G, n = B.shape
+    H = dt.shape[2]
+    s = SsmScoreShape(Bz, T, H, n, G, _dt(B))
+    out = torch.empty((Bz, n_vis), dtype=torch.float32, device=B.device)
+    nb = lib().str_mamba_importance_dynamic_workspace_size(ctypes.byref(s), c_int(n_vis), c_int(n_text))
+    ws = ctx.workspace(nb)
+    _check(lib().str_mamba_importance_dynamic(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(B), _p(C),
+                                              _p(dt), _p(A), _p(out), _p(ws), c_size_t(ws.numel()), _stream()),
+           "str_mamba_importance_dynamic")
     return out
 
 

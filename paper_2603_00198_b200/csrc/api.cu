@@ -58,6 +58,46 @@ extern "C" int str_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, 
     return str_mamba_importance_simt(ctx, s, n_vis, n_text, B, C, dt, scores_out, (cudaStream_t)stream);
 }
 
+// ---------------------------------------------------------------- (2a') Mamba importance with the cumulative decay
+// Workspace: chunk sums of dt A | U | V, where U, V are the decay weights in whichever layout is the larger.
+static size_t dyn_uv_bytes(const str_ssm_score_shape *s, int n_vis, int n_text, bool split, size_t *u_bytes) {
+    const size_t n_pad = (size_t)(n_text + 15) / 16 * 16;
+    const size_t ub = split ? (size_t)s->Bz * n_vis * s->G * 64 * 2 : (size_t)s->Bz * n_vis * s->H * 4;
+    const size_t vb = split ? (size_t)s->Bz * n_pad * s->G * 64 * 2 : (size_t)s->Bz * n_text * s->H * 4;
+    if (u_bytes) *u_bytes = align_up(ub, 256);
+    return align_up(ub, 256) + align_up(vb, 256);
+}
+
+extern "C" size_t str_mamba_importance_dynamic_workspace_size(const str_ssm_score_shape *s, int n_vis, int n_text) {
+    if (!s || s->Bz <= 0 || s->H <= 0 || s->G <= 0 || n_vis <= 0 || n_text <= 0) return 0;
+    const size_t a = dyn_uv_bytes(s, n_vis, n_text, false, nullptr), b = dyn_uv_bytes(s, n_vis, n_text, true, nullptr);
+    return str_mamba_dyn_part_bytes(s, n_vis) + (a > b ? a : b);
+}
+
+extern "C" int str_mamba_importance_dynamic(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text,
+                                            const void *B, const void *C, const float *dt, const float *A,
+                                            float *scores_out, void *workspace, size_t workspace_bytes, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_MAMBA_SCORE, stream);
+    if (!ctx || !s || !B || !C || !dt || !A) return STR_ERR_INVALID_ARG;
+    if (s->Bz <= 0 || s->H <= 0 || s->n <= 0 || s->G <= 0 || s->H % s->G != 0 || n_vis < 0 || n_text <= 0 ||
+        n_vis + n_text != s->T || !STR_DTYPE_OK(s->dtype))
+        return STR_ERR_INVALID_ARG;
+    if (n_vis == 0) return STR_OK;
+    if (!scores_out || !workspace) return STR_ERR_INVALID_ARG;
+    if (workspace_bytes < str_mamba_importance_dynamic_workspace_size(s, n_vis, n_text)) return STR_ERR_WORKSPACE_TOO_SMALL;
+    const bool tc = !str_force_simt() && ctx->encode_tiled && str_mamba_dyn_importance_tc_supported(s, n_vis, n_text, B, C);
+    const int n_pad = (n_text + 15) / 16 * 16;
+    float *part = (float *)workspace;
+    size_t u_bytes = 0;
+    dyn_uv_bytes(s, n_vis, n_text, tc, &u_bytes);
+    uint8_t *U = (uint8_t *)workspace + str_mamba_dyn_part_bytes(s, n_vis), *V = U + u_bytes;
+    int rc = str_mamba_dyn_weights(ctx, s, n_vis, n_text, n_pad, dt, A, part, U, V, tc, (cudaStream_t)stream);
+    if (rc != STR_OK) return rc;
+    if (tc) return str_mamba_dyn_importance_tc(ctx, s, n_vis, n_text, B, C, U, V, scores_out, (cudaStream_t)stream);
+    return str_mamba_dyn_importance_simt(ctx, s, n_vis, n_text, B, C, (const float *)U, (const float *)V, scores_out,
+                                         (cudaStream_t)stream);
+}
+
 // ---------------------------------------------------------------- (2b) attention importance
 extern "C" size_t str_attn_importance_workspace_size(const str_attn_score_shape *s, int n_vis, int n_text) {
     (void)n_vis;

@@ -58,7 +58,8 @@ static inline int str_launch_ok(str_ctx *ctx, int n = 1) {
 
 // Opt a kernel into `bytes` of dynamic shared memory once per context (the attribute belongs to the device the
 // context was created on, so it is tracked per context, not per process).
-enum { STR_SMEM_GEMM = 0, STR_SMEM_SSD, STR_SMEM_ATTN_FWD, STR_SMEM_MAMBA_SCORE, STR_SMEM_ATTN_ROWSTATS, STR_SMEM_ATTN_COLSUM };
+enum { STR_SMEM_GEMM = 0, STR_SMEM_SSD, STR_SMEM_ATTN_FWD, STR_SMEM_MAMBA_SCORE, STR_SMEM_ATTN_ROWSTATS, STR_SMEM_ATTN_COLSUM,
+       STR_SMEM_MAMBA_DYN_SCORE };
 template <typename F>
 static inline int str_ensure_smem(str_ctx *ctx, int slot, F kernel, size_t bytes) {
     // The attribute belongs to the device's copy of the kernel, not to this context: every context raises it to

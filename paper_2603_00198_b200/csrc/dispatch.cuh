@@ -30,6 +30,15 @@ int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, const void *q, co
 bool str_mamba_importance_tc_supported(const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C);
 int str_mamba_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C,
                             const float *dt, float *scores, cudaStream_t st);
+// "Full Mamba Dynamic" score: decay-weight pass (fp32 or bf16 high/low layout), then one of the two scoring kernels.
+size_t str_mamba_dyn_part_bytes(const str_ssm_score_shape *s, int n_vis);
+int str_mamba_dyn_weights(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, int n_pad, const float *dt,
+                          const float *A, float *part, void *U, void *V, bool split, cudaStream_t st);
+int str_mamba_dyn_importance_simt(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, const void *B,
+                                  const void *C, const float *U, const float *V, float *scores, cudaStream_t st);
+bool str_mamba_dyn_importance_tc_supported(const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C);
+int str_mamba_dyn_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C,
+                                const void *U, const void *V, float *scores, cudaStream_t st);
 // Key segments the tensor-core attention score may split its first pass into (sizes the workspace).
 #define STR_ATTN_SCORE_MAX_SEGMENTS 8
 bool str_attn_importance_tc_supported(const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k);

@@ -1,4 +1,4 @@
-"""GPU parity: importance scores (attention-layer score and Eq. 2) against the oracle, and the
+"""GPU parity: importance scores (attention-layer score, Eq. 2 and the Eq. 1 variant) against the oracle, and the
 score -> select pipeline with the swap tolerance."""
 import numpy as np
 import pytest
@@ -47,6 +47,57 @@ def test_mamba_importance_matches_eq2(ctx, dtype, n_vis, M, H, n, G, Bz):
         assert score_rel_err(got[b], ref) <= SCORE_TOL
         kept = binding.str_topk_select(ctx, dev(got[b:b + 1]), k).cpu().numpy()[0]
         assert_kept_matches(kept, oracle.topk_select(ref, k), ref)
+
+
+DYN_CASES = [
+    # dtype, n_vis, M, H, n, G, Bz
+    ("f32", 1024, 32, 8, 16, 1, 1),          # config 0 shape (plain fp32 kernel)
+    ("bf16", 4096, 128, 128, 128, 8, 1),     # config 1 shape: tensor cores, 16 heads per group
+    ("bf16", 1000, 100, 16, 128, 4, 2),      # padded text rows, ragged token tiles, 4 heads per group, batch
+    ("bf16", 300, 1, 8, 128, 8, 1),          # one text row, one head per group
+    ("bf16", 777, 200, 32, 128, 2, 1),       # more than 128 text rows: plain kernel
+    ("bf16", 1, 16, 4, 128, 1, 3),
+    ("bf16", 70, 3, 4, 32, 2, 1),            # d_state the tensor-core kernel does not tile
+    ("bf16", 2500, 64, 42, 128, 2, 1),       # 21 heads per group: 63 of the 64 decay columns in use
+]
+
+
+def _dyn_err(got, ref):
+    """Relative error where the oracle's score is within fp32's reach of the largest one; beyond that the
+    cumulative decay underflows in fp32 (the oracle, in fp64, still holds 1e-40 and smaller) and the GPU
+    value only has to be as negligible."""
+    floor = 1e-30 * ref.max()
+    big = ref >= floor
+    assert np.all(got[~big] <= 2 * floor)
+    return score_rel_err(got[big], ref[big]), int(big.sum())
+
+
+@pytest.mark.parametrize("dtype,n_vis,M,H,n,G,Bz", DYN_CASES)
+def test_mamba_full_dynamic_score_matches_eq1(ctx, dtype, n_vis, M, H, n, G, Bz):
+    T = n_vis + M
+    d = inputs.ssd_inputs(33, T, H, 16, n, G, dtype, batch=Bz)
+    got = binding.str_mamba_importance_dynamic(ctx, dev(d["B"], dtype), dev(d["C"], dtype), dev(d["dt"]), dev(d["A"]),
+                                               n_vis, M).cpu().numpy()
+    ctx.check_status()
+    for b in range(Bz):
+        ref = oracle.mamba_importance_full_dynamic(d["B"][b], d["C"][b], d["dt"][b], d["A"], n_vis, M)
+        err, n_big = _dyn_err(got[b], ref)
+        assert err <= SCORE_TOL
+        assert np.all(got[b] >= 0) and np.all(np.isfinite(got[b]))
+        # selection on this score, with a budget that stays above the underflow floor
+        k = max(1, min(n_vis // 4, n_big // 2))
+        kept = binding.str_topk_select(ctx, dev(got[b:b + 1]), k).cpu().numpy()[0]
+        assert_kept_matches(kept, oracle.topk_select(ref, k), ref)
+
+
+def test_mamba_full_dynamic_score_without_decay_is_eq2(ctx):
+    # A = 0: every Abar is one and the score must fall back to the content alignment of Eq. 2
+    n_vis, M, H, n, G = 1500, 96, 32, 128, 4
+    d = inputs.ssd_inputs(34, n_vis + M, H, 16, n, G, "bf16")
+    B, C, dt = dev(d["B"], "bf16"), dev(d["C"], "bf16"), dev(d["dt"])
+    dyn = binding.str_mamba_importance_dynamic(ctx, B, C, dt, dev(np.zeros(H, dtype=np.float32)), n_vis, M).cpu().numpy()[0]
+    eq2 = binding.str_mamba_importance(ctx, B, C, dt, n_vis, M).cpu().numpy()[0]
+    assert score_rel_err(dyn, eq2) <= 1e-4
 
 
 ATTN_CASES = [
