@@ -239,7 +239,7 @@ def run_ours(args):
     ctx = binding.Context(local)
     # weights: seeded on the host, one replica per rank (the path does not shard: replicas only)
     layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], "f32")
-    stack = binding.Stack(ctx, layers, cfg["dtype"], Bz, n_vis, M, K, Q=cfg["mamba"]["Q"])
+    stack = binding.Stack(ctx, layers, cfg["dtype"], Bz, n_vis, M, K, Q=cfg["mamba"]["Q"], mamba_score=args.mamba_score)
     del layers
     h_host = torch.from_numpy(inputs.hidden_inputs(cfg["seed"] + 1000 * rank, T0, D, "bf16", batch=Bz)).to(torch.bfloat16)
     h_pin = h_host.pin_memory()
@@ -345,7 +345,7 @@ def run_ours(args):
         "config": {"workload": "C3 12-layer hybrid stack [M,M,M,M,M,A]x2, %d visual + %d text tokens, batch %d, "
                                "schedule %s" % (n_vis, M, Bz, "/".join(str(a // 100) for a in (cfg["alpha_bp"][::4] if args.schedule == "step"
                                                                                   else cfg["alpha_bp"]))),
-                   "keep_counts": K, "l2": "inputs larger than L2 (hidden %d MB, workspace %d MB)"
+                   "mamba_score": args.mamba_score, "keep_counts": K, "l2": "inputs larger than L2 (hidden %d MB, workspace %d MB)"
                                            % (h_dev.numel() * 2 >> 20, stack.ws_bytes >> 20),
                    "multi_gpu": "replicas only (the path does not shard)"},
         "roofline": roof, "cpu_baseline": cpu,
@@ -487,6 +487,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the CPU oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--schedule", default="step", choices=["step", "sigmoid"], help="retention schedule of the stack")
+    ap.add_argument("--mamba-score", default="decoupled", choices=["decoupled", "full_dynamic"],
+                    help="Mamba-layer importance: Eq. 2 (the method) or |w| of Eq. 1 (the paper's scoring ablation)")
     ap.add_argument("--x0", type=float, default=0.11, help="midpoint of the sigmoid schedule (0.11 / 0.24 / 0.41)")
     ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | mamba_dyn_score | attn_score | attn_fwd | "
                                                 "topk | compact | gemm")

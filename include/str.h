@@ -219,6 +219,7 @@ int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const void *q, const
  * smaller than the incoming count.  Block wrapper: h <- h + Mixer(RMSNorm(h)).
  * ------------------------------------------------------------------------------------------ */
 enum { STR_LAYER_MAMBA = 0, STR_LAYER_ATTN = 1 };
+enum { STR_SCORE_DECOUPLED = 0, STR_SCORE_FULL_DYNAMIC = 1 };
 typedef struct {
     int kind;             /* STR_LAYER_MAMBA or STR_LAYER_ATTN                                  */
     const void *w_in;     /* device: Mamba in_proj [2*d_inner+2Gn+H, D] | attention W_qkv [(Hq+2Hkv)d, D] */
@@ -237,6 +238,7 @@ typedef struct {
     const str_layer *layers;           /* host array [n_layers]                              */
     const int *keep_counts;            /* host array [n_layers], from str_schedule_keep_counts */
     int score_every_layer;             /* nonzero: also compute (not apply) the score at layers that do not reduce */
+    int mamba_score_kind;              /* STR_SCORE_DECOUPLED (Eq. 2, the method) or STR_SCORE_FULL_DYNAMIC (Eq. 1, its ablation) */
 } str_stack_desc;
 size_t str_stack_workspace_size(const str_stack_desc *d);
 /* hidden_in device [Bz, n_vis+n_text, D] dtype.  Outputs (device): hidden_out

@@ -428,14 +428,16 @@ def attn_block(u, positions, prm, rnd=_identity):
     return out, dict(q=q, k=k, v=v, o=o, scale=scale)
 
 
-def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity):
+def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_score="decoupled"):
     """Token-reduced prefill of a layer stack (one sequence).
 
     hidden [T0,D] with the n_text text rows last; layers: list of ("M"|"A", prm);
     keep_counts[l] = visual tokens kept after layer l.  Layer l's mixer runs on the incoming
     tokens, its own score ranks the incoming visual tokens, and its OUTPUT is compacted when
     keep_counts[l] < n_cur.  Returns (hidden, positions, idx_map, trace) where trace lists per
-    layer dict(n_in, scores or None, kept or None)."""
+    layer dict(n_in, scores or None, kept or None).  ``mamba_score``: "decoupled" (Eq. 2, the method) or
+    "full_dynamic" (|w| of Eq. 1, the paper's scoring ablation)."""
+    assert mamba_score in ("decoupled", "full_dynamic")
     h = _f64(hidden)
     T0 = h.shape[0]
     n_cur = T0 - n_text
@@ -445,7 +447,10 @@ def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity):
     for (kind, prm), K in zip(layers, keep_counts):
         if kind == "M":
             out, mid = mamba2_block(h, prm, rnd)
-            score = (lambda: mamba_importance(mid["B"], mid["C"], mid["dt"], n_cur, n_text))
+            if mamba_score == "full_dynamic":
+                score = (lambda: mamba_importance_full_dynamic(mid["B"], mid["C"], mid["dt"], prm["A"], n_cur, n_text))
+            else:
+                score = (lambda: mamba_importance(mid["B"], mid["C"], mid["dt"], n_cur, n_text))
         else:
             out, mid = attn_block(h, pos, prm, rnd)
             score = (lambda: attn_importance(mid["q"], mid["k"], n_cur, n_text, mid["scale"]))

@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(_PKG, "libstr.so")
 
 STR_F32, STR_BF16 = 0, 1
 STR_LAYER_MAMBA, STR_LAYER_ATTN = 0, 1
+STR_SCORE_DECOUPLED, STR_SCORE_FULL_DYNAMIC = 0, 1
 c_int, c_float, c_size_t, c_void_p = ctypes.c_int, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
 
 
@@ -49,7 +50,7 @@ class StackDesc(ctypes.Structure):
                                       "conv_width", "Hq", "Hkv", "d")]
                 + [("rope_theta", c_float), ("norm_eps", c_float), ("n_layers", c_int),
                    ("layers", ctypes.POINTER(Layer)), ("keep_counts", ctypes.POINTER(c_int)),
-                   ("score_every_layer", c_int)])
+                   ("score_every_layer", c_int), ("mamba_score_kind", c_int)])
 
 
 PROF_CATEGORIES = ["gemm", "ssd_scan", "mamba_score", "attn_score", "topk", "compact", "attn_fwd", "elementwise"]
@@ -345,7 +346,7 @@ class Stack:
     [out_features, in_features] layout."""
 
     def __init__(self, ctx, layers, dtype, Bz, n_vis, n_text, keep_counts, Q=0, score_every_layer=False,
-                 rope_theta=1.0e6, norm_eps=1e-5):
+                 rope_theta=1.0e6, norm_eps=1e-5, mamba_score="decoupled"):
         self.ctx = ctx
         tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
         dev = "cuda:%d" % ctx.device
@@ -377,7 +378,8 @@ class Stack:
                               ms["H"], ms["p"], ms["n"], ms["G"], Q, 4 if m_shape else 0,
                               as_["Hq"], as_["Hkv"], as_["d"], rope_theta, norm_eps, len(layers),
                               ctypes.cast(arr, ctypes.POINTER(Layer)), ctypes.cast(self._kc, ctypes.POINTER(c_int)),
-                              1 if score_every_layer else 0)
+                              1 if score_every_layer else 0,
+                              {"decoupled": STR_SCORE_DECOUPLED, "full_dynamic": STR_SCORE_FULL_DYNAMIC}[mamba_score])
         self.tdt, self.dev = tdt, dev
         self.Bz, self.n_vis, self.n_text, self.D = Bz, n_vis, n_text, D
         self.keep_counts = [int(k) for k in keep_counts]

@@ -22,7 +22,8 @@ inline size_t imax(size_t a, size_t b) { return a > b ? a : b; }
 
 bool desc_ok(const str_stack_desc *d) {
     if (!d || d->Bz <= 0 || d->n_vis < 0 || d->n_text <= 0 || d->D <= 0 || d->n_layers <= 0 || !d->layers ||
-        !d->keep_counts || (d->dtype != STR_F32 && d->dtype != STR_BF16))
+        !d->keep_counts || (d->dtype != STR_F32 && d->dtype != STR_BF16) ||
+        (d->mamba_score_kind != STR_SCORE_DECOUPLED && d->mamba_score_kind != STR_SCORE_FULL_DYNAMIC))
         return false;
     bool has_m = false, has_a = false;
     int n_cur = d->n_vis;
@@ -77,6 +78,8 @@ Regions plan(const str_stack_desc *d) {
         sub = imax(sub, str_mamba2_prefill_workspace_size(&s));
         str_ssm_score_shape ss = {d->Bz, (int)T0, d->H, d->n, d->G, d->dtype};
         sub = imax(sub, str_mamba_importance_workspace_size(&ss, d->n_vis, d->n_text));
+        if (d->mamba_score_kind == STR_SCORE_FULL_DYNAMIC)
+            sub = imax(sub, str_mamba_importance_dynamic_workspace_size(&ss, d->n_vis, d->n_text));
         sub = imax(sub, str_gemm_workspace_size((int)R, (int)dip, d->D, d->dtype));
     }
     if (has_a) {
@@ -165,7 +168,10 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
                                        r.sub_bytes, stream));
             if (want_score && n_cur > 0) {
                 str_ssm_score_shape ss = {Bz, T, d->H, d->n, d->G, dtype};
-                STR_TRY(str_mamba_importance(ctx, &ss, n_cur, M, bufB, bufC, dt, scores, sub, r.sub_bytes, stream));
+                if (d->mamba_score_kind == STR_SCORE_FULL_DYNAMIC)
+                    STR_TRY(str_mamba_importance_dynamic(ctx, &ss, n_cur, M, bufB, bufC, dt, L.A, scores, sub, r.sub_bytes, stream));
+                else
+                    STR_TRY(str_mamba_importance(ctx, &ss, n_cur, M, bufB, bufC, dt, scores, sub, r.sub_bytes, stream));
             }
             if (reduce) {
                 STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));

@@ -147,3 +147,35 @@ def test_all_layer_sigmoid_schedule(ctx):
     # bulk of the surviving rows is compared, loosely
     row_err = np.abs(host(out)[0][a] - ref[c]).max(axis=1) / np.abs(ref).max()
     assert np.median(row_err) <= 5e-2
+
+
+MS_TC = dict(D=512, H=8, p=64, n=128, G=2, Q=128, conv=4)      # shapes the tensor-core kernels tile
+
+
+@pytest.mark.parametrize("dtype,shape", [("f32", MS), ("bf16", MS), ("bf16", MS_TC)])
+def test_single_mamba_layer_reduced_by_the_full_dynamic_score(ctx, dtype, shape):
+    """The scoring ablation inside the stack: selection by |w| of Eq. 1 instead of Eq. 2.  The budget is set
+    from the oracle's scores so that the selection threshold stays above fp32's underflow of the decay."""
+    n_vis, M = 600, 24
+    layers = inputs.stack_params(66, "M", shape, shape, dtype)
+    h0 = inputs.hidden_inputs(66, n_vis + M, shape["D"], dtype)
+    _, _, _, probe = oracle.stack_prefill(h0[0], M, layers, [n_vis // 4], _rnd(dtype), mamba_score="full_dynamic")
+    s_probe = probe[0]["scores"]
+    K = [int(max(8, min(n_vis // 4, (s_probe >= 1e-20 * s_probe.max()).sum() // 2)))]
+    ref, rpos, ridx, trace = oracle.stack_prefill(h0[0], M, layers, K, _rnd(dtype), mamba_score="full_dynamic")
+    st = binding.Stack(ctx, layers, dtype, 1, n_vis, M, K, Q=shape.get("Q", 0), mamba_score="full_dynamic")
+    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, dtype), want_trace=True)
+    ctx.check_status()
+    s_gpu, s_ref = tr[0]["scores"].cpu().numpy()[0], trace[0]["scores"]
+    big = s_ref >= 1e-20 * s_ref.max()
+    assert np.abs(s_gpu[big] / s_ref[big] - 1).max() <= (1e-3 if dtype == "f32" else 2e-2)
+    # this score favours the tokens next to the text: it is not the Eq. 2 ranking
+    eq2 = oracle.topk_select(oracle.stack_prefill(h0[0], M, layers, K, _rnd(dtype))[3][0]["scores"], K[0])
+    assert not np.array_equal(eq2, trace[0]["kept"])
+    kept = tr[0]["kept"].cpu().numpy()[0]
+    assert_kept_matches(kept, trace[0]["kept"], s_ref, tol=1e-4 if dtype == "f32" else 2e-2)
+    gi = idx.cpu().numpy()[0]
+    assert np.array_equal(gi[:K[0]], kept) and np.array_equal(gi[K[0]:], np.arange(n_vis, n_vis + M))
+    common, a, c = np.intersect1d(gi, ridx, return_indices=True)
+    assert len(common) >= 0.95 * len(ridx)
+    assert max_rel_err(host(out)[0][a], ref[c]) <= (2e-2 if dtype == "bf16" else 1e-3)
