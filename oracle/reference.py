@@ -218,13 +218,16 @@ def mamba_importance_full_dynamic(B, C, dt, A, n_vis, n_text):
     return s / (n_text * H)
 
 
-def attn_importance(q, k, n_vis, n_text, scale):
+def attn_importance(q, k, n_vis, n_text, scale, denominator="visual"):
     """s_i = 1/(M Hq) sum_{m,h} softmax_i( q_m^(h) . k_i^(kv(h)) * scale ), text -> visual.
 
-    The softmax normalises over the n_vis visual keys only (the paper's subscript i), so the
-    scores of one sequence sum to one.  q [T,Hq,d] (last n_text rows used), k [T,Hkv,d] (first
-    n_vis rows used); query head h reads KV head h // (Hq/Hkv).  Returns s [n_vis].
+    denominator="visual" (the paper's formula): the softmax normalises over the n_vis visual keys only (the
+    subscript i), so the scores of one sequence sum to one.  denominator="causal_row": the normaliser is the one
+    of the model's own causal attention row, i.e. it also holds the text keys m' <= m, so s_i is the attention
+    probability mass text query m really puts on visual token i (the scores then sum to less than one).
+    q [T,Hq,d] (last n_text rows used), k [T,Hkv,d]; query head h reads KV head h // (Hq/Hkv).  Returns s [n_vis].
     """
+    assert denominator in ("visual", "causal_row")
     q, k = _f64(q), _f64(k)
     T, Hq, d = q.shape
     Hkv = k.shape[1]
@@ -232,10 +235,15 @@ def attn_importance(q, k, n_vis, n_text, scale):
     s = np.zeros(n_vis)
     for h in range(Hq):
         kv = h // (Hq // Hkv)
-        logits = (q[n_vis:, h, :] @ k[:n_vis, kv, :].T) * scale   # [M, n_vis]
+        logits = (q[n_vis:, h, :] @ k[:, kv, :].T) * scale        # [M, T]
+        if denominator == "visual":
+            logits = logits[:, :n_vis]
+        else:
+            for m in range(n_text):
+                logits[m, n_vis + m + 1:] = -np.inf               # causal: text query m sees text keys m' <= m
         logits = logits - logits.max(axis=1, keepdims=True)
         e = np.exp(logits)
-        s += (e / e.sum(axis=1, keepdims=True)).sum(axis=0)
+        s += (e / e.sum(axis=1, keepdims=True))[:, :n_vis].sum(axis=0)
     return s / (n_text * Hq)
 
 
@@ -428,7 +436,7 @@ def attn_block(u, positions, prm, rnd=_identity):
     return out, dict(q=q, k=k, v=v, o=o, scale=scale)
 
 
-def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_score="decoupled"):
+def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_score="decoupled", attn_denominator="visual"):
     """Token-reduced prefill of a layer stack (one sequence).
 
     hidden [T0,D] with the n_text text rows last; layers: list of ("M"|"A", prm);
@@ -436,7 +444,7 @@ def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_scor
     tokens, its own score ranks the incoming visual tokens, and its OUTPUT is compacted when
     keep_counts[l] < n_cur.  Returns (hidden, positions, idx_map, trace) where trace lists per
     layer dict(n_in, scores or None, kept or None).  ``mamba_score``: "decoupled" (Eq. 2, the method) or
-    "full_dynamic" (|w| of Eq. 1, the paper's scoring ablation)."""
+    "full_dynamic" (|w| of Eq. 1, the paper's scoring ablation); ``attn_denominator`` as in attn_importance."""
     assert mamba_score in ("decoupled", "full_dynamic")
     h = _f64(hidden)
     T0 = h.shape[0]
@@ -453,7 +461,7 @@ def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_scor
                 score = (lambda: mamba_importance(mid["B"], mid["C"], mid["dt"], n_cur, n_text))
         else:
             out, mid = attn_block(h, pos, prm, rnd)
-            score = (lambda: attn_importance(mid["q"], mid["k"], n_cur, n_text, mid["scale"]))
+            score = (lambda: attn_importance(mid["q"], mid["k"], n_cur, n_text, mid["scale"], attn_denominator))
         rec = dict(n_in=n_cur, scores=None, kept=None)
         if K < n_cur:
             s = score()

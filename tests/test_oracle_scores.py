@@ -174,3 +174,44 @@ def test_full_dynamic_score_suppresses_early_tokens():
     assert np.all(np.diff(s) > 0) and s[0] < 0.2 * s[-1]
     flat = oracle.mamba_importance(B, C, dt, n_vis, M)
     np.testing.assert_allclose(flat, flat[0], rtol=1e-13)            # Eq. 2 does not see position at all
+
+
+# ---- attention score normalised by the model's own causal row (text keys m' <= m in the denominator) ----
+
+def _attn(seed, n_vis, M, Hq, Hkv, d):
+    r = np.random.default_rng(seed)
+    return r.normal(size=(n_vis + M, Hq, d)), r.normal(size=(n_vis + M, Hkv, d))
+
+
+def test_causal_row_attention_mass_is_what_the_attention_forward_applies():
+    # one-hot values turn the attention output into the attention probabilities themselves
+    n_vis, M, Hq, Hkv, d = 9, 4, 4, 2, 6
+    q, k = _attn(30, n_vis, M, Hq, Hkv, d)
+    T = n_vis + M
+    P = np.zeros((T, Hq, T))                                        # P[t, h, j] = causal softmax of row t
+    for c0 in range(0, T, d):                                       # d one-hot value columns per call
+        cols = np.eye(T)[:, c0:c0 + d]
+        v = np.zeros((T, Hkv, d)); v[:, :, :cols.shape[1]] = cols[:, None, :]
+        P[:, :, c0:c0 + cols.shape[1]] = oracle.attention_forward(q, k, v, 0.3)[:, :, :cols.shape[1]]
+    np.testing.assert_allclose(P.sum(axis=2), 1.0, rtol=1e-12)
+    ref = P[n_vis:, :, :n_vis].sum(axis=(0, 1)) / (M * Hq)
+    np.testing.assert_allclose(oracle.attn_importance(q, k, n_vis, M, 0.3, "causal_row"), ref, rtol=1e-12)
+
+
+def test_causal_row_attention_mass_closed_forms():
+    n_vis, M, Hq, Hkv, d = 7, 3, 2, 1, 4
+    q, k = _attn(31, n_vis, M, Hq, Hkv, d)
+    # zero queries: every causal row is uniform over its n_vis + m + 1 keys
+    s = oracle.attn_importance(np.zeros_like(q), k, n_vis, M, 1.0, "causal_row")
+    np.testing.assert_allclose(s, np.mean([1.0 / (n_vis + m + 1) for m in range(M)]), rtol=1e-13)
+    # the two normalisations differ by the share of each row's mass that stays on visual keys
+    sv = oracle.attn_importance(q, k, n_vis, M, 0.5)
+    sc = oracle.attn_importance(q, k, n_vis, M, 0.5, "causal_row")
+    assert abs(sv.sum() - 1.0) < 1e-12 and 0.0 < sc.sum() < 1.0 and np.all(sc < sv)
+    # a text key is invisible to earlier text queries: make the LAST text key overwhelmingly attractive; the
+    # first M-1 queries must keep all their visual mass (what is left over is the last query's share, >= 0)
+    k2 = k.copy(); k2[-1] = 50.0 * np.sign(q[n_vis:].mean(axis=(0, 1)))[None, :]
+    sc2 = oracle.attn_importance(q, k2, n_vis, M, 0.5, "causal_row")
+    first = oracle.attn_importance(q[:-1], k[:-1], n_vis, M - 1, 0.5, "causal_row") * (M - 1)
+    last_share = sc2 * M - first
+    assert np.all(last_share >= -1e-12) and last_share.sum() <= 1.0 + 1e-12
