@@ -239,7 +239,8 @@ def run_ours(args):
     ctx = binding.Context(local)
     # weights: seeded on the host, one replica per rank (the path does not shard: replicas only)
     layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], "f32")
-    stack = binding.Stack(ctx, layers, cfg["dtype"], Bz, n_vis, M, K, Q=cfg["mamba"]["Q"], mamba_score=args.mamba_score)
+    stack = binding.Stack(ctx, layers, cfg["dtype"], Bz, n_vis, M, K, Q=cfg["mamba"]["Q"], mamba_score=args.mamba_score,
+                          attn_denominator=args.attn_denominator)
     del layers
     h_host = torch.from_numpy(inputs.hidden_inputs(cfg["seed"] + 1000 * rank, T0, D, "bf16", batch=Bz)).to(torch.bfloat16)
     h_pin = h_host.pin_memory()
@@ -345,7 +346,7 @@ def run_ours(args):
         "config": {"workload": "C3 12-layer hybrid stack [M,M,M,M,M,A]x2, %d visual + %d text tokens, batch %d, "
                                "schedule %s" % (n_vis, M, Bz, "/".join(str(a // 100) for a in (cfg["alpha_bp"][::4] if args.schedule == "step"
                                                                                   else cfg["alpha_bp"]))),
-                   "mamba_score": args.mamba_score, "keep_counts": K, "l2": "inputs larger than L2 (hidden %d MB, workspace %d MB)"
+                   "mamba_score": args.mamba_score, "attn_denominator": args.attn_denominator, "keep_counts": K, "l2": "inputs larger than L2 (hidden %d MB, workspace %d MB)"
                                            % (h_dev.numel() * 2 >> 20, stack.ws_bytes >> 20),
                    "multi_gpu": "replicas only (the path does not shard)"},
         "roofline": roof, "cpu_baseline": cpu,
@@ -411,7 +412,7 @@ def run_micro(args):
         Hq, Hkv, d = at_["Hq"], at_["Hkv"], at_["d"]
         q = torch.randn(Bz, T, Hq, d, device=dev).to(bf)
         k = torch.randn(Bz, T, Hkv, d, device=dev).to(bf)
-        fn = lambda: binding.str_attn_importance(ctx, q, k, n_vis, M, 1.0 / np.sqrt(d))
+        fn = lambda: binding.str_attn_importance(ctx, q, k, n_vis, M, 1.0 / np.sqrt(d), denominator=args.attn_denominator)
         flops = 2 * Bz * n_vis * 2.0 * M * d * Hq
         nbytes = 2 * Bz * n_vis * 2.0 * Hkv * d
         bound = "tensor"
@@ -489,6 +490,8 @@ def main():
     ap.add_argument("--schedule", default="step", choices=["step", "sigmoid"], help="retention schedule of the stack")
     ap.add_argument("--mamba-score", default="decoupled", choices=["decoupled", "full_dynamic"],
                     help="Mamba-layer importance: Eq. 2 (the method) or |w| of Eq. 1 (the paper's scoring ablation)")
+    ap.add_argument("--attn-denominator", default="visual", choices=["visual", "causal_row"],
+                    help="normaliser of the attention-layer importance: visual keys only (the paper's formula) or the causal row")
     ap.add_argument("--x0", type=float, default=0.11, help="midpoint of the sigmoid schedule (0.11 / 0.24 / 0.41)")
     ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | mamba_dyn_score | attn_score | attn_fwd | "
                                                 "topk | compact | gemm")

@@ -107,10 +107,19 @@ int str_mamba_importance_dynamic(str_ctx *ctx, const str_ssm_score_shape *s, int
 typedef struct {
     int Bz, T, Hq, Hkv, d, dtype;
 } str_attn_score_shape;
+/* Normaliser of the attention score.  VISUAL: the paper's formula, softmax over the visual keys (scores sum to 1).
+ * CAUSAL_ROW: the denominator of the model's own causal attention row, which also holds the text keys m' <= m;
+ * the score is then the probability mass the text queries really put on each visual token (sums to < 1). */
+enum { STR_ATTN_DENOM_VISUAL = 0, STR_ATTN_DENOM_CAUSAL_ROW = 1 };
 size_t str_attn_importance_workspace_size(const str_attn_score_shape *s, int n_vis, int n_text);
 int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
                         const void *q, const void *k, float softmax_scale, float *scores_out,
                         void *workspace, size_t workspace_bytes, void *stream);
+/* Same with the normaliser chosen by `denominator` (STR_ATTN_DENOM_*); str_attn_importance is the VISUAL case.
+ * Same workspace size. */
+int str_attn_importance_ex(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
+                           const void *q, const void *k, float softmax_scale, int denominator,
+                           float *scores_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /* (2b, allocation-free variant)  The paper has no counterpart for this call; it exists for callers
  * that cannot allocate device memory (a plug-in inside a host with a fixed memory pool, a real-time
@@ -239,6 +248,7 @@ typedef struct {
     const int *keep_counts;            /* host array [n_layers], from str_schedule_keep_counts */
     int score_every_layer;             /* nonzero: also compute (not apply) the score at layers that do not reduce */
     int mamba_score_kind;              /* STR_SCORE_DECOUPLED (Eq. 2, the method) or STR_SCORE_FULL_DYNAMIC (Eq. 1, its ablation) */
+    int attn_score_denominator;        /* STR_ATTN_DENOM_VISUAL (the paper's formula) or STR_ATTN_DENOM_CAUSAL_ROW */
 } str_stack_desc;
 size_t str_stack_workspace_size(const str_stack_desc *d);
 /* hidden_in device [Bz, n_vis+n_text, D] dtype.  Outputs (device): hidden_out

@@ -50,7 +50,7 @@ class StackDesc(ctypes.Structure):
                                       "conv_width", "Hq", "Hkv", "d")]
                 + [("rope_theta", c_float), ("norm_eps", c_float), ("n_layers", c_int),
                    ("layers", ctypes.POINTER(Layer)), ("keep_counts", ctypes.POINTER(c_int)),
-                   ("score_every_layer", c_int), ("mamba_score_kind", c_int)])
+                   ("score_every_layer", c_int), ("mamba_score_kind", c_int), ("attn_score_denominator", c_int)])
 
 
 PROF_CATEGORIES = ["gemm", "ssd_scan", "mamba_score", "attn_score", "topk", "compact", "attn_fwd", "elementwise"]
@@ -61,7 +61,7 @@ EXPORTS = [
     "str_mamba2_prefill_workspace_size", "str_mamba2_prefill",
     "str_mamba_importance_workspace_size", "str_mamba_importance",
     "str_mamba_importance_dynamic_workspace_size", "str_mamba_importance_dynamic",
-    "str_attn_importance_workspace_size", "str_attn_importance", "str_attn_importance_static",
+    "str_attn_importance_workspace_size", "str_attn_importance", "str_attn_importance_ex", "str_attn_importance_static",
     "str_topk_select_workspace_size", "str_topk_select", "str_compact",
     "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
     "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_mamba_conv_split", "str_gated_rmsnorm",
@@ -206,16 +206,24 @@ def str_mamba_importance_dynamic(ctx, B, C, dt, A, n_vis, n_text):
     return out
 
 
-def str_attn_importance(ctx, q, k, n_vis, n_text, softmax_scale):
+STR_ATTN_DENOM = {"visual": 0, "causal_row": 1}
+
+
+def str_attn_importance(ctx, q, k, n_vis, n_text, softmax_scale, denominator="visual"):
     Bz, T, Hq, d = q.shape
     Hkv = k.shape[2]
     s = AttnScoreShape(Bz, T, Hq, Hkv, d, _dt(q))
     out = torch.empty((Bz, n_vis), dtype=torch.float32, device=q.device)
     nb = lib().str_attn_importance_workspace_size(ctypes.byref(s), c_int(n_vis), c_int(n_text))
     ws = ctx.workspace(nb)
-    _check(lib().str_attn_importance(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(q), _p(k),
-                                     c_float(softmax_scale), _p(out), _p(ws), c_size_t(ws.numel()), _stream()),
-           "str_attn_importance")
+    if denominator == "visual":
+        _check(lib().str_attn_importance(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(q), _p(k),
+                                         c_float(softmax_scale), _p(out), _p(ws), c_size_t(ws.numel()), _stream()),
+               "str_attn_importance")
+    else:
+        _check(lib().str_attn_importance_ex(ctx.handle, ctypes.byref(s), c_int(n_vis), c_int(n_text), _p(q), _p(k),
+                                            c_float(softmax_scale), c_int(STR_ATTN_DENOM[denominator]), _p(out), _p(ws),
+                                            c_size_t(ws.numel()), _stream()), "str_attn_importance_ex")
     return out
 
 
@@ -346,7 +354,7 @@ class Stack:
     [out_features, in_features] layout."""
 
     def __init__(self, ctx, layers, dtype, Bz, n_vis, n_text, keep_counts, Q=0, score_every_layer=False,
-                 rope_theta=1.0e6, norm_eps=1e-5, mamba_score="decoupled"):
+                 rope_theta=1.0e6, norm_eps=1e-5, mamba_score="decoupled", attn_denominator="visual"):
         self.ctx = ctx
         tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
         dev = "cuda:%d" % ctx.device
@@ -379,7 +387,8 @@ class Stack:
                               as_["Hq"], as_["Hkv"], as_["d"], rope_theta, norm_eps, len(layers),
                               ctypes.cast(arr, ctypes.POINTER(Layer)), ctypes.cast(self._kc, ctypes.POINTER(c_int)),
                               1 if score_every_layer else 0,
-                              {"decoupled": STR_SCORE_DECOUPLED, "full_dynamic": STR_SCORE_FULL_DYNAMIC}[mamba_score])
+                              {"decoupled": STR_SCORE_DECOUPLED, "full_dynamic": STR_SCORE_FULL_DYNAMIC}[mamba_score],
+                              STR_ATTN_DENOM[attn_denominator])
         self.tdt, self.dev = tdt, dev
         self.Bz, self.n_vis, self.n_text, self.D = Bz, n_vis, n_text, D
         self.keep_counts = [int(k) for k in keep_counts]

@@ -106,24 +106,33 @@ extern "C" size_t str_attn_importance_workspace_size(const str_attn_score_shape 
     return align_up((size_t)2 * s->Bz * s->Hq * n_text * (STR_ATTN_SCORE_MAX_SEGMENTS + 1) * sizeof(float), 256);
 }
 
-extern "C" int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
-                                   const void *q, const void *k, float softmax_scale, float *scores_out,
-                                   void *workspace, size_t workspace_bytes, void *stream) {
+extern "C" int str_attn_importance_ex(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
+                                      const void *q, const void *k, float softmax_scale, int denominator,
+                                      float *scores_out, void *workspace, size_t workspace_bytes, void *stream) {
     StrProfScope prof_scope(ctx, STR_CAT_ATTN_SCORE, stream);
     if (!ctx || !s || !q || !k) return STR_ERR_INVALID_ARG;
     if (s->Bz <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Hq % s->Hkv != 0 || s->d <= 0 || n_vis < 0 || n_text <= 0 ||
-        n_vis + n_text != s->T || !STR_DTYPE_OK(s->dtype))
+        n_vis + n_text != s->T || !STR_DTYPE_OK(s->dtype) ||
+        (denominator != STR_ATTN_DENOM_VISUAL && denominator != STR_ATTN_DENOM_CAUSAL_ROW))
         return STR_ERR_INVALID_ARG;
     if (n_vis == 0) return STR_OK;
     if (!scores_out || !workspace) return STR_ERR_INVALID_ARG;
     if (workspace_bytes < str_attn_importance_workspace_size(s, n_vis, n_text)) return STR_ERR_WORKSPACE_TOO_SMALL;
+    const bool causal_row = denominator == STR_ATTN_DENOM_CAUSAL_ROW;
     if (!str_force_simt() && ctx->encode_tiled && str_attn_importance_tc_supported(s, n_vis, n_text, q, k))
-        return str_attn_importance_tc(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, (float *)workspace,
+        return str_attn_importance_tc(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, (float *)workspace, causal_row,
                                       (cudaStream_t)stream);
     float *row_max = (float *)workspace;
     float *row_sum = row_max + (size_t)s->Bz * s->Hq * n_text;
-    return str_attn_importance_simt(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, row_max, row_sum,
+    return str_attn_importance_simt(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, row_max, row_sum, causal_row,
                                     (cudaStream_t)stream);
+}
+
+extern "C" int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
+                                   const void *q, const void *k, float softmax_scale, float *scores_out,
+                                   void *workspace, size_t workspace_bytes, void *stream) {
+    return str_attn_importance_ex(ctx, s, n_vis, n_text, q, k, softmax_scale, STR_ATTN_DENOM_VISUAL, scores_out, workspace,
+                                  workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------- glue: GEMM, attention forward

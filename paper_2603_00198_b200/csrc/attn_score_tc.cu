@@ -417,7 +417,7 @@ bool str_attn_importance_tc_supported(const str_attn_score_shape *s, int n_vis, 
 }
 
 int str_attn_importance_tc(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k,
-                           float scale, float *scores, float *workspace, cudaStream_t st) {
+                           float scale, float *scores, float *workspace, bool causal_row, cudaStream_t st) {
     const int n_pad = (n_text + 15) / 16 * 16, m_tiles = (n_text + 127) / 128;
     const int nseg = attn_score_segments(ctx, s, n_vis, n_text);
     const size_t rows = (size_t)s->Bz * s->Hq * n_text;
@@ -443,6 +443,8 @@ int str_attn_importance_tc(str_ctx *ctx, const str_attn_score_shape *s, int n_vi
                                                                       ws_max, ws_sum, ctx->status_dev);
     attn_merge_stats_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>((int)rows, n_text, nstore, ws_max, ws_sum, mg_max, mg_inv);
     rc = str_launch_ok(ctx, 2);
+    if (rc == STR_OK && causal_row)
+        rc = str_attn_text_keys_stats(ctx, s, n_vis, n_text, q, k, scale, true, mg_max, mg_inv, st);
     if (rc != STR_OK) return rc;
     const int tiles = ceil_div(n_vis, cs::TI);
     const int per_seq = ceil_div(ctx->sm_count, s->Bz);

@@ -6,7 +6,10 @@ int str_mamba_importance_simt(str_ctx *ctx, const str_ssm_score_shape *s, int n_
                               const void *C, const float *dt, float *scores, cudaStream_t st);
 int str_attn_importance_simt(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q,
                              const void *k, float scale, float *scores, float *row_max, float *row_sum,
-                             cudaStream_t st);
+                             bool causal_row, cudaStream_t st);
+// Folds the text keys m' <= m into the first pass's row statistics (causal-row normalisation of the attention score).
+int str_attn_text_keys_stats(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k,
+                             float scale, bool log2_inv, float *st_max, float *st_sum, cudaStream_t st);
 int str_ssd_simt(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float *dt, const float *A,
                  const void *B, const void *C, const float *D, const float *init_state, void *y,
                  float *final_state, cudaStream_t st);
@@ -43,6 +46,6 @@ int str_mamba_dyn_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int 
 #define STR_ATTN_SCORE_MAX_SEGMENTS 8
 bool str_attn_importance_tc_supported(const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k);
 int str_attn_importance_tc(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k,
-                           float scale, float *scores, float *workspace, cudaStream_t st);
+                           float scale, float *scores, float *workspace, bool causal_row, cudaStream_t st);
 int str_gated_rmsnorm_gather(str_ctx *ctx, int dtype, int Bz, int T_in, int n_vis, int n_text, int k, int d_inner, int ld_z,
                              float eps, const void *y, const void *z, const int32_t *kept, void *out, void *stream);

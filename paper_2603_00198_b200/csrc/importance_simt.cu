@@ -216,7 +216,7 @@ int launch_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, int n_vi
 template <typename T>
 int launch_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q,
                            const void *k, float scale, float *scores, float *row_max, float *row_sum,
-                           cudaStream_t st) {
+                           bool causal_row, cudaStream_t st) {
     const size_t smem1 = ((size_t)(TI + TM) * (s->d + 1) + 2 * TM * TI) * sizeof(float);
     const size_t smem2 = ((size_t)(TI + TM) * (s->d + 1) + 2 * TM + 4 * TI) * sizeof(float);
     if (smem1 > (size_t)ctx->max_smem_optin || smem2 > (size_t)ctx->max_smem_optin) return STR_ERR_UNSUPPORTED_SHAPE;
@@ -226,6 +226,8 @@ int launch_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, int n_vi
     attn_rowstats_kernel<T><<<g1, THREADS, smem1, st>>>(s->T, s->Hq, s->Hkv, s->d, n_vis, n_text, scale, (const T *)q,
                                                         (const T *)k, row_max, row_sum);
     int rc = str_launch_ok(ctx);
+    if (rc == STR_OK && causal_row)
+        rc = str_attn_text_keys_stats(ctx, s, n_vis, n_text, q, k, scale, false, row_max, row_sum, st);
     if (rc != STR_OK) return rc;
     dim3 g2(ceil_div(n_vis, TI), s->Bz);
     attn_colsum_kernel<T><<<g2, THREADS, smem2, st>>>(s->T, s->Hq, s->Hkv, s->d, n_vis, n_text, scale, (const T *)q,
@@ -244,10 +246,10 @@ int str_mamba_importance_simt(str_ctx *ctx, const str_ssm_score_shape *s, int n_
 
 int str_attn_importance_simt(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q,
                              const void *k, float scale, float *scores, float *row_max, float *row_sum,
-                             cudaStream_t st) {
+                             bool causal_row, cudaStream_t st) {
     return s->dtype == STR_BF16
-               ? launch_attn_importance<__nv_bfloat16>(ctx, s, n_vis, n_text, q, k, scale, scores, row_max, row_sum, st)
-               : launch_attn_importance<float>(ctx, s, n_vis, n_text, q, k, scale, scores, row_max, row_sum, st);
+               ? launch_attn_importance<__nv_bfloat16>(ctx, s, n_vis, n_text, q, k, scale, scores, row_max, row_sum, causal_row, st)
+               : launch_attn_importance<float>(ctx, s, n_vis, n_text, q, k, scale, scores, row_max, row_sum, causal_row, st);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -293,6 +295,6 @@ extern "C" int str_attn_importance_static(str_ctx *ctx, const str_attn_score_sha
     // Both halves are fully rewritten by the first pass before the second pass reads them, so nothing
     // left over from an earlier call is ever used and nothing needs clearing.
     float *row_max = base, *row_sum = base + rows;
-    return str_attn_importance_simt(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, row_max, row_sum,
+    return str_attn_importance_simt(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, row_max, row_sum, false,
                                     (cudaStream_t)stream);
 }

@@ -23,7 +23,8 @@ inline size_t imax(size_t a, size_t b) { return a > b ? a : b; }
 bool desc_ok(const str_stack_desc *d) {
     if (!d || d->Bz <= 0 || d->n_vis < 0 || d->n_text <= 0 || d->D <= 0 || d->n_layers <= 0 || !d->layers ||
         !d->keep_counts || (d->dtype != STR_F32 && d->dtype != STR_BF16) ||
-        (d->mamba_score_kind != STR_SCORE_DECOUPLED && d->mamba_score_kind != STR_SCORE_FULL_DYNAMIC))
+        (d->mamba_score_kind != STR_SCORE_DECOUPLED && d->mamba_score_kind != STR_SCORE_FULL_DYNAMIC) ||
+        (d->attn_score_denominator != STR_ATTN_DENOM_VISUAL && d->attn_score_denominator != STR_ATTN_DENOM_CAUSAL_ROW))
         return false;
     bool has_m = false, has_a = false;
     int n_cur = d->n_vis;
@@ -195,7 +196,8 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
             STR_TRY(str_attn_prefill(ctx, &as, bufA, bufB, bufC, scale, bufY, sub, r.sub_bytes, stream));
             if (want_score && n_cur > 0) {
                 str_attn_score_shape ss = {Bz, T, d->Hq, d->Hkv, d->d, dtype};
-                STR_TRY(str_attn_importance(ctx, &ss, n_cur, M, bufA, bufB, scale, scores, sub, r.sub_bytes, stream));
+                STR_TRY(str_attn_importance_ex(ctx, &ss, n_cur, M, bufA, bufB, scale, d->attn_score_denominator, scores, sub,
+                                               r.sub_bytes, stream));
             }
             if (reduce) {
                 STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));

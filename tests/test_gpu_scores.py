@@ -149,3 +149,25 @@ def test_score_argument_validation(ctx):
     a = inputs.attn_score_inputs(34, 40, 4, 2, 16, "f32")
     with pytest.raises(binding.StrError):
         binding.str_attn_importance(ctx, dev(a["q"]), dev(a["k"]), 41, 0, 1.0)
+
+
+@pytest.mark.parametrize("dtype,n_vis,M,Hq,Hkv,d,Bz", [
+    ("bf16", 16384, 128, 32, 8, 128, 1),     # config 2 shape, tensor cores
+    ("bf16", 1000, 100, 8, 2, 128, 2),       # padded text rows, ragged key tiles, batch
+    ("bf16", 300, 200, 4, 4, 128, 1),        # more than 128 text rows
+    ("f32", 1000, 33, 4, 2, 64, 2),          # plain fp32 path
+    ("bf16", 3, 2, 4, 1, 128, 1),            # fewer visual keys than text-visible keys matter most
+    ("bf16", 64, 1, 2, 2, 32, 1),
+])
+def test_attention_importance_causal_row_normaliser(ctx, dtype, n_vis, M, Hq, Hkv, d, Bz):
+    T = n_vis + M
+    x = inputs.attn_score_inputs(35, T, Hq, Hkv, d, dtype, batch=Bz)
+    scale = 1.0 / np.sqrt(d)
+    q, k = dev(x["q"], dtype), dev(x["k"], dtype)
+    got = binding.str_attn_importance(ctx, q, k, n_vis, M, scale, denominator="causal_row").cpu().numpy()
+    vis = binding.str_attn_importance(ctx, q, k, n_vis, M, scale).cpu().numpy()
+    ctx.check_status()
+    for b in range(Bz):
+        ref = oracle.attn_importance(x["q"][b], x["k"][b], n_vis, M, scale, "causal_row")
+        assert score_rel_err(got[b], ref) <= SCORE_TOL
+        assert got[b].sum() < 1.0 and np.all(got[b] <= vis[b] * (1 + 1e-5))      # some of every row's mass stays on text keys

@@ -179,3 +179,18 @@ def test_single_mamba_layer_reduced_by_the_full_dynamic_score(ctx, dtype, shape)
     common, a, c = np.intersect1d(gi, ridx, return_indices=True)
     assert len(common) >= 0.95 * len(ridx)
     assert max_rel_err(host(out)[0][a], ref[c]) <= (2e-2 if dtype == "bf16" else 1e-3)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_single_attention_layer_reduced_by_the_causal_row_score(ctx, dtype):
+    n_vis, M = 700, 24
+    layers = inputs.stack_params(67, "A", AS, AS, dtype)
+    h0 = inputs.hidden_inputs(67, n_vis + M, AS["D"], dtype)
+    K = [n_vis // 4]
+    ref, rpos, ridx, trace = oracle.stack_prefill(h0[0], M, layers, K, _rnd(dtype), attn_denominator="causal_row")
+    st = binding.Stack(ctx, layers, dtype, 1, n_vis, M, K, attn_denominator="causal_row")
+    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, dtype), want_trace=True)
+    ctx.check_status()
+    s_gpu, s_ref = tr[0]["scores"].cpu().numpy()[0], trace[0]["scores"]
+    assert s_ref.sum() < 1.0 and np.abs(s_gpu / s_ref - 1).max() <= (1e-3 if dtype == "f32" else 1e-2)
+    assert_kept_matches(tr[0]["kept"].cpu().numpy()[0], trace[0]["kept"], s_ref, tol=1e-4 if dtype == "f32" else 5e-3)
