@@ -189,6 +189,9 @@ int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const 
 int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, const void *in, void *out,
                 void *stream);
 
+/* out[i] = max(in[i], 0)^2, n elements of dtype; out may equal in.  (Activation of the FFN block.) */
+int str_relu_squared(str_ctx *ctx, int dtype, size_t n, const void *in, void *out, void *stream);
+
 /* Mamba-2 pre-scan step on the in_proj output zxbcdt [Bz*T, 2*d_inner + 2*G*n + H] =
  * [z | x B C | dt_raw]: causal depthwise conv (width W, zero left padding per sequence, taps
  * conv_w [d_inner+2Gn, W] fp32, last tap on the current token, bias conv_b fp32) + SiLU on the
@@ -225,14 +228,16 @@ int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const void *q, const
  * Whole stack: token-reduced prefill with a per-layer keep schedule (Sections 3.1-3.2).
  * Layer l's mixer runs on the incoming tokens, its own importance score ranks the incoming
  * visual tokens, and its OUTPUT is compacted to keep_counts[l] visual tokens when that is
- * smaller than the incoming count.  Block wrapper: h <- h + Mixer(RMSNorm(h)).
+ * smaller than the incoming count.  Block wrapper: h <- h + Mixer(RMSNorm(h)).  FFN layers (the
+ * hybrid's third block type, appendix "Models") only transform the rows they are given: their
+ * keep count must equal the incoming count.
  * ------------------------------------------------------------------------------------------ */
-enum { STR_LAYER_MAMBA = 0, STR_LAYER_ATTN = 1 };
+enum { STR_LAYER_MAMBA = 0, STR_LAYER_ATTN = 1, STR_LAYER_FFN = 2 };
 enum { STR_SCORE_DECOUPLED = 0, STR_SCORE_FULL_DYNAMIC = 1 };
 typedef struct {
-    int kind;             /* STR_LAYER_MAMBA or STR_LAYER_ATTN                                  */
-    const void *w_in;     /* device: Mamba in_proj [2*d_inner+2Gn+H, D] | attention W_qkv [(Hq+2Hkv)d, D] */
-    const void *w_out;    /* device: Mamba out_proj [D, d_inner]        | attention W_o [D, Hq*d]         */
+    int kind;             /* STR_LAYER_MAMBA, STR_LAYER_ATTN or STR_LAYER_FFN                   */
+    const void *w_in;     /* device: Mamba in_proj [2*d_inner+2Gn+H, D] | attention W_qkv [(Hq+2Hkv)d, D] | FFN W_up [ffn_dim, D] */
+    const void *w_out;    /* device: Mamba out_proj [D, d_inner]        | attention W_o [D, Hq*d]         | FFN W_down [D, ffn_dim] */
     const float *conv_w;  /* device, Mamba only: [d_inner+2Gn, W]                                */
     const float *conv_b;  /* device, Mamba only: [d_inner+2Gn]                                   */
     const float *dt_bias; /* device, Mamba only: [H]                                             */
@@ -249,6 +254,7 @@ typedef struct {
     int score_every_layer;             /* nonzero: also compute (not apply) the score at layers that do not reduce */
     int mamba_score_kind;              /* STR_SCORE_DECOUPLED (Eq. 2, the method) or STR_SCORE_FULL_DYNAMIC (Eq. 1, its ablation) */
     int attn_score_denominator;        /* STR_ATTN_DENOM_VISUAL (the paper's formula) or STR_ATTN_DENOM_CAUSAL_ROW */
+    int ffn_dim;                       /* width of the FFN layers, h <- h + W_down relu(W_up RMSNorm(h))^2; they never score or reduce */
 } str_stack_desc;
 size_t str_stack_workspace_size(const str_stack_desc *d);
 /* hidden_in device [Bz, n_vis+n_text, D] dtype.  Outputs (device): hidden_out

@@ -436,10 +436,22 @@ def attn_block(u, positions, prm, rnd=_identity):
     return out, dict(q=q, k=k, v=v, o=o, scale=scale)
 
 
+def ffn_block(u, prm, rnd=_identity):
+    """One pre-norm FFN block, u + W_down relu(W_up RMSNorm(u))^2.  prm: dict(D,F,W_up [D,F],W_down [F,D]).
+
+    The paper names FFN (MLP) blocks as the third block type of its hybrid (appendix "Models") and says nothing
+    about their inside; the squared-ReLU, ungated form is the one of the hybrid family it cites."""
+    u = _f64(u)
+    normed = rnd(rmsnorm(u))
+    up = rnd(normed @ _f64(prm["W_up"]))
+    act = rnd(np.maximum(up, 0.0) ** 2)
+    return rnd(u + act @ _f64(prm["W_down"]))
+
+
 def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_score="decoupled", attn_denominator="visual"):
     """Token-reduced prefill of a layer stack (one sequence).
 
-    hidden [T0,D] with the n_text text rows last; layers: list of ("M"|"A", prm);
+    hidden [T0,D] with the n_text text rows last; layers: list of ("M"|"A"|"F", prm);
     keep_counts[l] = visual tokens kept after layer l.  Layer l's mixer runs on the incoming
     tokens, its own score ranks the incoming visual tokens, and its OUTPUT is compacted when
     keep_counts[l] < n_cur.  Returns (hidden, positions, idx_map, trace) where trace lists per
@@ -453,6 +465,11 @@ def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_scor
     idx = np.arange(T0, dtype=np.int32)
     trace = []
     for (kind, prm), K in zip(layers, keep_counts):
+        if kind == "F":                                   # FFN layers transform the rows they get; they never score
+            assert K == n_cur
+            h = ffn_block(h, prm, rnd)
+            trace.append(dict(n_in=n_cur, scores=None, kept=None))
+            continue
         if kind == "M":
             out, mid = mamba2_block(h, prm, rnd)
             if mamba_score == "full_dynamic":

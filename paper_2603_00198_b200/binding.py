@@ -13,7 +13,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libstr.so")
 
 STR_F32, STR_BF16 = 0, 1
-STR_LAYER_MAMBA, STR_LAYER_ATTN = 0, 1
+STR_LAYER_MAMBA, STR_LAYER_ATTN, STR_LAYER_FFN = 0, 1, 2
 STR_SCORE_DECOUPLED, STR_SCORE_FULL_DYNAMIC = 0, 1
 c_int, c_float, c_size_t, c_void_p = ctypes.c_int, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
 
@@ -50,7 +50,8 @@ class StackDesc(ctypes.Structure):
                                       "conv_width", "Hq", "Hkv", "d")]
                 + [("rope_theta", c_float), ("norm_eps", c_float), ("n_layers", c_int),
                    ("layers", ctypes.POINTER(Layer)), ("keep_counts", ctypes.POINTER(c_int)),
-                   ("score_every_layer", c_int), ("mamba_score_kind", c_int), ("attn_score_denominator", c_int)])
+                   ("score_every_layer", c_int), ("mamba_score_kind", c_int), ("attn_score_denominator", c_int),
+                   ("ffn_dim", c_int)])
 
 
 PROF_CATEGORIES = ["gemm", "ssd_scan", "mamba_score", "attn_score", "topk", "compact", "attn_fwd", "elementwise"]
@@ -64,7 +65,7 @@ EXPORTS = [
     "str_attn_importance_workspace_size", "str_attn_importance", "str_attn_importance_ex", "str_attn_importance_static",
     "str_topk_select_workspace_size", "str_topk_select", "str_compact",
     "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
-    "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_mamba_conv_split", "str_gated_rmsnorm",
+    "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_relu_squared", "str_mamba_conv_split", "str_gated_rmsnorm",
     "str_rope_split", "str_attn_prefill_workspace_size", "str_attn_prefill",
     "str_stack_workspace_size", "str_stack_prefill", "str_stack_host_workspace_size",
     "str_stack_prefill_host",
@@ -302,6 +303,13 @@ def str_rmsnorm(ctx, x, eps=1e-5):
     return out
 
 
+def str_relu_squared(ctx, x, inplace=False):
+    out = x if inplace else torch.empty_like(x)
+    _check(lib().str_relu_squared(ctx.handle, c_int(_dt(x)), c_size_t(x.numel()), _p(x), _p(out), _stream()),
+           "str_relu_squared")
+    return out
+
+
 def str_mamba_conv_split(ctx, zxbcdt, conv_w, conv_b, dt_bias, Bz, T, H, p, n, G):
     W = conv_w.shape[1]
     dev, dtp = zxbcdt.device, zxbcdt.dtype
@@ -362,6 +370,7 @@ class Stack:
         arr = (Layer * len(layers))()
         m_shape = a_shape = None
         D = None
+        ffn_dim = 0
         for i, (kind, prm) in enumerate(layers):
             def up(a, t=tdt):
                 ten = torch.from_numpy(a).to(dev).to(t).contiguous()
@@ -373,6 +382,9 @@ class Stack:
                 arr[i] = Layer(STR_LAYER_MAMBA, up(prm["W_in"].T.copy()), up(prm["W_out"].T.copy()),
                                up(prm["conv_w"], torch.float32), up(prm["conv_b"], torch.float32),
                                up(prm["dt_bias"], torch.float32), up(prm["A"], torch.float32))
+            elif kind == "F":
+                ffn_dim = prm["F"]
+                arr[i] = Layer(STR_LAYER_FFN, up(prm["W_up"].T.copy()), up(prm["W_down"].T.copy()), None, None, None, None)
             else:
                 a_shape = prm
                 rope_theta = prm["theta"]
@@ -388,7 +400,7 @@ class Stack:
                               ctypes.cast(arr, ctypes.POINTER(Layer)), ctypes.cast(self._kc, ctypes.POINTER(c_int)),
                               1 if score_every_layer else 0,
                               {"decoupled": STR_SCORE_DECOUPLED, "full_dynamic": STR_SCORE_FULL_DYNAMIC}[mamba_score],
-                              STR_ATTN_DENOM[attn_denominator])
+                              STR_ATTN_DENOM[attn_denominator], ffn_dim)
         self.tdt, self.dev = tdt, dev
         self.Bz, self.n_vis, self.n_text, self.D = Bz, n_vis, n_text, D
         self.keep_counts = [int(k) for k in keep_counts]

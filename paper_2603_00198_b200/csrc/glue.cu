@@ -329,6 +329,46 @@ extern "C" int str_rmsnorm(str_ctx *ctx, int dtype, int rows, int D, float eps, 
     return str_launch_ok(ctx);
 }
 
+// Squared ReLU, element-wise (the FFN block's activation); in place when out == in.
+template <typename T>
+__global__ void __launch_bounds__(256) relu2_kernel(size_t n, const T *__restrict__ in, T *__restrict__ out) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float v = fmaxf(ldf(in + i), 0.f);
+        stf(out + i, v * v);
+    }
+}
+__global__ void __launch_bounds__(256) relu2_bf16_vec_kernel(size_t n8, const uint4 *__restrict__ in, uint4 *__restrict__ out) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+        const uint4 v = in[i];
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float lo = fmaxf(__uint_as_float(w[j] << 16), 0.f), hi = fmaxf(__uint_as_float(w[j] & 0xFFFF0000u), 0.f);
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(lo * lo, hi * hi);
+            w[j] = *reinterpret_cast<const uint32_t *>(&pk);
+        }
+        out[i] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+extern "C" int str_relu_squared(str_ctx *ctx, int dtype, size_t n, const void *in, void *out, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
+    if (!ctx || !in || !out || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
+    if (n == 0) return STR_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int cap = ctx->sm_count * 16;
+    if (dtype == STR_BF16 && n % 8 == 0 && (((uintptr_t)in | (uintptr_t)out) & 15) == 0) {
+        const size_t n8 = n / 8, blocks = (n8 + 255) / 256;
+        relu2_bf16_vec_kernel<<<(unsigned)(blocks < (size_t)cap ? blocks : cap), 256, 0, st>>>(n8, (const uint4 *)in, (uint4 *)out);
+    } else {
+        const size_t blocks = (n + 255) / 256;
+        const unsigned g = (unsigned)(blocks < (size_t)cap ? blocks : cap);
+        if (dtype == STR_BF16) relu2_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(n, (const __nv_bfloat16 *)in, (__nv_bfloat16 *)out);
+        else relu2_kernel<float><<<g, 256, 0, st>>>(n, (const float *)in, (float *)out);
+    }
+    return str_launch_ok(ctx);
+}
+
 static int launch_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps, const void *y,
                                 const void *z, void *out, RowGather rg, cudaStream_t st) {
     if (dtype == STR_BF16 && d_inner % 8 == 0 && ld_z % 8 == 0 && d_inner <= 256 * 8 * 4 &&

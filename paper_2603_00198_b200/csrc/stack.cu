@@ -36,6 +36,8 @@ bool desc_ok(const str_stack_desc *d) {
         } else if (L.kind == STR_LAYER_ATTN) {
             has_a = true;
             if (!L.w_in || !L.w_out) return false;
+        } else if (L.kind == STR_LAYER_FFN) {
+            if (!L.w_in || !L.w_out || d->ffn_dim <= 0 || d->keep_counts[l] != n_cur) return false;
         } else {
             return false;
         }
@@ -54,7 +56,12 @@ Regions plan(const str_stack_desc *d) {
     const size_t e = dtype_size(d->dtype);
     const size_t T0 = (size_t)d->n_vis + d->n_text, R = (size_t)d->Bz * T0;
     bool has_m = false, has_a = false;
-    for (int l = 0; l < d->n_layers; ++l) (d->layers[l].kind == STR_LAYER_MAMBA ? has_m : has_a) = true;
+    bool has_f = false;
+    for (int l = 0; l < d->n_layers; ++l) {
+        const int kind = d->layers[l].kind;
+        (kind == STR_LAYER_MAMBA ? has_m : kind == STR_LAYER_ATTN ? has_a : has_f) = true;
+    }
+    const size_t dff = has_f ? (size_t)d->ffn_dim : 0;
     const size_t d_inner = has_m ? (size_t)d->H * d->p : 0, gn = has_m ? (size_t)d->G * d->n : 0;
     const size_t dip = has_m ? 2 * d_inner + 2 * gn + d->H : 0;
     const size_t qd = has_a ? (size_t)d->Hq * d->d : 0, kd = has_a ? (size_t)d->Hkv * d->d : 0;
@@ -64,7 +71,7 @@ Regions plan(const str_stack_desc *d) {
     r.hidden[0] = take(R * d->D * e);
     r.hidden[1] = take(R * d->D * e);
     r.normed = take(R * d->D * e);
-    r.proj = take(R * imax(dip, dqkv) * e);
+    r.proj = take(R * imax(imax(dip, dqkv), dff) * e);
     r.bufA = take(R * imax(d_inner, qd) * e);
     r.bufB = take(R * imax(gn, kd) * e);
     r.bufC = take(R * imax(gn, kd) * e);
@@ -90,6 +97,7 @@ Regions plan(const str_stack_desc *d) {
         sub = imax(sub, str_attn_prefill_workspace_size(&at));
         sub = imax(sub, str_gemm_workspace_size((int)R, (int)dqkv, d->D, d->dtype));
     }
+    if (has_f) sub = imax(sub, str_gemm_workspace_size((int)R, (int)dff, d->D, d->dtype));
     sub = imax(sub, str_topk_select_workspace_size(d->Bz, d->n_vis, d->n_vis));
     r.sub_bytes = align_up(sub, 256);
     r.sub = take(r.sub_bytes);
@@ -186,6 +194,12 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
                 STR_TRY(str_gated_rmsnorm(ctx, dtype, rows, d_inner, dip, d->norm_eps, bufY, proj, bufA, stream));
                 STR_TRY(str_gemm(ctx, dtype, rows, D, d_inner, bufA, L.w_out, cur, dst, sub, r.sub_bytes, stream));
             }
+        } else if (L.kind == STR_LAYER_FFN) {
+            // h <- h + W_down relu(W_up RMSNorm(h))^2; the activation runs in place on the up-projection
+            const int F = d->ffn_dim;
+            STR_TRY(str_gemm(ctx, dtype, rows, F, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+            STR_TRY(str_relu_squared(ctx, dtype, (size_t)rows * F, proj, proj, stream));
+            STR_TRY(str_gemm(ctx, dtype, rows, D, F, proj, L.w_out, cur, dst, sub, r.sub_bytes, stream));
         } else {
             const int qd = d->Hq * d->d, kd = d->Hkv * d->d;
             STR_TRY(str_gemm(ctx, dtype, rows, qd + 2 * kd, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));

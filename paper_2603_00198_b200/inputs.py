@@ -139,13 +139,26 @@ def attn_layer_params(seed, layer, shape, dtype):
     return prm
 
 
-def stack_params(seed, pattern, mamba_shape, attn_shape, dtype):
+def ffn_layer_params(seed, layer, D, F, dtype):
+    """Random-init FFN block parameters.  W_up [D, F], W_down [F, D]; the down projection is scaled so that the
+    block's output stays O(1) after the squared activation."""
+    g = rng(seed, 200 + layer)
+    prm = dict(D=D, F=F)
+    prm["W_up"] = to_grid(g.standard_normal((D, F), dtype=np.float32) / np.sqrt(D), dtype)
+    prm["W_down"] = to_grid(g.standard_normal((F, D), dtype=np.float32) / np.sqrt(3.0 * F), dtype)
+    return prm
+
+
+def stack_params(seed, pattern, mamba_shape, attn_shape, dtype, ffn_dim=0):
     layers = []
     for l, kind in enumerate(pattern):
         if kind == "M":
             layers.append(("M", mamba_layer_params(seed, l, mamba_shape, dtype)))
         elif kind == "A":
             layers.append(("A", attn_layer_params(seed, l, attn_shape, dtype)))
+        elif kind == "F":
+            D = (mamba_shape or attn_shape)["D"]
+            layers.append(("F", ffn_layer_params(seed, l, D, ffn_dim or 4 * D, dtype)))
         else:
             raise ValueError(kind)
     return layers

@@ -126,3 +126,13 @@ def test_attention_forward_growing_logits_rescale(ctx):
         o = host(binding.str_attn_prefill(ctx, dev(q2, "bf16"), dev(kk, "bf16"), dev(v, "bf16"), scale))
         assert np.all(np.isfinite(o))
         assert max_rel_err(o[0], oracle.attention_forward(q2[0], kk[0], v[0], scale)) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("dtype,n", [("bf16", 8 * 1000), ("bf16", 1003), ("f32", 777), ("bf16", 8)])
+def test_relu_squared(ctx, dtype, n):
+    v = inputs.to_grid(inputs.hidden_inputs(57, 1, n, dtype)[0] * 2.0, dtype)
+    ref = np.maximum(v.astype(np.float64), 0.0) ** 2
+    x = dev(v, dtype)
+    assert max_rel_err(host(binding.str_relu_squared(ctx, x)), ref) <= TOL[dtype]
+    binding.str_relu_squared(ctx, x, inplace=True)
+    assert max_rel_err(host(x), ref) <= TOL[dtype]

@@ -194,3 +194,45 @@ def test_single_attention_layer_reduced_by_the_causal_row_score(ctx, dtype):
     s_gpu, s_ref = tr[0]["scores"].cpu().numpy()[0], trace[0]["scores"]
     assert s_ref.sum() < 1.0 and np.abs(s_gpu / s_ref - 1).max() <= (1e-3 if dtype == "f32" else 1e-2)
     assert_kept_matches(tr[0]["kept"].cpu().numpy()[0], trace[0]["kept"], s_ref, tol=1e-4 if dtype == "f32" else 5e-3)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_hybrid_stack_with_ffn_layers(ctx, dtype):
+    """The hybrid's three block types (appendix "Models": Mamba-2, FFN, attention) under a progressive schedule;
+    FFN layers run on whatever rows are left and never reduce."""
+    n_vis, M, Bz = 512, 16, 2
+    pattern = "MFAFMF"
+    layers = inputs.stack_params(68, pattern, MS, AS, dtype, ffn_dim=320)
+    h0 = inputs.hidden_inputs(68, n_vis + M, 128, dtype, batch=Bz)
+    K = [512, 512, 256, 256, 128, 128]
+    st = binding.Stack(ctx, layers, dtype, Bz, n_vis, M, K)
+    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, dtype), want_trace=True)
+    ctx.check_status()
+    assert [t["layer"] for t in tr] == [2, 4] and out.shape == (Bz, 128 + M, 128)
+    for b in range(Bz):
+        ref, rpos, ridx, trace = oracle.stack_prefill(h0[b], M, layers, K, _rnd(dtype))
+        gi = idx[b].cpu().numpy()
+        assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], np.arange(n_vis, n_vis + M))
+        swaps = assert_kept_matches(tr[0]["kept"][b].cpu().numpy(), trace[2]["kept"], trace[2]["scores"],
+                                    tol=1e-3 if dtype == "f32" else 5e-3)
+        common, a, c = np.intersect1d(gi, ridx, return_indices=True)
+        assert len(common) >= 0.97 * len(ridx)
+        row_err = np.abs(host(out)[b][a] - ref[c]).max(axis=1) / np.abs(ref).max()
+        if swaps == 0 and len(common) == len(ridx):
+            assert row_err.max() <= (5e-2 if dtype == "bf16" else 2e-3)
+        else:
+            assert np.median(row_err) <= 2e-2 and (row_err > 5e-2).mean() <= 0.25
+    # a keep count that would make an FFN layer reduce is refused
+    with pytest.raises(Exception):
+        bad = binding.Stack(ctx, layers, dtype, Bz, n_vis, M, [512, 256, 256, 256, 128, 128])
+        binding.str_stack_prefill(bad, dev(h0, dtype))
+
+
+def test_single_ffn_layer_teacher_forced(ctx):
+    n_vis, M = 300, 20
+    layers = inputs.stack_params(69, "F", MS_TC, MS_TC, "bf16", ffn_dim=1024)
+    h0 = inputs.hidden_inputs(69, n_vis + M, 512, "bf16")
+    st = binding.Stack(ctx, layers, "bf16", 1, n_vis, M, [n_vis])
+    out, pos, idx = binding.str_stack_prefill(st, dev(h0, "bf16"))
+    ref = oracle.ffn_block(h0[0], layers[0][1], oracle.round_to_bf16)
+    assert max_rel_err(host(out)[0], ref) <= 2e-2

@@ -1,6 +1,7 @@
 """CPU pins for the block glue around the recurrence.  The paper does not define these pieces,
 so they are pinned to textbook definitions, library routines and brute force on tiny inputs."""
 import numpy as np
+import pytest
 from scipy.special import softmax
 
 import oracle
@@ -97,3 +98,43 @@ def test_stack_identity_schedule_and_text_rows_last():
     assert np.array_equal(pos, idx)
     assert trace[0]["kept"] is None and len(trace[1]["kept"]) == 12 and len(trace[2]["kept"]) == 6
     np.testing.assert_allclose(trace[1]["scores"].sum(), 1.0, rtol=1e-12)   # layer 2 is attention
+
+
+def test_ffn_block_textbook_cases():
+    # the paper names FFN blocks without defining them; these pin the restatement to its own definition
+    r = np.random.default_rng(7)
+    D, F, T = 6, 10, 5
+    u = r.normal(size=(T, D))
+    prm = dict(D=D, F=F, W_up=r.normal(size=(D, F)), W_down=r.normal(size=(F, D)))
+    out = oracle.ffn_block(u, prm)
+    ref = np.zeros_like(u)
+    for t in range(T):                                   # explicit loops
+        nrm = u[t] / np.sqrt(np.mean(u[t] ** 2) + 1e-5)
+        hid = [max(sum(nrm[i] * prm["W_up"][i, f] for i in range(D)), 0.0) ** 2 for f in range(F)]
+        ref[t] = u[t] + [sum(hid[f] * prm["W_down"][f, j] for f in range(F)) for j in range(D)]
+    np.testing.assert_allclose(out, ref, rtol=1e-12)
+    # a zero down-projection leaves the residual stream alone; negating the up-projection of a row with all
+    # positive pre-activations switches the block off for it; scaling W_up by 2 scales the update by 4
+    np.testing.assert_array_equal(oracle.ffn_block(u, dict(prm, W_down=np.zeros((F, D)))), u)
+    pos_up = np.abs(prm["W_up"])
+    u_pos = np.abs(u)
+    np.testing.assert_allclose(oracle.ffn_block(u_pos, dict(prm, W_up=-pos_up)), u_pos, rtol=1e-13)
+    np.testing.assert_allclose(oracle.ffn_block(u, dict(prm, W_up=2 * prm["W_up"])) - u, 4 * (out - u), rtol=1e-12)
+
+
+def test_stack_with_ffn_layers_keeps_the_row_set():
+    from paper_2603_00198_b200 import inputs
+    ms = dict(D=32, H=4, p=8, n=8, G=2, Q=16, conv=4)
+    at = dict(D=32, Hq=4, Hkv=2, d=8, theta=1.0e6)
+    layers = inputs.stack_params(6, "MFAF", ms, at, "f32", ffn_dim=48)
+    n_vis, M = 24, 4
+    h0 = inputs.hidden_inputs(6, n_vis + M, 32, "f32")[0]
+    out, pos, idx, trace = oracle.stack_prefill(h0, M, layers, [12, 12, 6, 6])
+    assert out.shape == (6 + M, 32) and trace[1]["kept"] is None and trace[3]["kept"] is None
+    assert len(trace[0]["kept"]) == 12 and len(trace[2]["kept"]) == 6
+    # an FFN layer acts row by row: running it on the compacted rows equals compacting its output
+    h1, _ = oracle.mamba2_block(h0, layers[0][1])
+    rows = np.concatenate([trace[0]["kept"], np.arange(n_vis, n_vis + M)])
+    np.testing.assert_allclose(oracle.ffn_block(h1[rows], layers[1][1]), oracle.ffn_block(h1, layers[1][1])[rows], rtol=1e-13)
+    with pytest.raises(AssertionError):
+        oracle.stack_prefill(h0, M, layers, [12, 6, 6, 6])          # an FFN layer may not reduce
