@@ -42,6 +42,13 @@ def peaks():
 def workload(args):
     from paper_2603_00198_b200 import inputs
     cfg = dict(inputs.CONFIGS["C3"])
+    cfg["ffn_dim"] = 0
+    if args.pattern:
+        # secondary workloads: any sequence of Mamba-2 / attention / FFN layers (e.g. the hybrid's M F ... A F
+        # interleaving or an attention + FFN Transformer), three equal retention stages unless told otherwise
+        cfg["pattern"] = args.pattern
+        cfg["ffn_dim"] = args.ffn_dim or 4 * cfg["mamba"]["D"]
+        cfg["alpha_bp"] = inputs.sweep_alpha_bp(args.final_bp or 2500, len(args.pattern))
     if args.n_vis:
         cfg["n_vis"] = args.n_vis
     if args.final_bp:
@@ -53,6 +60,15 @@ def workload(args):
         cfg["alpha_bp"] = binding.str_sigmoid_schedule_bp(len(cfg["pattern"]), 20.0, args.x0, 1.0, 0.125)
     cfg["batch"] = args.batch
     return cfg
+
+
+def ffn_keep_counts(pattern, K, n_vis):
+    """FFN layers never reduce: a cut that the schedule places on one is taken by the next Mamba / attention layer."""
+    out, n_cur = [], n_vis
+    for kind, k in zip(pattern, K):
+        n_cur = n_cur if kind == "F" else min(k, n_cur)
+        out.append(n_cur)
+    return out
 
 
 # ------------------------------------------------------------------ algorithmic work per category
@@ -70,7 +86,11 @@ def work_model(cfg, keep_counts):
     for kind, K in zip(cfg["pattern"], keep_counts):
         T = n_cur + M
         To = min(K, n_cur) + M          # a reducing layer projects only the rows it keeps
-        if kind == "M":
+        if kind == "F":
+            F = cfg["ffn_dim"]
+            w["gemm"]["flops"] += 4.0 * Bz * T * D * F
+            w["gemm"]["bytes"] += 2.0 * (2 * Bz * T * (D + F) + 2 * D * F + Bz * T * D)
+        elif kind == "M":
             w["gemm"]["flops"] += 2.0 * Bz * T * D * dip + 2.0 * Bz * To * d_inner * D
             w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dip) + D * dip) + 2.0 * (Bz * To * (d_inner + 2 * D) + d_inner * D)
             w["ssd_scan"]["flops"] += Bz * T * (G * 2 * n * (Q + 1) / 2 + H * (2 * p * (Q + 1) / 2 + 4 * n * p))
@@ -154,9 +174,9 @@ def oracle_sample_tokens_per_s(cfg, n_vis_s, n_text_s, seed):
     same schedule.  Returns (tokens/s, seconds, threads)."""
     import oracle
     from paper_2603_00198_b200 import inputs
-    layers = inputs.stack_params(seed, cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"])
+    layers = inputs.stack_params(seed, cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"], ffn_dim=cfg.get("ffn_dim", 0))
     h0 = inputs.hidden_inputs(seed, n_vis_s + n_text_s, cfg["mamba"]["D"], cfg["dtype"])[0]
-    K = oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0)
+    K = ffn_keep_counts(cfg["pattern"], oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0), n_vis_s)
     t0 = time.perf_counter()
     oracle.stack_prefill(h0, n_text_s, layers, K, oracle.round_to_bf16)
     sec = time.perf_counter() - t0
@@ -174,9 +194,9 @@ def run_reference(args):
     cores = os.cpu_count() or 1
     n_text_s = 16
     n_vis_s = args.ref_tokens - n_text_s
-    layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"])
+    layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"], ffn_dim=cfg.get("ffn_dim", 0))
     h0 = inputs.hidden_inputs(cfg["seed"], n_vis_s + n_text_s, cfg["mamba"]["D"], cfg["dtype"])[0]
-    K = oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0)
+    K = ffn_keep_counts(cfg["pattern"], oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0), n_vis_s)
 
     def step():
         oracle.stack_prefill(h0, n_text_s, layers, K, oracle.round_to_bf16)
@@ -235,10 +255,11 @@ def run_ours(args):
     Bz, n_vis, M, D = cfg["batch"], cfg["n_vis"], cfg["n_text"], cfg["mamba"]["D"]
     T0 = n_vis + M
     K = binding.str_schedule_keep_counts(cfg["alpha_bp"], n_vis, cfg["min_keep"])
+    K = ffn_keep_counts(cfg["pattern"], K, n_vis)
 
     ctx = binding.Context(local)
     # weights: seeded on the host, one replica per rank (the path does not shard: replicas only)
-    layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], "f32")
+    layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], "f32", ffn_dim=cfg["ffn_dim"])
     stack = binding.Stack(ctx, layers, cfg["dtype"], Bz, n_vis, M, K, Q=cfg["mamba"]["Q"], mamba_score=args.mamba_score,
                           attn_denominator=args.attn_denominator)
     del layers
@@ -343,8 +364,10 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": "C3 12-layer hybrid stack [M,M,M,M,M,A]x2, %d visual + %d text tokens, batch %d, "
-                               "schedule %s" % (n_vis, M, Bz, "/".join(str(a // 100) for a in (cfg["alpha_bp"][::4] if args.schedule == "step"
+        "config": {"workload": "%s, %d visual + %d text tokens, batch %d, "
+                               "schedule %s" % ("C3 12-layer hybrid stack [M,M,M,M,M,A]x2" if not args.pattern else
+                                                "%d-layer stack %s (M Mamba-2, A attention, F FFN %d)" % (len(cfg["pattern"]), cfg["pattern"], cfg["ffn_dim"]),
+                                                n_vis, M, Bz, "/".join(str(a // 100) for a in (cfg["alpha_bp"][::4] if args.schedule == "step"
                                                                                   else cfg["alpha_bp"]))),
                    "mamba_score": args.mamba_score, "attn_denominator": args.attn_denominator, "keep_counts": K, "l2": "inputs larger than L2 (hidden %d MB, workspace %d MB)"
                                            % (h_dev.numel() * 2 >> 20, stack.ws_bytes >> 20),
@@ -488,6 +511,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the CPU oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--schedule", default="step", choices=["step", "sigmoid"], help="retention schedule of the stack")
+    ap.add_argument("--pattern", default="", help="layer pattern of a secondary workload, e.g. MFMFAFMFMFAF or AFAFAFAF")
+    ap.add_argument("--ffn-dim", type=int, default=0, help="FFN width of --pattern workloads (default 4 D)")
     ap.add_argument("--mamba-score", default="decoupled", choices=["decoupled", "full_dynamic"],
                     help="Mamba-layer importance: Eq. 2 (the method) or |w| of Eq. 1 (the paper's scoring ablation)")
     ap.add_argument("--attn-denominator", default="visual", choices=["visual", "causal_row"],
