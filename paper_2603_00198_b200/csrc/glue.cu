@@ -369,6 +369,58 @@ extern "C" int str_relu_squared(str_ctx *ctx, int dtype, size_t n, const void *i
     return str_launch_ok(ctx);
 }
 
+// RoPE + split, bf16, 16 bytes per access: one CTA per token row.  The rotation angles depend on the row's
+// position and the pair index only, so their sines and cosines (fp64 angle, reduced to [0, 2 pi), as in the
+// scalar kernel) are formed once per row in shared memory and shared by all heads; each thread then rotates 8
+// pairs (elements i..i+7 of the first half with the matching ones of the second half) or copies 8 v columns.
+__global__ void __launch_bounds__(256)
+rope_split_bf16_vec_kernel(int Hq, int Hkv, int d, double log2_theta, const int32_t *__restrict__ positions,
+                           const __nv_bfloat16 *__restrict__ qkv, __nv_bfloat16 *__restrict__ q_out,
+                           __nv_bfloat16 *__restrict__ k_out, __nv_bfloat16 *__restrict__ v_out) {
+    extern __shared__ float cs_sn[];                    // [half] cos | [half] sin
+    const int half = d / 2, h8 = half / 8;
+    const size_t row = blockIdx.x;
+    const int ld = (Hq + 2 * Hkv) * d;
+    const __nv_bfloat16 *base = qkv + row * ld;
+    const double pos = (double)positions[row];
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        const double inv_freq = exp2(-2.0 * (double)i / (double)d * log2_theta);
+        double ang = pos * inv_freq;
+        ang -= 6.283185307179586476925 * floor(ang * 0.15915494309189533576888);
+        float sn, cs;
+        sincosf((float)ang, &sn, &cs);
+        cs_sn[i] = cs;
+        cs_sn[half + i] = sn;
+    }
+    __syncthreads();
+    const int n_rot = (Hq + Hkv) * h8, n_v = Hkv * d / 8;
+    for (int e = threadIdx.x; e < n_rot + n_v; e += blockDim.x) {
+        if (e < n_rot) {
+            const int head = e / h8, i0 = (e - head * h8) * 8;
+            const uint4 va = __ldg(reinterpret_cast<const uint4 *>(base + head * d + i0));
+            const uint4 vb = __ldg(reinterpret_cast<const uint4 *>(base + head * d + half + i0));
+            float a[8], b[8];
+            unpack8(va, a);
+            unpack8(vb, b);
+            uint32_t oa[4], ob[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float c0 = cs_sn[i0 + 2 * j], s0 = cs_sn[half + i0 + 2 * j];
+                const float c1 = cs_sn[i0 + 2 * j + 1], s1 = cs_sn[half + i0 + 2 * j + 1];
+                oa[j] = pack2(a[2 * j] * c0 - b[2 * j] * s0, a[2 * j + 1] * c1 - b[2 * j + 1] * s1);
+                ob[j] = pack2(b[2 * j] * c0 + a[2 * j] * s0, b[2 * j + 1] * c1 + a[2 * j + 1] * s1);
+            }
+            __nv_bfloat16 *dst = head < Hq ? q_out + (row * Hq + head) * d : k_out + (row * Hkv + (head - Hq)) * d;
+            *reinterpret_cast<uint4 *>(dst + i0) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+            *reinterpret_cast<uint4 *>(dst + half + i0) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+        } else {
+            const int c = (e - n_rot) * 8;
+            *reinterpret_cast<uint4 *>(v_out + row * (size_t)(Hkv * d) + c) =
+                __ldg(reinterpret_cast<const uint4 *>(base + (Hq + Hkv) * d + c));
+        }
+    }
+}
+
 static int launch_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps, const void *y,
                                 const void *z, void *out, RowGather rg, cudaStream_t st) {
     if (dtype == STR_BF16 && d_inner % 8 == 0 && ld_z % 8 == 0 && d_inner <= 256 * 8 * 4 &&
@@ -454,7 +506,12 @@ extern "C" int str_rope_split(str_ctx *ctx, int dtype, int Bz, int T, int Hq, in
     dim3 grid(Bz * T, ceil_div(work, 256));
     cudaStream_t st = (cudaStream_t)stream;
     const double l2t = log2((double)theta);
-    if (dtype == STR_BF16)
+    if (dtype == STR_BF16 && d % 16 == 0 && d <= 8192 &&
+        (((uintptr_t)qkv | (uintptr_t)q_out | (uintptr_t)k_out | (uintptr_t)v_out) & 15) == 0)
+        rope_split_bf16_vec_kernel<<<Bz * T, 256, (size_t)d * sizeof(float), st>>>(
+            Hq, Hkv, d, l2t, positions, (const __nv_bfloat16 *)qkv, (__nv_bfloat16 *)q_out, (__nv_bfloat16 *)k_out,
+            (__nv_bfloat16 *)v_out);
+    else if (dtype == STR_BF16)
         rope_split_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(Hq, Hkv, d, l2t, positions, (const __nv_bfloat16 *)qkv,
                                                               (__nv_bfloat16 *)q_out, (__nv_bfloat16 *)k_out,
                                                               (__nv_bfloat16 *)v_out);
