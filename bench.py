@@ -91,8 +91,10 @@ def work_model(cfg, keep_counts):
             w["gemm"]["flops"] += 4.0 * Bz * T * D * F
             w["gemm"]["bytes"] += 2.0 * (2 * Bz * T * (D + F) + 2 * D * F + Bz * T * D)
         elif kind == "M":
-            w["gemm"]["flops"] += 2.0 * Bz * T * D * dip + 2.0 * Bz * To * d_inner * D
-            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dip) + D * dip) + 2.0 * (Bz * To * (d_inner + 2 * D) + d_inner * D)
+            # a reducing layer projects the gate z (d_inner of the dip columns) for the rows it keeps only
+            w["gemm"]["flops"] += 2.0 * Bz * D * (T * (dip - d_inner) + To * d_inner) + 2.0 * Bz * To * d_inner * D
+            w["gemm"]["bytes"] += 2.0 * (Bz * T * (D + dip - d_inner) + Bz * To * (D + d_inner) + D * dip) \
+                + 2.0 * (Bz * To * (d_inner + 2 * D) + d_inner * D)
             w["ssd_scan"]["flops"] += Bz * T * (G * 2 * n * (Q + 1) / 2 + H * (2 * p * (Q + 1) / 2 + 4 * n * p))
             w["ssd_scan"]["bytes"] += Bz * T * (2 * (2 * H * p + 2 * G * n) + 4 * H)
             if K < n_cur:

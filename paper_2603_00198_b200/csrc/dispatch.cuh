@@ -47,5 +47,10 @@ int str_mamba_dyn_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int 
 bool str_attn_importance_tc_supported(const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k);
 int str_attn_importance_tc(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text, const void *q, const void *k,
                            float scale, float *scores, float *workspace, bool causal_row, cudaStream_t st);
+// y rows gathered by `kept` (+ the text rows); z either gathered the same way or already compacted (z_compacted).
 int str_gated_rmsnorm_gather(str_ctx *ctx, int dtype, int Bz, int T_in, int n_vis, int n_text, int k, int d_inner, int ld_z,
-                             float eps, const void *y, const void *z, const int32_t *kept, void *out, void *stream);
+                             float eps, const void *y, const void *z, bool z_compacted, const int32_t *kept, void *out,
+                             void *stream);
+int str_mamba_conv_split_rows(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, int n, int G, int W, bool has_z,
+                              const void *zxbcdt, const float *conv_w, const float *conv_b, const float *dt_bias,
+                              void *x_out, void *B_out, void *C_out, float *dt_out, void *stream);

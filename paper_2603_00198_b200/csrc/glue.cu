@@ -31,7 +31,8 @@ rmsnorm_kernel(int D, float eps, const T *__restrict__ in, T *__restrict__ out) 
 
 // Source row of output row r when the rows are gathered on the fly (the same map as str_compact: per
 // sequence the k kept visual rows, then the text rows); the identity when kept == nullptr.
-struct RowGather { const int32_t *kept; int T_in, n_vis, k, T_out; };
+// z_direct: the gate rows are already compacted (row r of z belongs to output row r); y is still gathered.
+struct RowGather { const int32_t *kept; int T_in, n_vis, k, T_out; bool z_direct; };
 __device__ __forceinline__ size_t gather_src_row(const RowGather &g, size_t r) {
     if (!g.kept) return r;
     const size_t b = r / g.T_out;
@@ -47,7 +48,7 @@ gated_rmsnorm_kernel(int d_inner, int ld_z, float eps, const T *__restrict__ y, 
     __shared__ float red[32];
     const size_t srow = gather_src_row(rg, blockIdx.x);
     const T *yr = y + srow * d_inner;
-    const T *zr = z + srow * ld_z;
+    const T *zr = z + (rg.z_direct ? (size_t)blockIdx.x : srow) * ld_z;
     T *o = out + (size_t)blockIdx.x * d_inner;
     float ss = 0.f;
     for (int c = threadIdx.x; c < d_inner; c += blockDim.x) {
@@ -62,13 +63,13 @@ gated_rmsnorm_kernel(int d_inner, int ld_z, float eps, const T *__restrict__ y, 
 // One thread per (token, conv channel); consecutive threads walk consecutive channels.
 template <typename T>
 __global__ void __launch_bounds__(256)
-mamba_conv_split_kernel(int Tlen, int H, int p, int n, int G, int W, const T *__restrict__ zxbcdt,
+mamba_conv_split_kernel(int Tlen, int H, int p, int n, int G, int W, int zoff, const T *__restrict__ zxbcdt,
                         const float *__restrict__ conv_w, const float *__restrict__ conv_b,
                         const float *__restrict__ dt_bias, T *__restrict__ x_out, T *__restrict__ B_out,
                         T *__restrict__ C_out, float *__restrict__ dt_out) {
     const int d_inner = H * p, gn = G * n;
     const int conv_dim = d_inner + 2 * gn;
-    const int ld = 2 * d_inner + 2 * gn + H;
+    const int ld = zoff + conv_dim + H;                  // zoff = d_inner with the z columns in front, 0 without
     const int cols = conv_dim + H;                       // conv channels, then the H dt columns
     const size_t row = blockIdx.x;                       // b * Tlen + t (grid.x: no 65535 limit)
     const int t = (int)(row % Tlen);
@@ -77,13 +78,13 @@ mamba_conv_split_kernel(int Tlen, int H, int p, int n, int G, int W, const T *__
     const T *base = zxbcdt + row * ld;
     if (c >= conv_dim) {
         const int h = c - conv_dim;
-        dt_out[row * H + h] = softplus_f(ldf(base + d_inner + conv_dim + h) + dt_bias[h]);
+        dt_out[row * H + h] = softplus_f(ldf(base + zoff + conv_dim + h) + dt_bias[h]);
         return;
     }
     float acc = conv_b[c];
     for (int j = 0; j < W; ++j) {
         const int back = W - 1 - j;                      // tap j reads token t - (W-1) + j
-        if (t - back >= 0) acc = fmaf(conv_w[(size_t)c * W + j], ldf(base - (size_t)back * ld + d_inner + c), acc);
+        if (t - back >= 0) acc = fmaf(conv_w[(size_t)c * W + j], ldf(base - (size_t)back * ld + zoff + c), acc);
     }
     const float v = silu_f(acc);
     if (c < d_inner) stf(x_out + row * d_inner + c, v);
@@ -195,7 +196,7 @@ gated_rmsnorm_bf16_vec_kernel(int d_inner, int ld_z, float eps, const __nv_bfloa
     const int nvec = d_inner >> 3;
     const size_t srow = gather_src_row(rg, blockIdx.x);
     const uint4 *yr = reinterpret_cast<const uint4 *>(y + srow * d_inner);
-    const uint4 *zr = reinterpret_cast<const uint4 *>(z + srow * ld_z);
+    const uint4 *zr = reinterpret_cast<const uint4 *>(z + (rg.z_direct ? (size_t)blockIdx.x : srow) * ld_z);
     uint4 *o = reinterpret_cast<uint4 *>(out + (size_t)blockIdx.x * d_inner);
     uint4 yv[VPT], zv[VPT];
 #pragma unroll
@@ -241,14 +242,14 @@ __device__ __forceinline__ void unpack4(const uint2 &v, float (&f)[4]) {
     f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
 }
 __global__ void __launch_bounds__(256, 3)
-mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __nv_bfloat16 *__restrict__ zxbcdt,
+mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, int zoff, const __nv_bfloat16 *__restrict__ zxbcdt,
                                  const float *__restrict__ conv_w, const float *__restrict__ conv_b,
                                  const float *__restrict__ dt_bias, __nv_bfloat16 *__restrict__ x_out,
                                  __nv_bfloat16 *__restrict__ B_out, __nv_bfloat16 *__restrict__ C_out,
                                  float *__restrict__ dt_out) {
     const int d_inner = H * p, gn = G * n;
     const int conv_dim = d_inner + 2 * gn;
-    const int ld = 2 * d_inner + 2 * gn + H;
+    const int ld = zoff + conv_dim + H;
     const int tiles = (Tlen + CONV_TT - 1) / CONV_TT;
     const int b = blockIdx.x / tiles, t0 = (blockIdx.x % tiles) * CONV_TT;
     const int t1 = min(Tlen, t0 + CONV_TT);
@@ -257,7 +258,7 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
         for (int e = threadIdx.x; e < (t1 - t0) * H; e += blockDim.x) {
             const int t = t0 + e / H, h = e % H;
             dt_out[(row0 + t) * H + h] =
-                softplus_f(__bfloat162float(zxbcdt[(row0 + t) * ld + d_inner + conv_dim + h]) + dt_bias[h]);
+                softplus_f(__bfloat162float(zxbcdt[(row0 + t) * ld + zoff + conv_dim + h]) + dt_bias[h]);
         }
         return;
     }
@@ -275,7 +276,7 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, const __n
     if (c0 < d_inner) { dst = x_out + c0; dst_ld = d_inner; }
     else if (c0 < d_inner + gn) { dst = B_out + (c0 - d_inner); dst_ld = gn; }
     else { dst = C_out + (c0 - d_inner - gn); dst_ld = gn; }
-    const __nv_bfloat16 *src = zxbcdt + d_inner + c0;
+    const __nv_bfloat16 *src = zxbcdt + zoff + c0;
     float h3[CONV_CPT], h2[CONV_CPT], h1[CONV_CPT];     // inputs of tokens t-3, t-2, t-1
     {
         const uint2 zero = make_uint2(0u, 0u);
@@ -442,7 +443,7 @@ extern "C" int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner,
     if (!ctx || !y || !z || !out || rows < 0 || d_inner <= 0 || ld_z < d_inner || !STR_DTYPE_OK(dtype))
         return STR_ERR_INVALID_ARG;
     if (rows == 0) return STR_OK;
-    return launch_gated_rmsnorm(ctx, dtype, rows, d_inner, ld_z, eps, y, z, out, RowGather{nullptr, 0, 0, 0, 0},
+    return launch_gated_rmsnorm(ctx, dtype, rows, d_inner, ld_z, eps, y, z, out, RowGather{nullptr, 0, 0, 0, 0, false},
                                 (cudaStream_t)stream);
 }
 
@@ -450,21 +451,22 @@ extern "C" int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner,
 // kept[b][j] for j < k and from text row n_vis + (j - k) after that, so the rows a reducing layer is about to
 // drop are never normalised or projected.
 int str_gated_rmsnorm_gather(str_ctx *ctx, int dtype, int Bz, int T_in, int n_vis, int n_text, int k, int d_inner, int ld_z,
-                             float eps, const void *y, const void *z, const int32_t *kept, void *out, void *stream) {
+                             float eps, const void *y, const void *z, bool z_compacted, const int32_t *kept, void *out,
+                             void *stream) {
     StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
     if (!ctx || !y || !z || !out || !kept || Bz <= 0 || k < 0 || k > n_vis || T_in != n_vis + n_text || d_inner <= 0 ||
         ld_z < d_inner || !STR_DTYPE_OK(dtype))
         return STR_ERR_INVALID_ARG;
     const int rows = Bz * (k + n_text);
     if (rows == 0) return STR_OK;
-    return launch_gated_rmsnorm(ctx, dtype, rows, d_inner, ld_z, eps, y, z, out, RowGather{kept, T_in, n_vis, k, k + n_text},
+    return launch_gated_rmsnorm(ctx, dtype, rows, d_inner, ld_z, eps, y, z, out, RowGather{kept, T_in, n_vis, k, k + n_text, z_compacted},
                                 (cudaStream_t)stream);
 }
 
-extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, int n, int G, int W,
-                                    const void *zxbcdt, const float *conv_w, const float *conv_b,
-                                    const float *dt_bias, void *x_out, void *B_out, void *C_out, float *dt_out,
-                                    void *stream) {
+// has_z: rows are [z | x B C | dt_raw]; otherwise [x B C | dt_raw] (the gate columns are projected separately).
+int str_mamba_conv_split_rows(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, int n, int G, int W, bool has_z,
+                              const void *zxbcdt, const float *conv_w, const float *conv_b, const float *dt_bias,
+                              void *x_out, void *B_out, void *C_out, float *dt_out, void *stream) {
     StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
     if (!ctx || !zxbcdt || !conv_w || !conv_b || !dt_bias || !x_out || !B_out || !C_out || !dt_out || Bz <= 0 ||
         T <= 0 || H <= 0 || p <= 0 || n <= 0 || G <= 0 || W <= 0 || !STR_DTYPE_OK(dtype))
@@ -474,24 +476,33 @@ extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int 
     dim3 grid(Bz * T, ceil_div(cols, 256));
     cudaStream_t st = (cudaStream_t)stream;
     const int d_inner_ = H * p, gn_ = G * n;
+    const int zoff = has_z ? d_inner_ : 0;
     if (dtype == STR_BF16 && W == 4 && d_inner_ % 8 == 0 && gn_ % 8 == 0 && H % 8 == 0 &&
         (((uintptr_t)zxbcdt | (uintptr_t)x_out | (uintptr_t)B_out | (uintptr_t)C_out | (uintptr_t)conv_w) & 15) == 0) {
         const int tiles = ceil_div(T, CONV_TT);
         dim3 vgrid(Bz * tiles, ceil_div((d_inner_ + 2 * gn_) / CONV_CPT, 256) + 1);
         mamba_conv_split_bf16_vec_kernel<<<vgrid, 256, 0, st>>>(
-            T, H, p, n, G, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
+            T, H, p, n, G, zoff, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
             (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out);
         return str_launch_ok(ctx);
     }
     if (dtype == STR_BF16)
         mamba_conv_split_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
-            T, H, p, n, G, W, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
+            T, H, p, n, G, W, zoff, (const __nv_bfloat16 *)zxbcdt, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
             (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out);
     else
-        mamba_conv_split_kernel<float><<<grid, 256, 0, st>>>(T, H, p, n, G, W, (const float *)zxbcdt, conv_w, conv_b,
+        mamba_conv_split_kernel<float><<<grid, 256, 0, st>>>(T, H, p, n, G, W, zoff, (const float *)zxbcdt, conv_w, conv_b,
                                                             dt_bias, (float *)x_out, (float *)B_out, (float *)C_out,
                                                             dt_out);
     return str_launch_ok(ctx);
+}
+
+extern "C" int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, int n, int G, int W,
+                                    const void *zxbcdt, const float *conv_w, const float *conv_b,
+                                    const float *dt_bias, void *x_out, void *B_out, void *C_out, float *dt_out,
+                                    void *stream) {
+    return str_mamba_conv_split_rows(ctx, dtype, Bz, T, H, p, n, G, W, true, zxbcdt, conv_w, conv_b, dt_bias, x_out, B_out,
+                                     C_out, dt_out, stream);
 }
 
 extern "C" int str_rope_split(str_ctx *ctx, int dtype, int Bz, int T, int Hq, int Hkv, int d, float theta,

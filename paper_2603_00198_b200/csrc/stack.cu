@@ -169,9 +169,16 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
         const int rows_out = reduce ? Bz * (K + M) : rows;
         if (L.kind == STR_LAYER_MAMBA) {
             const int d_inner = d->H * d->p, gn = d->G * d->n, dip = 2 * d_inner + 2 * gn + d->H;
-            STR_TRY(str_gemm(ctx, dtype, rows, dip, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
-            STR_TRY(str_mamba_conv_split(ctx, dtype, Bz, T, d->H, d->p, d->n, d->G, d->conv_width, proj, L.conv_w,
-                                         L.conv_b, L.dt_bias, bufA, bufB, bufC, dt, stream));
+            if (reduce) {
+                // the gate z is only needed for the rows that survive: project [x B C | dt] for every row now (the
+                // weight rows after the first d_inner) and z for the kept rows after the selection
+                const char *w_rest = (const char *)L.w_in + (size_t)d_inner * D * dtype_size(dtype);
+                STR_TRY(str_gemm(ctx, dtype, rows, dip - d_inner, D, normed, w_rest, nullptr, proj, sub, r.sub_bytes, stream));
+            } else {
+                STR_TRY(str_gemm(ctx, dtype, rows, dip, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+            }
+            STR_TRY(str_mamba_conv_split_rows(ctx, dtype, Bz, T, d->H, d->p, d->n, d->G, d->conv_width, !reduce, proj,
+                                              L.conv_w, L.conv_b, L.dt_bias, bufA, bufB, bufC, dt, stream));
             str_ssd_shape s = {Bz, T, d->H, d->p, d->n, d->G, d->Q, dtype};
             STR_TRY(str_mamba2_prefill(ctx, &s, bufA, dt, L.A, bufB, bufC, nullptr, nullptr, bufY, nullptr, sub,
                                        r.sub_bytes, stream));
@@ -184,11 +191,17 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
             }
             if (reduce) {
                 STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));
-                // residual rows, positions and the index map of the survivors (normed is free after in_proj)
+                // z of the survivors: their normed rows are gathered into the layer's output buffer (free until the
+                // output projection writes it), projected with the first d_inner weight rows into the projection
+                // buffer (its [x B C | dt] content was consumed by the conv)
+                STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, normed, nullptr, nullptr, kept, dst, nullptr, nullptr,
+                                    stream));
+                STR_TRY(str_gemm(ctx, dtype, rows_out, d_inner, D, dst, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+                // residual rows, positions and the index map of the survivors (normed is free now)
                 STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, cur, pos[psel], idx[psel], kept, normed, pdst, idst,
                                     stream));
-                STR_TRY(str_gated_rmsnorm_gather(ctx, dtype, Bz, T, n_cur, M, K, d_inner, dip, d->norm_eps, bufY, proj, kept,
-                                                 bufA, stream));
+                STR_TRY(str_gated_rmsnorm_gather(ctx, dtype, Bz, T, n_cur, M, K, d_inner, d_inner, d->norm_eps, bufY, proj, true,
+                                                 kept, bufA, stream));
                 STR_TRY(str_gemm(ctx, dtype, rows_out, D, d_inner, bufA, L.w_out, normed, dst, sub, r.sub_bytes, stream));
             } else {
                 STR_TRY(str_gated_rmsnorm(ctx, dtype, rows, d_inner, dip, d->norm_eps, bufY, proj, bufA, stream));
