@@ -58,6 +58,28 @@ def test_mamba_importance_full_length_sampled_tokens(ctx, n_vis):
     assert score_rel_err(got[sample], ref) <= 1e-3
 
 
+def test_mamba_full_dynamic_score_full_length(ctx):
+    """Eq. 1 variant at the benchmark's length: the cumulative decay of a token depends on every dt between it and
+    the text rows, so the oracle is evaluated on the whole sequence (seconds in fp64)."""
+    H, n, G = MS["H"], MS["n"], MS["G"]
+    n_vis, T = N_VIS, N_VIS + M
+    g = inputs.rng(86, n_vis)
+    Bm = inputs.to_grid(g.standard_normal((1, T, G, n), dtype=np.float32), "bf16")
+    Cm = inputs.to_grid(g.standard_normal((1, T, G, n), dtype=np.float32), "bf16")
+    dt = g.uniform(1e-3, 1e-1, size=(1, T, H)).astype(np.float32)
+    A = (-np.exp(g.uniform(0.0, np.log(16.0), size=H))).astype(np.float32)
+    got = binding.str_mamba_importance_dynamic(ctx, dev(Bm, "bf16"), dev(Cm, "bf16"), dev(dt), dev(A), n_vis, M).cpu().numpy()[0]
+    ctx.check_status()
+    ref = oracle.mamba_importance_full_dynamic(Bm[0], Cm[0], dt[0], A, n_vis, M)
+    floor = 1e-30 * ref.max()
+    big = ref >= floor
+    assert big.sum() > 500 and np.all(got[~big] <= 2 * floor) and np.all(got >= 0)
+    assert score_rel_err(got[big], ref[big]) <= 1e-3
+    k = int(big.sum() // 2)
+    kept = binding.str_topk_select(ctx, dev(got[None]), k).cpu().numpy()[0]
+    assert_kept_matches(kept, oracle.topk_select(ref, k), ref)
+
+
 def test_gemm_full_size_sampled_entries(ctx):
     Mrows, K = N_VIS + M, MS["D"]
     N = 2 * MS["H"] * MS["p"] + 2 * MS["G"] * MS["n"] + MS["H"]            # in_proj width 18560
