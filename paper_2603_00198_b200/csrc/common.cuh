@@ -23,6 +23,8 @@ struct str_ctx {
     void *encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), or nullptr
     long long launches;       // host-side count of kernels launched through this context
     size_t smem_attr[8];      // dynamic shared memory already opted into on this device, per tensor-core kernel
+    cudaStream_t copy_stream; // host-buffer entry point: input chunks are copied on this stream while the caller's
+    cudaEvent_t copy_ev[8];   // stream computes; [0] orders the copies after the caller's earlier work, [1..] = chunk landed
     bool prof_on;             // record an event pair per leaf call
     std::vector<str_prof_span> prof_spans;
     std::vector<cudaEvent_t> prof_free;

@@ -16,6 +16,8 @@ extern "C" int str_create(int device, str_ctx **out) {
     c->launches = 0;
     c->prof_on = false;
     for (size_t &v : c->smem_attr) v = 0;
+    c->copy_stream = nullptr;
+    for (cudaEvent_t &ev : c->copy_ev) ev = nullptr;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return STR_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;
@@ -38,6 +40,9 @@ extern "C" int str_destroy(str_ctx *ctx) {
     cudaFree(ctx->status_dev);
     for (auto &sp : ctx->prof_spans) { cudaEventDestroy(sp.beg); cudaEventDestroy(sp.end); }
     for (auto &ev : ctx->prof_free) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : ctx->copy_ev)
+        if (ev) cudaEventDestroy(ev);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     delete ctx;
     return STR_OK;
 }

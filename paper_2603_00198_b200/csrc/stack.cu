@@ -112,15 +112,20 @@ extern "C" size_t str_stack_workspace_size(const str_stack_desc *d) {
     return plan(d).total;
 }
 
+// Input feed of the host-buffer entry point: the hidden states arrive in `chunks` row blocks of `rows_per_chunk`
+// rows, block j being complete once `ready[j]` has fired.  Only the first layer's norm and first projection read
+// the input row by row, so only they are issued per block.
+struct StackFeed { int chunks; int rows_per_chunk; cudaEvent_t *ready; };
+
 #define STR_TRY(call)              \
     do {                           \
         int _rc = (call);          \
         if (_rc != STR_OK) return _rc; \
     } while (0)
 
-extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in, void *hidden_out,
-                                 int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace,
-                                 float *scores_trace, void *workspace, size_t workspace_bytes, void *stream) {
+static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in, void *hidden_out,
+                              int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace, float *scores_trace,
+                              void *workspace, size_t workspace_bytes, void *stream, const StackFeed *feed) {
     if (!ctx || !desc_ok(d) || !hidden_in || !hidden_out || !workspace) return STR_ERR_INVALID_ARG;
     if (((uintptr_t)workspace & 255) != 0) return STR_ERR_INVALID_ARG;
     const Regions r = plan(d);
@@ -159,7 +164,21 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
         int32_t *kept = (reduce && kept_trace) ? kept_trace + kept_off : kept_int;
         void *mix_out = (last && !reduce) ? hidden_out : hid[hsel];
 
-        STR_TRY(str_rmsnorm(ctx, dtype, rows, D, d->norm_eps, cur, normed, stream));
+        // RMSNorm of the layer input and the layer's first projection [rows x N] = normed W^T into `proj`
+        auto norm_and_project = [&](int N, const void *w) -> int {
+            const bool fed = feed && l == 0;
+            const int step = fed ? feed->rows_per_chunk : rows;
+            const size_t esz = dtype_size(dtype);
+            for (int j = 0, r0 = 0; r0 < rows; ++j, r0 += step) {
+                const int nr = rows - r0 < step ? rows - r0 : step;
+                if (fed) STR_CUDA_OK(cudaStreamWaitEvent(st, feed->ready[j], 0));
+                STR_TRY(str_rmsnorm(ctx, dtype, nr, D, d->norm_eps, (const char *)cur + (size_t)r0 * D * esz,
+                                    (char *)normed + (size_t)r0 * D * esz, stream));
+                STR_TRY(str_gemm(ctx, dtype, nr, N, D, (const char *)normed + (size_t)r0 * D * esz, w, nullptr,
+                                 (char *)proj + (size_t)r0 * N * esz, sub, r.sub_bytes, stream));
+            }
+            return STR_OK;
+        };
         // A reducing layer selects BEFORE the mixer's epilogue: the score only needs the projections, so the rows
         // about to be dropped skip the gate / norm / output projection (their inputs still feed the scan state
         // and the attention keys).  The surviving rows come out bit-identical to computing every row first.
@@ -173,9 +192,9 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
                 // the gate z is only needed for the rows that survive: project [x B C | dt] for every row now (the
                 // weight rows after the first d_inner) and z for the kept rows after the selection
                 const char *w_rest = (const char *)L.w_in + (size_t)d_inner * D * dtype_size(dtype);
-                STR_TRY(str_gemm(ctx, dtype, rows, dip - d_inner, D, normed, w_rest, nullptr, proj, sub, r.sub_bytes, stream));
+                STR_TRY(norm_and_project(dip - d_inner, w_rest));
             } else {
-                STR_TRY(str_gemm(ctx, dtype, rows, dip, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+                STR_TRY(norm_and_project(dip, L.w_in));
             }
             STR_TRY(str_mamba_conv_split_rows(ctx, dtype, Bz, T, d->H, d->p, d->n, d->G, d->conv_width, !reduce, proj,
                                               L.conv_w, L.conv_b, L.dt_bias, bufA, bufB, bufC, dt, stream));
@@ -210,12 +229,12 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
         } else if (L.kind == STR_LAYER_FFN) {
             // h <- h + W_down relu(W_up RMSNorm(h))^2; the activation runs in place on the up-projection
             const int F = d->ffn_dim;
-            STR_TRY(str_gemm(ctx, dtype, rows, F, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+            STR_TRY(norm_and_project(F, L.w_in));
             STR_TRY(str_relu_squared(ctx, dtype, (size_t)rows * F, proj, proj, stream));
             STR_TRY(str_gemm(ctx, dtype, rows, D, F, proj, L.w_out, cur, dst, sub, r.sub_bytes, stream));
         } else {
             const int qd = d->Hq * d->d, kd = d->Hkv * d->d;
-            STR_TRY(str_gemm(ctx, dtype, rows, qd + 2 * kd, D, normed, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
+            STR_TRY(norm_and_project(qd + 2 * kd, L.w_in));
             STR_TRY(str_rope_split(ctx, dtype, Bz, T, d->Hq, d->Hkv, d->d, d->rope_theta, pos[psel], proj, bufA, bufB,
                                    bufC, stream));
             str_attn_shape as = {Bz, T, d->Hq, d->Hkv, d->d, dtype};
@@ -256,6 +275,13 @@ extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const vo
     return STR_OK;
 }
 
+extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in, void *hidden_out,
+                                 int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace,
+                                 float *scores_trace, void *workspace, size_t workspace_bytes, void *stream) {
+    return stack_prefill_impl(ctx, d, hidden_in, hidden_out, positions_out, idx_map_out, kept_trace, scores_trace, workspace,
+                              workspace_bytes, stream, nullptr);
+}
+
 extern "C" size_t str_stack_host_workspace_size(const str_stack_desc *d) {
     if (!desc_ok(d)) return 0;
     const size_t e = dtype_size(d->dtype);
@@ -278,9 +304,27 @@ extern "C" int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, con
     void *out_dev = ws; ws += align_up(Rout * d->D * e, 256);
     int32_t *pos_dev = (int32_t *)ws; ws += align_up(Rout * 4, 256);
     int32_t *idx_dev = (int32_t *)ws; ws += align_up(Rout * 4, 256);
-    STR_CUDA_OK(cudaMemcpyAsync(in_dev, hidden_in_host, Rin * d->D * e, cudaMemcpyHostToDevice, st));
-    int rc = str_stack_prefill(ctx, d, in_dev, out_dev, pos_dev, idx_dev, nullptr, nullptr, ws,
-                               workspace_bytes - (size_t)(ws - (char *)workspace), stream);
+    // The input is copied in a few row blocks on a stream of the context's own, so that the first layer's norm and
+    // projection of block j run while block j+1 is still on its way (pinned host memory makes the copies
+    // asynchronous; with pageable memory they simply serialise).  Stream and events are created on first use.
+    constexpr int CHUNKS = 4;
+    if (!ctx->copy_stream) {
+        STR_CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i <= CHUNKS; ++i) STR_CUDA_OK(cudaEventCreateWithFlags(&ctx->copy_ev[i], cudaEventDisableTiming));
+    }
+    const size_t per = align_up((Rin + CHUNKS - 1) / CHUNKS, 128);          // rows per block: whole GEMM row tiles
+    STR_CUDA_OK(cudaEventRecord(ctx->copy_ev[0], st));                       // after whatever the caller queued before
+    STR_CUDA_OK(cudaStreamWaitEvent(ctx->copy_stream, ctx->copy_ev[0], 0));
+    int nblk = 0;
+    for (size_t r0 = 0; r0 < Rin; r0 += per, ++nblk) {
+        const size_t nr = Rin - r0 < per ? Rin - r0 : per;
+        STR_CUDA_OK(cudaMemcpyAsync((char *)in_dev + r0 * d->D * e, (const char *)hidden_in_host + r0 * d->D * e, nr * d->D * e,
+                                    cudaMemcpyHostToDevice, ctx->copy_stream));
+        STR_CUDA_OK(cudaEventRecord(ctx->copy_ev[1 + nblk], ctx->copy_stream));
+    }
+    const StackFeed feed = {nblk, (int)per, ctx->copy_ev + 1};
+    int rc = stack_prefill_impl(ctx, d, in_dev, out_dev, pos_dev, idx_dev, nullptr, nullptr, ws,
+                                workspace_bytes - (size_t)(ws - (char *)workspace), stream, &feed);
     if (rc != STR_OK) return rc;
     STR_CUDA_OK(cudaMemcpyAsync(hidden_out_host, out_dev, Rout * d->D * e, cudaMemcpyDeviceToHost, st));
     if (idx_map_out_host)
