@@ -61,3 +61,9 @@ def test_argument_validation_needs_no_gpu(libstr):
     assert libstr.str_topk_select(None, 1, 8, 4, None, None, None, ctypes.c_size_t(0), None) == -1
     assert libstr.str_compact(None, 1, 8, 6, 2, 3, 16, 1, None, None, None, None, None, None, None, None) == -1
     assert libstr.str_destroy(None) == -1
+    # the score variants and the FFN activation too
+    assert libstr.str_mamba_importance_dynamic(None, None, 8, 2, None, None, None, None, None, None, ctypes.c_size_t(0), None) == -1
+    assert libstr.str_attn_importance_ex(None, None, 8, 2, None, None, ctypes.c_float(1.0), 0, None, None, ctypes.c_size_t(0), None) == -1
+    assert libstr.str_relu_squared(None, 1, ctypes.c_size_t(8), None, None, None) == -1
+    libstr.str_mamba_importance_dynamic_workspace_size.restype = ctypes.c_size_t
+    assert libstr.str_mamba_importance_dynamic_workspace_size(None, 8, 2) == 0

@@ -171,3 +171,32 @@ def test_attention_importance_causal_row_normaliser(ctx, dtype, n_vis, M, Hq, Hk
         ref = oracle.attn_importance(x["q"][b], x["k"][b], n_vis, M, scale, "causal_row")
         assert score_rel_err(got[b], ref) <= SCORE_TOL
         assert got[b].sum() < 1.0 and np.all(got[b] <= vis[b] * (1 + 1e-5))      # some of every row's mass stays on text keys
+
+
+def test_score_variants_reject_bad_arguments(ctx):
+    d = inputs.ssd_inputs(36, 40, 8, 16, 128, 2, "bf16")
+    B, C, dt, A = dev(d["B"], "bf16"), dev(d["C"], "bf16"), dev(d["dt"]), dev(d["A"])
+    s = binding.SsmScoreShape(1, 40, 8, 128, 2, binding.STR_BF16)
+    L = binding.lib()
+    import ctypes
+    out = dev(np.zeros((1, 32), dtype=np.float32))
+    nb = L.str_mamba_importance_dynamic_workspace_size(ctypes.byref(s), 32, 8)
+    ws = ctx.workspace(nb)
+    args = lambda n_vis, n_text, ws_bytes: (ctx.handle, ctypes.byref(s), n_vis, n_text, binding._p(B), binding._p(C), binding._p(dt),
+                                            binding._p(A), binding._p(out), binding._p(ws), ctypes.c_size_t(ws_bytes), binding._stream())
+    assert L.str_mamba_importance_dynamic(*args(32, 8, nb)) == 0
+    assert L.str_mamba_importance_dynamic(*args(30, 8, nb)) == -1            # n_vis + n_text != T
+    assert L.str_mamba_importance_dynamic(*args(32, 8, 16)) == -3            # workspace too small
+    x = inputs.attn_score_inputs(36, 40, 4, 2, 128, "bf16")
+    q, k = dev(x["q"], "bf16"), dev(x["k"], "bf16")
+    with pytest.raises(KeyError):
+        binding.str_attn_importance(ctx, q, k, 32, 8, 0.1, denominator="rows")
+    sa = binding.AttnScoreShape(1, 40, 4, 2, 128, binding.STR_BF16)
+    nb = L.str_attn_importance_workspace_size(ctypes.byref(sa), 32, 8)
+    ws = ctx.workspace(nb)
+    rc = L.str_attn_importance_ex(ctx.handle, ctypes.byref(sa), 32, 8, binding._p(q), binding._p(k), ctypes.c_float(0.1), 7,
+                                  binding._p(out), binding._p(ws), ctypes.c_size_t(nb), binding._stream())
+    assert rc == -1                                                            # unknown normaliser
+    ctx.check_status()
+    # zero visual tokens: nothing to score, nothing written
+    assert binding.str_mamba_importance_dynamic(ctx, B[:, 32:], C[:, 32:], dt[:, 32:], A, 0, 8).shape == (1, 0)
