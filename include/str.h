@@ -146,7 +146,10 @@ int str_attn_importance_static(str_ctx *ctx, const str_attn_score_shape *s, int 
  * lower index is kept.  Radix select on the order-preserving integer image of fp32.
  *   scores device [Bz,n_vis] fp32 (any finite values; NaN unsupported),
  *   kept_idx_out device [Bz,k] int32.  k == n_vis gives 0..n_vis-1; k == 0 writes nothing;
- *   k > n_vis or k < 0 -> INVALID_ARG. */
+ *   k > n_vis or k < 0 -> INVALID_ARG.
+ * Workspace: none for rows of up to 131072 scores.  Longer rows are split over many CTAs that meet in the
+ * workspace (256-byte aligned, size from the query); without it they are still selected correctly, by one
+ * CTA per row that re-reads the row on every pass. */
 size_t str_topk_select_workspace_size(int Bz, int n_vis, int k);
 int str_topk_select(str_ctx *ctx, int Bz, int n_vis, int k, const float *scores,
                     int32_t *kept_idx_out, void *workspace, size_t workspace_bytes, void *stream);

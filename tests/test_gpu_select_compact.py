@@ -29,6 +29,22 @@ def test_topk_matches_full_sort(ctx, kind, n, k):
         assert np.array_equal(got[b], oracle.topk_select(s[b], k)), (kind, n, k, b)
 
 
+@pytest.mark.parametrize("kind", ["uniform", "ties", "equal", "descending"])
+@pytest.mark.parametrize("n,k,Bz", [(131073, 1000, 1), (200000, 100000, 2), (1048576, 262144, 1), (300001, 300000, 1)])
+def test_topk_long_rows_split_over_many_ctas(ctx, kind, n, k, Bz):
+    s = inputs.score_vectors(13, n, kind, batch=Bz)
+    got = binding.str_topk_select(ctx, dev(s), k).cpu().numpy()
+    for b in range(Bz):
+        assert np.array_equal(got[b], oracle.topk_select(s[b], k)), (kind, n, k, b)
+    if kind == "ties" and Bz == 1:
+        # without a workspace the same rows take the one-CTA kernel: same answer
+        import ctypes
+        out = dev(np.zeros((Bz, k), dtype=np.int32))
+        rc = binding.lib().str_topk_select(ctx.handle, Bz, n, k, binding._p(dev(s)), binding._p(out), None, ctypes.c_size_t(0),
+                                           binding._stream())
+        assert rc == 0 and np.array_equal(out.cpu().numpy(), got)
+
+
 def test_topk_edge_budgets(ctx):
     s = inputs.score_vectors(12, 777, "uniform", batch=3)
     full = binding.str_topk_select(ctx, dev(s), 777).cpu().numpy()
