@@ -269,6 +269,29 @@ int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const void *hidden_
                       void *hidden_out, int32_t *positions_out, int32_t *idx_map_out,
                       int32_t *kept_trace, float *scores_trace, void *workspace,
                       size_t workspace_bytes, void *stream);
+/* Optional inputs and outputs of the stack, for callers that continue from a reduced context or hand the result to
+ * a decoder (Section 2 "stateful compression": the tokens a Mamba layer drops stay absorbed in its state; later steps
+ * run on the kept set).  Every pointer is a device pointer owned by the caller and may be NULL.
+ *   positions_in / idx_map_in [Bz, n_vis+n_text] int32: original token ids of the incoming rows (strictly ascending per
+ *     sequence); NULL means 0 .. n_vis+n_text-1.  positions_in feeds the rotary embedding, idx_map_in is carried
+ *     through the compactions into idx_map_out.
+ *   mamba_final_states: for each Mamba layer, in layer order, the recurrent state after the last incoming token,
+ *     [Bz,H,p,n] fp32, packed one after the other.
+ *   attn_k_out / attn_v_out: for each attention layer, in layer order, the post-RoPE keys / the values of the rows that
+ *     LEAVE the layer (the kept visual rows, then the text rows), [Bz, K_l+n_text, Hkv, d] dtype, packed one after the
+ *     other; attn_pos_out likewise [Bz, K_l+n_text] int32 holds their original positions. */
+typedef struct {
+    const int32_t *positions_in;
+    const int32_t *idx_map_in;
+    float *mamba_final_states;
+    void *attn_k_out;
+    void *attn_v_out;
+    int32_t *attn_pos_out;
+} str_stack_io;
+/* str_stack_prefill with the optional inputs / outputs above (io == NULL: exactly str_stack_prefill). */
+int str_stack_prefill_ex(str_ctx *ctx, const str_stack_desc *d, const str_stack_io *io, const void *hidden_in,
+                         void *hidden_out, int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace,
+                         float *scores_trace, void *workspace, size_t workspace_bytes, void *stream);
 /* Same, with HOST hidden_in / hidden_out / idx_map_out buffers (pinned memory recommended):
  * copies the input to the device, runs the stack, copies the results back, and synchronises
  * `stream` before returning.  The device staging area is part of the workspace

@@ -411,11 +411,11 @@ def mamba2_block(u, prm, rnd=_identity):
     Bm = xBC[:, d_inner:d_inner + G * n].reshape(T, G, n)
     Cm = xBC[:, d_inner + G * n:].reshape(T, G, n)
     dt = softplus(dt_raw + _f64(prm["dt_bias"])[None, :])
-    y, _ = mamba2_recurrence(x, dt, prm["A"], Bm, Cm)
+    y, final_state = mamba2_recurrence(x, dt, prm["A"], Bm, Cm)
     y = rnd(y)
     gated = rnd(rmsnorm(y.reshape(T, d_inner) * silu(z)))
     out = rnd(u + gated @ _f64(prm["W_out"]))
-    return out, dict(x=x, B=Bm, C=Cm, dt=dt, y=y)
+    return out, dict(x=x, B=Bm, C=Cm, dt=dt, y=y, final_state=final_state)
 
 
 def attn_block(u, positions, prm, rnd=_identity):
@@ -448,7 +448,8 @@ def ffn_block(u, prm, rnd=_identity):
     return rnd(u + act @ _f64(prm["W_down"]))
 
 
-def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_score="decoupled", attn_denominator="visual"):
+def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_score="decoupled", attn_denominator="visual",
+                  positions=None, idx_map=None, keep_inputs=False):
     """Token-reduced prefill of a layer stack (one sequence).
 
     hidden [T0,D] with the n_text text rows last; layers: list of ("M"|"A"|"F", prm);
@@ -456,19 +457,24 @@ def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_scor
     tokens, its own score ranks the incoming visual tokens, and its OUTPUT is compacted when
     keep_counts[l] < n_cur.  Returns (hidden, positions, idx_map, trace) where trace lists per
     layer dict(n_in, scores or None, kept or None).  ``mamba_score``: "decoupled" (Eq. 2, the method) or
-    "full_dynamic" (|w| of Eq. 1, the paper's scoring ablation); ``attn_denominator`` as in attn_importance."""
+    "full_dynamic" (|w| of Eq. 1, the paper's scoring ablation); ``attn_denominator`` as in attn_importance.
+    ``positions`` / ``idx_map``: original token ids of the incoming rows (default 0..T0-1), for continuing from a
+    reduced context.  Every trace record also carries what a decoder would take over from the layer: the final
+    recurrent state of a Mamba layer, the keys / values / positions of the rows leaving an attention layer; with
+    ``keep_inputs`` it carries the layer's input (hidden, positions, idx_map) as well, for teacher-forced tests."""
     assert mamba_score in ("decoupled", "full_dynamic")
     h = _f64(hidden)
     T0 = h.shape[0]
     n_cur = T0 - n_text
-    pos = np.arange(T0, dtype=np.int32)
-    idx = np.arange(T0, dtype=np.int32)
+    pos = np.arange(T0, dtype=np.int32) if positions is None else np.asarray(positions, dtype=np.int32).copy()
+    idx = np.arange(T0, dtype=np.int32) if idx_map is None else np.asarray(idx_map, dtype=np.int32).copy()
     trace = []
     for (kind, prm), K in zip(layers, keep_counts):
+        inputs = dict(hidden_in=h.copy(), positions_in=pos.copy(), idx_map_in=idx.copy()) if keep_inputs else {}
         if kind == "F":                                   # FFN layers transform the rows they get; they never score
             assert K == n_cur
             h = ffn_block(h, prm, rnd)
-            trace.append(dict(n_in=n_cur, scores=None, kept=None))
+            trace.append(dict(n_in=n_cur, scores=None, kept=None, **inputs))
             continue
         if kind == "M":
             out, mid = mamba2_block(h, prm, rnd)
@@ -479,13 +485,19 @@ def stack_prefill(hidden, n_text, layers, keep_counts, rnd=_identity, mamba_scor
         else:
             out, mid = attn_block(h, pos, prm, rnd)
             score = (lambda: attn_importance(mid["q"], mid["k"], n_cur, n_text, mid["scale"], attn_denominator))
-        rec = dict(n_in=n_cur, scores=None, kept=None)
+        rec = dict(n_in=n_cur, scores=None, kept=None, **inputs)
+        rows_out = np.arange(n_cur + n_text)
         if K < n_cur:
             s = score()
             kept = topk_select(s, K)
+            rows_out = np.concatenate([kept.astype(np.int64), np.arange(n_cur, n_cur + n_text)])
             out, pos, idx = compact(out, pos, idx, kept, n_text)
             rec.update(scores=s, kept=kept)
             n_cur = K
+        if kind == "M":
+            rec.update(final_state=mid["final_state"])
+        else:
+            rec.update(k=mid["k"][rows_out], v=mid["v"][rows_out], kv_positions=pos.copy())
         h = out
         trace.append(rec)
     return h, pos, idx, trace

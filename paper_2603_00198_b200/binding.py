@@ -54,6 +54,11 @@ class StackDesc(ctypes.Structure):
                    ("ffn_dim", c_int)])
 
 
+class StackIO(ctypes.Structure):
+    _fields_ = [("positions_in", c_void_p), ("idx_map_in", c_void_p), ("mamba_final_states", c_void_p),
+                ("attn_k_out", c_void_p), ("attn_v_out", c_void_p), ("attn_pos_out", c_void_p)]
+
+
 PROF_CATEGORIES = ["gemm", "ssd_scan", "mamba_score", "attn_score", "topk", "compact", "attn_fwd", "elementwise"]
 
 EXPORTS = [
@@ -67,7 +72,7 @@ EXPORTS = [
     "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
     "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_relu_squared", "str_mamba_conv_split", "str_gated_rmsnorm",
     "str_rope_split", "str_attn_prefill_workspace_size", "str_attn_prefill",
-    "str_stack_workspace_size", "str_stack_prefill", "str_stack_host_workspace_size",
+    "str_stack_workspace_size", "str_stack_prefill", "str_stack_prefill_ex", "str_stack_host_workspace_size",
     "str_stack_prefill_host",
 ]
 
@@ -440,6 +445,51 @@ def str_stack_prefill(stack, hidden_in, want_trace=False):
         ko += stack.Bz * K
         so += stack.Bz * n_in
     return out, pos, idx, trace
+
+
+def str_stack_prefill_ex(stack, hidden_in, positions_in=None, idx_map_in=None, want_handoff=False):
+    """str_stack_prefill with the optional inputs (original token ids of the incoming rows) and, with
+    ``want_handoff``, the decoder hand-off outputs: the final state of every Mamba layer and the keys, values and
+    positions of the rows leaving every attention layer.  Returns a dict."""
+    ctx = stack.ctx
+    T_out = stack.K_last + stack.n_text
+    out = torch.empty((stack.Bz, T_out, stack.D), dtype=stack.tdt, device=stack.dev)
+    pos = torch.empty((stack.Bz, T_out), dtype=torch.int32, device=stack.dev)
+    idx = torch.empty((stack.Bz, T_out), dtype=torch.int32, device=stack.dev)
+    d = stack.desc
+    kinds = [stack._layers[i].kind for i in range(d.n_layers)]
+    states, ks, vs, kvpos = [], [], [], []
+    fs_all = k_all = v_all = p_all = None
+    if want_handoff:
+        n_m = sum(1 for k in kinds if k == STR_LAYER_MAMBA)
+        rows_a = [stack.Bz * (stack.keep_counts[l] + stack.n_text) for l, k in enumerate(kinds) if k == STR_LAYER_ATTN]
+        if n_m:
+            fs_all = torch.empty((n_m, stack.Bz, d.H, d.p, d.n), dtype=torch.float32, device=stack.dev)
+        if rows_a:
+            k_all = torch.empty((sum(rows_a), d.Hkv, d.d), dtype=stack.tdt, device=stack.dev)
+            v_all = torch.empty_like(k_all)
+            p_all = torch.empty((sum(rows_a),), dtype=torch.int32, device=stack.dev)
+    io = StackIO(_p(positions_in), _p(idx_map_in), _p(fs_all), _p(k_all), _p(v_all), _p(p_all))
+    ws = ctx.workspace(stack.ws_bytes)
+    _check(lib().str_stack_prefill_ex(ctx.handle, ctypes.byref(stack.desc), ctypes.byref(io), _p(hidden_in), _p(out), _p(pos),
+                                      _p(idx), _p(None), _p(None), _p(ws), c_size_t(ws.numel()), _stream()),
+           "str_stack_prefill_ex")
+    res = dict(hidden=out, positions=pos, idx_map=idx)
+    if want_handoff:
+        mi, ro = 0, 0
+        for l, k in enumerate(kinds):
+            if k == STR_LAYER_MAMBA:
+                states.append((l, fs_all[mi]))
+                mi += 1
+            elif k == STR_LAYER_ATTN:
+                n = stack.Bz * (stack.keep_counts[l] + stack.n_text)
+                shp = (stack.Bz, stack.keep_counts[l] + stack.n_text)
+                ks.append((l, k_all[ro:ro + n].view(*shp, d.Hkv, d.d)))
+                vs.append((l, v_all[ro:ro + n].view(*shp, d.Hkv, d.d)))
+                kvpos.append((l, p_all[ro:ro + n].view(*shp)))
+                ro += n
+        res.update(mamba_final_states=states, attn_k=ks, attn_v=vs, attn_pos=kvpos)
+    return res
 
 
 def str_stack_prefill_host(stack, hidden_in_host, hidden_out_host, idx_out_host):

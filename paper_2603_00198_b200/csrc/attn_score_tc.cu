@@ -55,7 +55,7 @@ attn_rowstats_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         if (threadIdx.x == 0) atomicCAS(status, 0, STR_ERR_CUDA);
         return;
     }
-    if (*(volatile int *)status != 0) return;
+    if (tc::cta_should_leave(status)) return;     // an earlier CTA failed: the whole CTA leaves at once
     if (threadIdx.x == 0) {
         tc::mbar_init(bars + B_Q, 1);
         for (int s = 0; s < 2; ++s) {
@@ -227,7 +227,7 @@ attn_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         if (threadIdx.x == 0) atomicCAS(status, 0, STR_ERR_CUDA);
         return;
     }
-    if (*(volatile int *)status != 0) return;
+    if (tc::cta_should_leave(status)) return;     // an earlier CTA failed: the whole CTA leaves at once
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) { tc::mbar_init(bars + B_FULL0 + s, 1); tc::mbar_init(bars + B_EMPTY0 + s, 1); }
         for (int s = 0; s < 2; ++s) {

@@ -56,7 +56,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         return;
     }
     // once any CTA has recorded an error the rest of the grid leaves at once
-    if (*(volatile int *)status != 0) return;
+    if (tc::cta_should_leave(status)) return;     // an earlier CTA failed: the whole CTA leaves at once
     if (threadIdx.x == 0) {
         tc::mbar_init(bars + B_Q, 1);
         for (int s = 0; s < 2; ++s) {
@@ -117,25 +117,23 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // One elected thread runs the loop and issues each product as one block of eight tcgen05.mma (see
+        // tc_common.cuh: issued statement by statement the products lose the issue slot to the softmax warps).
+        if (tc::elect_one()) {
             const uint32_t id_s = tc::make_idesc_bf16(BQ, BKV, 0, 0);     // Q (K-major) x K (K-major)
             const uint32_t id_o = tc::make_idesc_bf16(BQ, HD, 0, 1);      // P (tensor memory) x V (MN-major)
             const uint32_t sbase = tc::smem_u32(smem);
             auto issue_s = [&](int i, int slot) {
                 const uint32_t qa = sbase + OFF_Q + (uint32_t)i * 2 * TILE_16K;
                 const uint32_t ka = sbase + OFF_K + (uint32_t)slot * 2 * TILE_16K;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    tc::mma_ss(tmem + TM_S + (uint32_t)i * 128, tc::desc_kmajor_sw128(qa + (ks >> 2) * TILE_16K, (ks & 3) * 16),
-                               tc::desc_kmajor_sw128(ka + (ks >> 2) * TILE_16K, (ks & 3) * 16), id_s, ks != 0);
+                tc::mma8_ss<tc::StepKMajor2x64, tc::StepKMajor2x64>(tmem + TM_S + (uint32_t)i * 128, tc::desc_kmajor_sw128(qa, 0),
+                                                                    tc::desc_kmajor_sw128(ka, 0), id_s, false);
                 tc::mma_commit(bars + B_SF0 + i);
             };
             auto issue_pv = [&](int i, int slot, bool first) {
                 const uint32_t va = sbase + OFF_V + (uint32_t)slot * 2 * TILE_16K;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    tc::mma_ts(tmem + TM_O + (uint32_t)i * 128, tmem + TM_S + (uint32_t)i * 128 + (uint32_t)ks * 8,
-                               tc::make_smem_desc(va + ks * 2048, TILE_16K, 1024, tc::SWZ_128B), id_o, !(first && ks == 0));
+                tc::mma8_ts<tc::StepTmem8, tc::StepMNMajor>(tmem + TM_O + (uint32_t)i * 128, tmem + TM_S + (uint32_t)i * 128,
+                                                            tc::make_smem_desc(va, TILE_16K, 1024, tc::SWZ_128B), id_o, !first);
             };
             bool ok = tc::mbar_wait(bars + B_Q, 0, abort_flag) && tc::mbar_wait(bars + B_KF0, 0, abort_flag);
             if (ok) {
@@ -173,6 +171,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             }
             if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         }
+        __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax warps
         const int i = warp >> 2, quad = warp & 3;

@@ -86,7 +86,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        // one elected thread for the whole loop; each 64-column stage is one block of four tcgen05.mma
+        if (tc::elect_one()) {
             const uint32_t idesc = tc::make_idesc_bf16(BM, BN, 0, 0);
             int it = 0, local = 0;
             bool ok = true;
@@ -102,16 +103,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     if (!tc::mbar_wait(full + s, ph, abort_flag)) { ok = false; break; }
                     tc::tc_fence_after();
                     const uint32_t sa = tc::smem_u32(smem + (size_t)s * STAGE_BYTES);
-#pragma unroll
-                    for (int kk = 0; kk < BK / UMMA_K; ++kk)
-                        tc::mma_ss(d_tmem, tc::desc_kmajor_sw128(sa, kk * UMMA_K),
-                                   tc::desc_kmajor_sw128(sa + A_BYTES, kk * UMMA_K), idesc, (kb | kk) != 0);
+                    static_assert(BK / UMMA_K == 4, "one stage is four K-slices");
+                    tc::mma4_ss<tc::StepKMajor64, tc::StepKMajor64>(d_tmem, tc::desc_kmajor_sw128(sa, 0),
+                                                                    tc::desc_kmajor_sw128(sa + A_BYTES, 0), idesc, kb != 0);
                     tc::mma_commit(empty + s);
                 }
                 if (ok) tc::mma_commit(acc_full + acc);
             }
             if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         }
+        __syncwarp();
     } else {
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
         int local = 0;

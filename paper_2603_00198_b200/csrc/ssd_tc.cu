@@ -18,42 +18,22 @@
 // The chunk loop is software-pipelined across warp roles that only meet at mbarriers; the only
 // serial chains from chunk to chunk are  dS_c -> state update -> Y_inter_{c+1}  and
 // dS_c -> Xs_{c+1} -> dS_{c+1}  (single Xs buffer):
-//   warps 0-3, 14, 15  W_c from CB_c (one thread per token row and 64-column half; the upper halves of
-//                      row blocks 0 and 1 are all zero and are written by warps 0 and 1)
-//   warps 4-7          state update (one thread per state row n, 64 fp32 registers of state), then half of Xs_{c+1};
+//   warps 0-3, 14, 15  W_c from CB_c in 16-column pieces of a 32-row quadrant (one thread per token row)
+//   warps 4-7          state update (one thread per state row n, 64 fp32 registers of state);
 //                      lane 0 of warp 4 is the TMA producer (B,C ring of 2, X ring of 3, 128-byte swizzle): seeing
 //                      dS_c complete is what frees the slots of chunk c+2, so there are no slot-release barriers
-//   warps 8-11         the other half of Xs_{c+1}, then the epilogue of chunk c (one thread per token row)
+//   warps 8-11         Xs_{c+1}, then the epilogue of chunk c (one thread per token row)
 //   warp 12            the decay vectors of each chunk (cumulative sum, exponentials) into a ring of 4; depends on
 //                      dt only and runs up to three chunks ahead of its readers
-//   warp 13            MMA issuer; iteration c issues  CB_c, Y_intra_{c-1}, Y_inter_c, dS_c
+//   warp 13            MMA issuer (one elected thread); iteration c issues  CB_c, Y_intra_{c-1}, Y_inter_c, dS_c
 // Loops are kept rolled where registers allow: the instruction footprint of all roles together has to
 // stay inside the instruction cache, or every role slows down together.
-// Tensor memory: CB/W 2 x 128 columns | Y_inter 2 x 64 | Y_intra 64 | dS 64.  W's K-slices 0-3 (keys
-// 0-63) sit in columns [0,32) of the CB buffer and K-slices 4-7 in columns [64,96), so each W warp
-// only overwrites accumulator columns that it has read itself.
+// Tensor memory: CB/W 2 x 128 columns | Y_inter 2 x 64 | Y_intra 64 | dS 64.  W's K-slice ks (keys
+// 16 ks .. 16 ks + 15) sits in columns [16 ks, 16 ks + 8) of the CB buffer it was computed from, so a
+// thread only overwrites accumulator columns that it has read itself.
 // All mbarrier waits are bounded; a give-up records STR_ERR_TIMEOUT and tears the CTA down.
 #include "dispatch.cuh"
 #include "tc_common.cuh"
-
-// Optional device-side timeline (compile with -DSTR_SSD_TRACE): lane 0 of selected warps of one CTA
-// stores the SM clock at a few points of chunks 16..31.  Compiled out of the library build.
-#ifdef STR_SSD_TRACE
-#ifndef STR_SSD_TRACE_QUAD
-#define STR_SSD_TRACE_QUAD 0
-#endif
-__device__ long long g_ssd_trace[8 * 16 * 8];
-#define SSD_TR(role, c, pt)                                                                              \
-    do {                                                                                                 \
-        if (blockIdx.x == 5 && blockIdx.y == 0 && (c) >= 16 && (c) < 32 && lane == 0)                    \
-            g_ssd_trace[((role) * 16 + ((c) - 16)) * 8 + (pt)] = clock64();                              \
-    } while (0)
-extern "C" int str_ssd_trace_fetch(long long *host) { return (int)cudaMemcpyFromSymbol(host, g_ssd_trace, sizeof(g_ssd_trace)); }
-#define SSD_TRQ STR_SSD_TRACE_QUAD
-#else
-#define SSD_TR(role, c, pt) do { } while (0)
-#define SSD_TRQ 0
-#endif
 
 namespace {
 
@@ -67,8 +47,8 @@ constexpr int OFF_XS = OFF_C + 4 * TILE_16K;              // 16 KB
 constexpr int OFF_SB = OFF_XS + TILE_16K;                 // 16 KB
 constexpr int OFF_DEC = OFF_SB + TILE_16K;                // 4 x 3200 B
 constexpr int OFF_BARS = OFF_DEC + DEC_DEPTH * DEC_FLOATS * 4;
-// decay vectors of one chunk (floats): log2-domain cumulative decay, dt, column / state / row factors
-constexpr int D_LS = 0, D_DT = 128, D_COLF = 256, D_XW = 384, D_ROWF = 512, D_EROW = 640, D_BLK = 768, D_EEND = 784;
+// decay vectors of one chunk (floats): log2-domain cumulative decay l_j, log2(dt_j) - l_j, column / state / row factors
+constexpr int D_LS = 0, D_NLC = 128, D_COLF = 256, D_XW = 384, D_ROWF = 512, D_EROW = 640, D_BLK = 768, D_EEND = 784;
 enum {
     B_XF = 0, B_BCF = 3, B_DECF = 5, B_DECE = 9, B_CBF = 13, B_WF = 15, B_XSF = 17, B_DSF, B_DSE,
     B_SF, B_YF, B_YE, B_COUNT
@@ -85,32 +65,55 @@ __device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane) {
     if (lane == 0) tc::mbar_arrive(bar);
 }
 
-// Whole-warp wait: every lane polls, then the lanes agree on the outcome.
-__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile int *abort) {
-    return __all_sync(0xffffffffu, tc::mbar_wait(bar, parity, abort));
-}
-
 // Descriptor arithmetic: the 14-bit start-address field holds (shared address >> 4); every operand of
 // this kernel lies below 256 KB, so adding a byte offset >> 4 to the descriptor never carries out of it.
 __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
-// Byte offset of K-slice ks (16 elements) inside a K-major operand stored as two 64-column, 16 KB halves.
-__device__ __forceinline__ uint32_t kmajor_off(int ks) { return (uint32_t)(ks >> 2) * TILE_16K + (uint32_t)(ks & 3) * 32; }
-
-// Half of Xs_c = exp(l_end - l_j) dt_j x_j (same swizzled layout as the X tile): 128 threads, four 16-byte
-// units each; `part` 0 and 1 are done by two different warp groups.
-__device__ __forceinline__ void scale_x_half(const uint8_t *x_tile, uint8_t *xs_tile, const float *dec_xw, int tid_g, int part) {
+// Xs_c = exp(l_end - l_j) dt_j x_j (same swizzled layout as the X tile): 128 threads, eight 16-byte units each.
+// The row factor is narrowed to bf16 and applied with packed bf16 multiplies (one instruction per two elements).
+__device__ __forceinline__ void scale_x(const uint8_t *x_tile, uint8_t *xs_tile, const float *dec_xw, int tid_g) {
     const uint4 *src = (const uint4 *)x_tile;
     uint4 *dst = (uint4 *)xs_tile;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int u = tid_g + 128 * (4 * part + i);
-        const float sc = dec_xw[u >> 3];
-        const uint4 v = src[u];
-        uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+    for (int i = 0; i < 8; ++i) {
+        const int u = tid_g + 128 * i;
+        const __nv_bfloat162 sc = __float2bfloat162_rn(dec_xw[u >> 3]);
+        uint4 v = src[u];
+        __nv_bfloat162 *pv = reinterpret_cast<__nv_bfloat162 *>(&v);
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            wv[j] = tc::pack_bf16x2(__uint_as_float(wv[j] << 16) * sc, __uint_as_float(wv[j] & 0xFFFF0000u) * sc);
-        dst[u] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+        for (int j = 0; j < 4; ++j) pv[j] = __hmul2(pv[j], sc);
+        dst[u] = v;
+    }
+}
+
+// One 16-column piece of W = CB o decay for this thread's token row: fp32 CB values in, eight packed bf16 pairs out.
+// Diagonal 32x32 block: one exponential per element, exp2(l_t + (log2 dt_j - l_j)), masked above the diagonal.
+__device__ __forceinline__ void w_piece_diag(const uint32_t (&v)[16], uint32_t (&packed)[8], const float *dec, int col0, int row, float l_t) {
+    const float2 lt2 = make_float2(l_t, l_t);
+#pragma unroll
+    for (int i4 = 0; i4 < 4; ++i4) {
+        const float4 nl = *(const float4 *)(dec + D_NLC + col0 + 4 * i4);
+        const int j0 = col0 + 4 * i4;
+        const float2 a01 = __fadd2_rn(lt2, make_float2(nl.x, nl.y)), a23 = __fadd2_rn(lt2, make_float2(nl.z, nl.w));
+        const float f0 = (j0 <= row) ? tc::ex2(a01.x) : 0.f;
+        const float f1 = (j0 + 1 <= row) ? tc::ex2(a01.y) : 0.f;
+        const float f2 = (j0 + 2 <= row) ? tc::ex2(a23.x) : 0.f;
+        const float f3 = (j0 + 3 <= row) ? tc::ex2(a23.y) : 0.f;
+        const float2 r01 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i4]), __uint_as_float(v[4 * i4 + 1])), make_float2(f0, f1));
+        const float2 r23 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i4 + 2]), __uint_as_float(v[4 * i4 + 3])), make_float2(f2, f3));
+        packed[2 * i4] = tc::pack_bf16x2(r01.x, r01.y);
+        packed[2 * i4 + 1] = tc::pack_bf16x2(r23.x, r23.y);
+    }
+}
+// Block below the diagonal: exp(l_t - l_j) dt_j = f (row part times block-pair scalar) * column part, each <= 1.
+__device__ __forceinline__ void w_piece_below(const uint32_t (&v)[16], uint32_t (&packed)[8], const float *dec, int col0, float f) {
+    const float2 ff = make_float2(f, f);
+#pragma unroll
+    for (int i4 = 0; i4 < 4; ++i4) {
+        const float4 cf = *(const float4 *)(dec + D_COLF + col0 + 4 * i4);
+        const float2 r01 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i4]), __uint_as_float(v[4 * i4 + 1])), __fmul2_rn(ff, make_float2(cf.x, cf.y)));
+        const float2 r23 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i4 + 2]), __uint_as_float(v[4 * i4 + 3])), __fmul2_rn(ff, make_float2(cf.z, cf.w)));
+        packed[2 * i4] = tc::pack_bf16x2(r01.x, r01.y);
+        packed[2 * i4 + 1] = tc::pack_bf16x2(r23.x, r23.y);
     }
 }
 
@@ -137,7 +140,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (threadIdx.x == 0) atomicCAS(status, 0, STR_ERR_CUDA);
         return;
     }
-    if (*(volatile int *)status != 0) return;         // an earlier CTA failed: leave at once
+    if (tc::cta_should_leave(status)) return;     // an earlier CTA failed: the whole CTA leaves at once
     if (threadIdx.x == 0) {
         for (int i = 0; i < X_SLOTS; ++i) tc::mbar_init(bars + B_XF + i, 1);
         for (int i = 0; i < 2; ++i) {
@@ -145,7 +148,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             tc::mbar_init(bars + B_CBF + i, 1); tc::mbar_init(bars + B_WF + i, W_WARPS);
         }
         for (int i = 0; i < DEC_DEPTH; ++i) { tc::mbar_init(bars + B_DECF + i, 1); tc::mbar_init(bars + B_DECE + i, DEC_READERS); }
-        tc::mbar_init(bars + B_XSF, 8); tc::mbar_init(bars + B_DSF, 1); tc::mbar_init(bars + B_DSE, 4);
+        tc::mbar_init(bars + B_XSF, 4); tc::mbar_init(bars + B_DSF, 1); tc::mbar_init(bars + B_DSE, 4);
         tc::mbar_init(bars + B_SF, 4); tc::mbar_init(bars + B_YF, 1); tc::mbar_init(bars + B_YE, 4);
         abort_flag[0] = 0; abort_flag[1] = 0;
         tc::fence_mbar_init();
@@ -175,7 +178,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 dn[i] = t < Tlen ? __ldg(dtb + (size_t)t * H) : 0.f;
             }
             if (!tc::mbar_wait(bars + B_DECE + d, ((c >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
-            SSD_TR(0, c, 2);
             float l[4];
             l[0] = dv[0] * Ah2;
 #pragma unroll
@@ -187,7 +189,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (lane >= o) incl += v;
             }
             const float excl = incl - l[3];
-            SSD_TR(0, c, 4);
             const float l_start = __shfl_sync(0xffffffffu, excl, lane & ~7);     // start of this 32-token block
             const float l_endb = __shfl_sync(0xffffffffu, incl, lane | 7);       // end of this 32-token block
             const float l_end = __shfl_sync(0xffffffffu, incl, 31);
@@ -195,185 +196,138 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const float bs = __shfl_sync(0xffffffffu, excl, ((lane >> 2) & 3) * 8);
             const float be = __shfl_sync(0xffffffffu, incl, (lane & 3) * 8 + 7);
             float *dec = decs + d * DEC_FLOATS;
-            float o_ls[4], o_colf[4], o_xw[4], o_rowf[4], o_erow[4];
+            float o_ls[4], o_nlc[4], o_colf[4], o_xw[4], o_rowf[4], o_erow[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const float li = excl + l[i];
                 o_ls[i] = li;
+                o_nlc[i] = tc::lg2(dv[i]) - li;          // exp2(l_t + nlc_j) = exp(l_t - l_j) dt_j; a padded token (dt = 0) gives -inf
                 o_colf[i] = tc::ex2(l_endb - li) * dv[i];
                 o_xw[i] = tc::ex2(l_end - li) * dv[i];
                 o_rowf[i] = tc::ex2(li - l_start);
                 o_erow[i] = tc::ex2(li);
             }
-            SSD_TR(0, c, 5);
             *(float4 *)(dec + D_LS + 4 * lane) = make_float4(o_ls[0], o_ls[1], o_ls[2], o_ls[3]);
-            *(float4 *)(dec + D_DT + 4 * lane) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+            *(float4 *)(dec + D_NLC + 4 * lane) = make_float4(o_nlc[0], o_nlc[1], o_nlc[2], o_nlc[3]);
             *(float4 *)(dec + D_COLF + 4 * lane) = make_float4(o_colf[0], o_colf[1], o_colf[2], o_colf[3]);
             *(float4 *)(dec + D_XW + 4 * lane) = make_float4(o_xw[0], o_xw[1], o_xw[2], o_xw[3]);
             *(float4 *)(dec + D_ROWF + 4 * lane) = make_float4(o_rowf[0], o_rowf[1], o_rowf[2], o_rowf[3]);
             *(float4 *)(dec + D_EROW + 4 * lane) = make_float4(o_erow[0], o_erow[1], o_erow[2], o_erow[3]);
             if (lane < 16) dec[D_BLK + lane] = ((lane & 3) < (lane >> 2)) ? tc::ex2(bs - be) : 0.f;
             if (lane == 0) dec[D_EEND] = tc::ex2(l_end);
-            SSD_TR(0, c, 6);
             warp_arrive(bars + B_DECF + d, lane);
-            SSD_TR(0, c, 3);
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
     } else if (warp == 13) {
         // ------------------------------------------------------------------ MMA issuer
-        // The whole warp runs the loop (so descriptors and addresses stay warp-uniform); one elected lane
-        // issues.  Product order per iteration: CB_c, Y_intra_{c-1}, Y_inter_c, dS_c.
-        const uint32_t id_cb = tc::make_idesc_bf16(128, 128, 0, 0);   // C (K-major) x B (K-major)
-        const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major / tensor-memory A x MN-major B
-        const uint32_t id_nn = tc::make_idesc_bf16(128, 64, 1, 1);    // MN-major A x MN-major B
-        const uint32_t sbase = tc::smem_u32(smem);
-        // descriptors of the first K-slice of every operand; K-slice ks of a K-major operand sits
-        // (ks / 4) * 16 KB + (ks % 4) * 32 bytes further on, of an MN-major operand ks * 2 KB further on
-        const uint64_t dk_c0 = tc::desc_kmajor_sw128(sbase + OFF_C, 0), dk_b0 = tc::desc_kmajor_sw128(sbase + OFF_B, 0);
-        const uint64_t dm_b0 = tc::make_smem_desc(sbase + OFF_B, TILE_16K, 1024, tc::SWZ_128B);
-        const uint64_t dm_xs = tc::make_smem_desc(sbase + OFF_XS, TILE_16K, 1024, tc::SWZ_128B);
-        const uint64_t dm_sb = tc::make_smem_desc(sbase + OFF_SB, TILE_16K, 1024, tc::SWZ_128B);
-        const uint64_t dm_x0 = tc::make_smem_desc(sbase + OFF_X, TILE_16K, 1024, tc::SWZ_128B);
-        bool ok = true;
+        // One elected thread runs the whole loop (the region is entered once, so the compiler knows it to be
+        // single-threaded) and issues every product as one straight-line block of eight tcgen05.mma: issued any
+        // other way the products cost two to five times the tensor pipe's own time as soon as the arithmetic
+        // warps of this scheduler are busy.  Product order per iteration: CB_c, Y_intra_{c-1}, Y_inter_c, dS_c.
+        if (tc::elect_one()) {
+            const uint32_t id_cb = tc::make_idesc_bf16(128, 128, 0, 0);   // C (K-major) x B (K-major)
+            const uint32_t id_kn = tc::make_idesc_bf16(128, 64, 0, 1);    // K-major / tensor-memory A x MN-major B
+            const uint32_t id_nn = tc::make_idesc_bf16(128, 64, 1, 1);    // MN-major A x MN-major B
+            const uint32_t sbase = tc::smem_u32(smem);
+            const uint64_t dk_c0 = tc::desc_kmajor_sw128(sbase + OFF_C, 0), dk_b0 = tc::desc_kmajor_sw128(sbase + OFF_B, 0);
+            const uint64_t dm_b0 = tc::make_smem_desc(sbase + OFF_B, TILE_16K, 1024, tc::SWZ_128B);
+            const uint64_t dm_xs = tc::make_smem_desc(sbase + OFF_XS, TILE_16K, 1024, tc::SWZ_128B);
+            const uint64_t dm_sb = tc::make_smem_desc(sbase + OFF_SB, TILE_16K, 1024, tc::SWZ_128B);
+            const uint64_t dm_x0 = tc::make_smem_desc(sbase + OFF_X, TILE_16K, 1024, tc::SWZ_128B);
+            bool ok = true;
 #pragma unroll 1
-        for (int c = 0; c <= nchunks && ok; ++c) {
-            const int s = c & 1;
-            const uint64_t dk_c = desc_add(dk_c0, (uint32_t)s * 2 * TILE_16K), dk_b = desc_add(dk_b0, (uint32_t)s * 2 * TILE_16K);
-            SSD_TR(1, c, 0);
-            if (c < nchunks) {
-                ok = warp_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag);
-                if (!ok) break;
-                SSD_TR(1, c, 1);
-                tc::tc_fence_after();
-                if (tc::elect_one()) {
-#pragma unroll 1
-                    for (int ks = 0; ks < 8; ++ks)      // CB_c = C B^T
-                        tc::mma_ss(tmem + TM_CB + (uint32_t)s * 128, desc_add(dk_c, kmajor_off(ks)), desc_add(dk_b, kmajor_off(ks)),
-                                   id_cb, ks != 0);
+            for (int c = 0; c <= nchunks && ok; ++c) {
+                const int s = c & 1;
+                const uint64_t dk_c = desc_add(dk_c0, (uint32_t)s * 2 * TILE_16K), dk_b = desc_add(dk_b0, (uint32_t)s * 2 * TILE_16K);
+                if (c < nchunks) {
+                    ok = tc::mbar_wait(bars + B_BCF + s, (c >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    tc::mma8_ss<tc::StepKMajor2x64, tc::StepKMajor2x64>(tmem + TM_CB + (uint32_t)s * 128, dk_c, dk_b, id_cb, false);   // CB_c = C B^T
                     tc::mma_commit(bars + B_CBF + s);
                 }
-                __syncwarp();
-                SSD_TR(1, c, 2);
-            }
-            if (c >= 1) {
-                const int cp = c - 1, sp = cp & 1;
-                // the epilogue has read the Y accumulators of chunk c-2; W_{c-1} is in tensor memory
-                SSD_TR(7, c, 0);
-                ok = c < 2 || warp_wait(bars + B_YE, (c - 2) & 1, abort_flag);
-                SSD_TR(7, c, 1);
-                ok = ok && warp_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag);
-                SSD_TR(7, c, 2);
-                if (!ok) break;
-                SSD_TR(1, c, 3);
-                tc::tc_fence_after();
-                const uint64_t dm_x = desc_add(dm_x0, (uint32_t)(cp % X_SLOTS) * TILE_16K);
-                const uint32_t tW = tmem + TM_CB + (uint32_t)sp * 128;
-                if (tc::elect_one()) {
-#pragma unroll 1
-                    for (int ks = 0; ks < 8; ++ks)      // Y_intra_{c-1} = W X; K-slices 4-7 of W start at column 64
-                        tc::mma_ts(tmem + TM_YI, tW + (uint32_t)((ks >> 2) * 64 + (ks & 3) * 8), desc_add(dm_x, ks * 2048), id_kn,
-                                   ks != 0);
+                if (c >= 1) {
+                    const int cp = c - 1, sp = cp & 1;
+                    // the epilogue has read the Y accumulators of chunk c-2; W_{c-1} is in tensor memory
+                    ok = (c < 2 || tc::mbar_wait(bars + B_YE, (c - 2) & 1, abort_flag)) &&
+                         tc::mbar_wait(bars + B_WF + sp, (cp >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    // Y_intra_{c-1} = W X; K-slice ks of W sits in columns [16 ks, 16 ks + 8)
+                    tc::mma8_ts<tc::StepTmem16, tc::StepMNMajor>(tmem + TM_YI, tmem + TM_CB + (uint32_t)sp * 128,
+                                                                     desc_add(dm_x0, (uint32_t)(cp % X_SLOTS) * TILE_16K), id_kn, false);
                     tc::mma_commit(bars + B_YF);
                 }
-                __syncwarp();
-                SSD_TR(1, c, 4);
-            }
-            if (c < nchunks) {
-                if (c > 0) {
-                    ok = warp_wait(bars + B_SF, (c - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    SSD_TR(1, c, 5);
-                    tc::tc_fence_after();
-                    if (tc::elect_one()) {
-#pragma unroll 1
-                        for (int ks = 0; ks < 8; ++ks)  // Y_inter_c = C S_{c-1}^T
-                            tc::mma_ss(tmem + TM_YO + (uint32_t)s * 64, desc_add(dk_c, kmajor_off(ks)), desc_add(dm_sb, ks * 2048), id_kn,
-                                       ks != 0);
+                if (c < nchunks) {
+                    if (c > 0) {
+                        ok = tc::mbar_wait(bars + B_SF, (c - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc::tc_fence_after();
+                        // Y_inter_c = C S_{c-1}^T
+                        tc::mma8_ss<tc::StepKMajor2x64, tc::StepMNMajor>(tmem + TM_YO + (uint32_t)s * 64, dk_c, dm_sb, id_kn, false);
                     }
-                    __syncwarp();
-                }
-                ok = warp_wait(bars + B_XSF, c & 1, abort_flag) && (c == 0 || warp_wait(bars + B_DSE, (c - 1) & 1, abort_flag));
-                if (!ok) break;
-                SSD_TR(1, c, 6);
-                tc::tc_fence_after();
-                const uint64_t dm_b = desc_add(dm_b0, (uint32_t)s * 2 * TILE_16K);
-                if (tc::elect_one()) {
-#pragma unroll 1
-                    for (int ks = 0; ks < 8; ++ks)      // dS_c^T = B^T Xs
-                        tc::mma_ss(tmem + TM_DS, desc_add(dm_b, ks * 2048), desc_add(dm_xs, ks * 2048), id_nn, ks != 0);
+                    ok = tc::mbar_wait(bars + B_XSF, c & 1, abort_flag) && (c == 0 || tc::mbar_wait(bars + B_DSE, (c - 1) & 1, abort_flag));
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    // dS_c^T = B^T Xs
+                    tc::mma8_ss<tc::StepMNMajor, tc::StepMNMajor>(tmem + TM_DS, desc_add(dm_b0, (uint32_t)s * 2 * TILE_16K), dm_xs, id_nn, false);
                     tc::mma_commit(bars + B_DSF);
                 }
-                __syncwarp();
-                SSD_TR(1, c, 7);
             }
+            if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         }
-        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+        __syncwarp();
     } else if (warp < 4 || warp >= 14) {
         // ------------------------------------------------------------------ W_c = CB_c o decay
+        // Work is dealt out in 16-column pieces of a 32-row quadrant (a warp can only reach the tensor-memory lanes
+        // of its own quadrant); the later row quadrants have more pieces below the diagonal and get two warps:
+        //   quadrant 0: columns 0-31        quadrant 1: 0-63        quadrant 2: 0-63 | 64-95        quadrant 3: 0-79 | 80-127
+        // plus zeros for the pieces above the diagonal.  The bf16 result of piece [16k, 16k+16) goes to the 32-bit
+        // columns [16k, 16k+8) of the same accumulator buffer, i.e. into columns the same thread has just read, so
+        // pieces need no ordering among themselves.
         const int quad = warp & 3, half = warp >= 14 ? 1 : 0;
         const int row = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const int first = half ? (quad == 2 ? 64 : 80) : 0;
+        const int n_real = half ? (quad == 2 ? 2 : 3) : (quad == 0 ? 2 : quad == 1 ? 4 : quad + 2);
+        const int zero_first = half ? 96 : (quad == 0 ? 32 : 64);
+        const int n_zero = half ? (quad == 2 ? 2 : 0) : (quad == 0 ? 6 : quad == 1 ? 4 : 0);
         bool ok = true;
 #pragma unroll 1
         for (int c = 0; c < nchunks; ++c) {
             const int d = c & (DEC_DEPTH - 1), s = c & 1;
             const float *dec = decs + d * DEC_FLOATS;
             if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
-            if (warp == 3) SSD_TR(2, c, 0); else if (warp == 15) SSD_TR(3, c, 0); else if (warp == 0) SSD_TR(4, c, 0);
             const float l_t = dec[D_LS + row], rf = dec[D_ROWF + row];
             if (!tc::mbar_wait(bars + B_CBF + s, (c >> 1) & 1, abort_flag)) { ok = false; break; }
-            if (warp == 3) SSD_TR(2, c, 1); else if (warp == 15) SSD_TR(3, c, 1); else if (warp == 0) SSD_TR(4, c, 1);
             tc::tc_fence_after();
-            const uint32_t tW = tmem + lane_base + TM_CB + (uint32_t)(s * 128 + half * 64);
-            uint32_t v[16], vn[16];
-            tc::tmem_ld16(tW, vn);
-#pragma unroll 1
-            for (int k = 0; k < 4; ++k) {             // 16-column pieces of this warp's 64 columns
-                const int col0 = half * 64 + k * 16, bj = col0 >> 5;
-                tc::tmem_ld_wait();
+            const uint32_t tW = tmem + lane_base + TM_CB + (uint32_t)(s * 128);
+            // every piece is fetched before any is worked on: a tensor-memory load takes a few hundred clocks to
+            // return while the tensor pipe is busy
+            uint32_t v[5][16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = vn[i];
-                if (k < 3) tc::tmem_ld16(tW + (uint32_t)((k + 1) * 16), vn);     // in flight while piece k is worked on
-                uint32_t packed[8];
-                if (bj > quad) {
+            for (int k = 0; k < 5; ++k)
+                if (k < n_real) tc::tmem_ld16(tW + (uint32_t)(first + 16 * k), v[k]);
+            tc::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) packed[i] = 0u;
-                } else if (bj == quad) {
-#pragma unroll
-                    for (int i4 = 0; i4 < 4; ++i4) {
-                        const float4 lj = *(const float4 *)(dec + D_LS + col0 + 4 * i4);
-                        const float4 dj = *(const float4 *)(dec + D_DT + col0 + 4 * i4);
-                        const int j0 = col0 + 4 * i4;
-                        const float f0 = (j0 <= row) ? tc::ex2(l_t - lj.x) * dj.x : 0.f;
-                        const float f1 = (j0 + 1 <= row) ? tc::ex2(l_t - lj.y) * dj.y : 0.f;
-                        const float f2 = (j0 + 2 <= row) ? tc::ex2(l_t - lj.z) * dj.z : 0.f;
-                        const float f3 = (j0 + 3 <= row) ? tc::ex2(l_t - lj.w) * dj.w : 0.f;
-                        packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * f0, __uint_as_float(v[4 * i4 + 1]) * f1);
-                        packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * f2, __uint_as_float(v[4 * i4 + 3]) * f3);
-                    }
-                } else {
-                    const float f = rf * dec[D_BLK + quad * 4 + bj];
-#pragma unroll
-                    for (int i4 = 0; i4 < 4; ++i4) {
-                        const float4 cf = *(const float4 *)(dec + D_COLF + col0 + 4 * i4);
-                        packed[2 * i4] = tc::pack_bf16x2(__uint_as_float(v[4 * i4]) * (f * cf.x), __uint_as_float(v[4 * i4 + 1]) * (f * cf.y));
-                        packed[2 * i4 + 1] = tc::pack_bf16x2(__uint_as_float(v[4 * i4 + 2]) * (f * cf.z), __uint_as_float(v[4 * i4 + 3]) * (f * cf.w));
-                    }
+            for (int k = 0; k < 5; ++k) {
+                if (k < n_real) {
+                    const int col0 = first + 16 * k, bj = col0 >> 5;
+                    uint32_t packed[8];
+                    if (bj == quad) w_piece_diag(v[k], packed, dec, col0, row, l_t);
+                    else w_piece_below(v[k], packed, dec, col0, rf * dec[D_BLK + quad * 4 + bj]);
+                    tc::tmem_st8(tW + (uint32_t)col0, packed);
                 }
-                // the 8 bf16 pairs of piece k go to 32-bit columns [8k, 8k+8) of this half: accumulator columns of
-                // pieces k/2 <= k, in registers by now; the load in flight reads piece k+1, columns >= 16(k+1)
-                tc::tmem_st8(tW + (uint32_t)(k * 8), packed);
             }
-            if (quad < 2) {                           // columns 64..127 of row blocks 0 and 1 lie above the diagonal
-                uint32_t zero[16];
+            if (n_zero > 0) {
+                uint32_t zero[8];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) zero[i] = 0u;
-                tc::tmem_st16(tW + 64, zero);
-                tc::tmem_st16(tW + 80, zero);
+                for (int i = 0; i < 8; ++i) zero[i] = 0u;
+#pragma unroll 1
+                for (int k = 0; k < n_zero; ++k) tc::tmem_st8(tW + (uint32_t)(zero_first + 16 * k), zero);
             }
             tc::tmem_st_wait();
             tc::tc_fence_before();
-            if (warp == 3) SSD_TR(2, c, 2); else if (warp == 15) SSD_TR(3, c, 2); else if (warp == 0) SSD_TR(4, c, 2);
             warp_arrive(bars + B_WF + s, lane);
             if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
         }
@@ -382,23 +336,10 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // ------------------------------------------------------------------ state update
         const int quad = warp & 3, row = quad * 32 + lane;        // row = state index n
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const int tid_s = threadIdx.x - 128;
         float S[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) S[i] = 0.f;
         bool ok = true;
-        // this group's half of Xs_c (the other half is the epilogue group's); chunk 0 before the loop, chunk c+1
-        // right after the state update of chunk c (the Xs buffer is free once dS_c has completed)
-        auto xs_half = [&](int c) -> bool {
-            const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
-            if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) return false;
-            if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) return false;
-            scale_x_half(smem + OFF_X + sx * TILE_16K, smem + OFF_XS, decs + d * DEC_FLOATS + D_XW, tid_s, 0);
-            tc::fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(bars + B_XSF);
-            return true;
-        };
         // Lane 0 of the first state warp is the TMA producer.  The operands of chunk c+2 go into the slots of chunk
         // c (B, C: ring of 2) and chunk c-1 (X: ring of 3) once dS_c is seen complete: the tensor pipe runs in
         // order, so CB_c, Y_inter_c, Y_intra_{c-1} and dS_{c-1} (issued after all of Xs_{c-1} was written, i.e.
@@ -421,7 +362,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             load_chunk(0);
             if (nchunks > 1) load_chunk(1);
         }
-        ok = xs_half(0);
 #pragma unroll 1
         for (int c = 0; c < nchunks && ok; ++c) {
             const int d = c & (DEC_DEPTH - 1);
@@ -429,9 +369,7 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const float eend = decs[d * DEC_FLOATS + D_EEND];
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
-            if (quad == SSD_TRQ) SSD_TR(5, c, 0);
             if (!tc::mbar_wait(bars + B_DSF, c & 1, abort_flag)) { ok = false; break; }
-            if (quad == SSD_TRQ) SSD_TR(5, c, 1);
             tc::tc_fence_after();
             uint8_t *srow = smem + OFF_SB + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
@@ -444,7 +382,12 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     warp_arrive(bars + B_DSE, lane);
                 }
 #pragma unroll
-                for (int i = 0; i < 32; ++i) S[hf * 32 + i] = fmaf(eend, S[hf * 32 + i], __uint_as_float(v[i]));
+                for (int i = 0; i < 32; i += 2) {
+                    const float2 r = __ffma2_rn(make_float2(eend, eend), make_float2(S[hf * 32 + i], S[hf * 32 + i + 1]),
+                                                make_float2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+                    S[hf * 32 + i] = r.x;
+                    S[hf * 32 + i + 1] = r.y;
+                }
                 // bf16 copy of S^T for the next chunk's Y_inter (dS_c complete implies Y_inter_c complete, so
                 // the previous copy is no longer being read)
 #pragma unroll
@@ -458,9 +401,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             tc::fence_proxy_async();
             warp_arrive(bars + B_SF, lane);
             if (loader && c + 2 < nchunks) load_chunk(c + 2);
-            if (quad == SSD_TRQ) SSD_TR(5, c, 2);
-            if (c + 1 < nchunks && !xs_half(c + 1)) { ok = false; break; }
-            if (quad == SSD_TRQ) SSD_TR(5, c, 3);
         }
         if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
         if (!ok && loader) {                          // let copies already issued land before the CTA goes away
@@ -484,7 +424,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         bool ok = true;
 #pragma unroll 1
         for (int c = 0; c <= nchunks; ++c) {
-            if (quad == SSD_TRQ) SSD_TR(6, c, 0);
             if (c < nchunks) {
                 // Xs_c = exp(l_end - l_j) dt_j x_j, same swizzled layout as the X tile
                 const int d = c & (DEC_DEPTH - 1), sx = c % X_SLOTS;
@@ -492,12 +431,10 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (!tc::mbar_wait(bars + B_DECF + d, (c >> 2) & 1, abort_flag)) { ok = false; break; }
                 if (!tc::mbar_wait(bars + B_XF + sx, (c / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
                 if (c > 0 && !tc::mbar_wait(bars + B_DSF, (c - 1) & 1, abort_flag)) { ok = false; break; }   // Xs buffer free
-                if (quad == SSD_TRQ) SSD_TR(6, c, 1);
-                scale_x_half(smem + OFF_X + sx * TILE_16K, smem + OFF_XS, dec + D_XW, tid_g, 1);
+                scale_x(smem + OFF_X + sx * TILE_16K, smem + OFF_XS, dec + D_XW, tid_g);
                 tc::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bars + B_XSF);
-                if (quad == SSD_TRQ) SSD_TR(6, c, 2);
             }
             if (c >= 1) {
                 const int cp = c - 1, d = cp & (DEC_DEPTH - 1), t0 = cp * Q;
@@ -505,7 +442,6 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bars + B_DECE + d);
                 if (!tc::mbar_wait(bars + B_YF, cp & 1, abort_flag)) { ok = false; break; }
-                if (quad == SSD_TRQ) SSD_TR(6, c, 3);
                 tc::tc_fence_after();
                 uint4 *dst = (uint4 *)(yb + (size_t)(t0 + row) * H * P);
                 const bool valid = t0 + row < Tlen;
@@ -515,7 +451,12 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc::tmem_ld_wait();
                 if (cp > 0) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) ya[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(ya[i])));
+                    for (int i = 0; i < 32; i += 2) {
+                        const float2 r = __ffma2_rn(make_float2(er, er), make_float2(__uint_as_float(yo[i]), __uint_as_float(yo[i + 1])),
+                                                    make_float2(__uint_as_float(ya[i]), __uint_as_float(ya[i + 1])));
+                        ya[i] = __float_as_uint(r.x);
+                        ya[i + 1] = __float_as_uint(r.y);
+                    }
                 }
                 // second half in flight while the first is narrowed and stored
                 tc::tmem_ld32(tmem + lane_base + TM_YI + 32, yb2);
@@ -531,10 +472,14 @@ ssd_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc::tmem_ld_wait();
                 tc::tc_fence_before();               // both accumulators are in registers
                 warp_arrive(bars + B_YE, lane);
-                if (quad == SSD_TRQ) SSD_TR(6, c, 4);
                 if (cp > 0) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) yb2[i] = __float_as_uint(fmaf(er, __uint_as_float(yo[i]), __uint_as_float(yb2[i])));
+                    for (int i = 0; i < 32; i += 2) {
+                        const float2 r = __ffma2_rn(make_float2(er, er), make_float2(__uint_as_float(yo[i]), __uint_as_float(yo[i + 1])),
+                                                    make_float2(__uint_as_float(yb2[i]), __uint_as_float(yb2[i + 1])));
+                        yb2[i] = __float_as_uint(r.x);
+                        yb2[i + 1] = __float_as_uint(r.y);
+                    }
                 }
                 if (valid) {
 #pragma unroll

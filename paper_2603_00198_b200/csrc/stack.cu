@@ -123,7 +123,7 @@ struct StackFeed { int chunks; int rows_per_chunk; cudaEvent_t *ready; };
         if (_rc != STR_OK) return _rc; \
     } while (0)
 
-static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in, void *hidden_out,
+static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_stack_io *io, const void *hidden_in, void *hidden_out,
                               int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace, float *scores_trace,
                               void *workspace, size_t workspace_bytes, void *stream, const StackFeed *feed) {
     if (!ctx || !desc_ok(d) || !hidden_in || !hidden_out || !workspace) return STR_ERR_INVALID_ARG;
@@ -147,7 +147,15 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const void 
         const int rows = Bz * (n_cur + M);
         iota_rows_kernel<<<ceil_div(rows, 256), 256, 0, st>>>(rows, n_cur + M, pos[0], idx[0]);
         STR_TRY(str_launch_ok(ctx));
+        // a caller that continues from a reduced context brings the original token ids of its rows
+        if (io && io->positions_in)
+            STR_CUDA_OK(cudaMemcpyAsync(pos[0], io->positions_in, (size_t)rows * 4, cudaMemcpyDeviceToDevice, st));
+        if (io && io->idx_map_in)
+            STR_CUDA_OK(cudaMemcpyAsync(idx[0], io->idx_map_in, (size_t)rows * 4, cudaMemcpyDeviceToDevice, st));
     }
+    float *fs_out = io ? io->mamba_final_states : nullptr;
+    char *k_out = io ? (char *)io->attn_k_out : nullptr, *v_out = io ? (char *)io->attn_v_out : nullptr;
+    int32_t *kvpos_out = io ? io->attn_pos_out : nullptr;
     const void *cur = hidden_in;
     int hsel = 0;      // next free hidden buffer
     int psel = 0;      // current positions / idx buffer
@@ -199,8 +207,9 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const void 
             STR_TRY(str_mamba_conv_split_rows(ctx, dtype, Bz, T, d->H, d->p, d->n, d->G, d->conv_width, !reduce, proj,
                                               L.conv_w, L.conv_b, L.dt_bias, bufA, bufB, bufC, dt, stream));
             str_ssd_shape s = {Bz, T, d->H, d->p, d->n, d->G, d->Q, dtype};
-            STR_TRY(str_mamba2_prefill(ctx, &s, bufA, dt, L.A, bufB, bufC, nullptr, nullptr, bufY, nullptr, sub,
+            STR_TRY(str_mamba2_prefill(ctx, &s, bufA, dt, L.A, bufB, bufC, nullptr, nullptr, bufY, fs_out, sub,
                                        r.sub_bytes, stream));
+            if (fs_out) fs_out += (size_t)Bz * d->H * d->p * d->n;
             if (want_score && n_cur > 0) {
                 str_ssm_score_shape ss = {Bz, T, d->H, d->n, d->G, dtype};
                 if (d->mamba_score_kind == STR_SCORE_FULL_DYNAMIC)
@@ -256,6 +265,22 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const void 
             } else {
                 STR_TRY(str_gemm(ctx, dtype, rows, D, qd, bufY, L.w_out, cur, dst, sub, r.sub_bytes, stream));
             }
+            // hand-off to a decoder: keys, values and positions of the rows that leave the layer
+            if (k_out || v_out || kvpos_out) {
+                const size_t kv_bytes = (size_t)rows_out * kd * dtype_size(dtype);
+                if (reduce) {
+                    if (k_out) STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, kd, dtype, bufB, nullptr, nullptr, kept, k_out, nullptr, nullptr, stream));
+                    if (v_out) STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, kd, dtype, bufC, nullptr, nullptr, kept, v_out, nullptr, nullptr, stream));
+                    if (kvpos_out) STR_CUDA_OK(cudaMemcpyAsync(kvpos_out, pdst, (size_t)rows_out * 4, cudaMemcpyDeviceToDevice, st));
+                } else {
+                    if (k_out) STR_CUDA_OK(cudaMemcpyAsync(k_out, bufB, kv_bytes, cudaMemcpyDeviceToDevice, st));
+                    if (v_out) STR_CUDA_OK(cudaMemcpyAsync(v_out, bufC, kv_bytes, cudaMemcpyDeviceToDevice, st));
+                    if (kvpos_out) STR_CUDA_OK(cudaMemcpyAsync(kvpos_out, pos[psel], (size_t)rows_out * 4, cudaMemcpyDeviceToDevice, st));
+                }
+                if (k_out) k_out += kv_bytes;
+                if (v_out) v_out += kv_bytes;
+                if (kvpos_out) kvpos_out += rows_out;
+            }
         }
         cur = dst;
         if (dst == hid[0]) hsel = 1;
@@ -278,8 +303,15 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const void 
 extern "C" int str_stack_prefill(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in, void *hidden_out,
                                  int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace,
                                  float *scores_trace, void *workspace, size_t workspace_bytes, void *stream) {
-    return stack_prefill_impl(ctx, d, hidden_in, hidden_out, positions_out, idx_map_out, kept_trace, scores_trace, workspace,
-                              workspace_bytes, stream, nullptr);
+    return stack_prefill_impl(ctx, d, nullptr, hidden_in, hidden_out, positions_out, idx_map_out, kept_trace, scores_trace,
+                              workspace, workspace_bytes, stream, nullptr);
+}
+
+extern "C" int str_stack_prefill_ex(str_ctx *ctx, const str_stack_desc *d, const str_stack_io *io, const void *hidden_in,
+                                    void *hidden_out, int32_t *positions_out, int32_t *idx_map_out, int32_t *kept_trace,
+                                    float *scores_trace, void *workspace, size_t workspace_bytes, void *stream) {
+    return stack_prefill_impl(ctx, d, io, hidden_in, hidden_out, positions_out, idx_map_out, kept_trace, scores_trace,
+                              workspace, workspace_bytes, stream, nullptr);
 }
 
 extern "C" size_t str_stack_host_workspace_size(const str_stack_desc *d) {
@@ -323,7 +355,7 @@ extern "C" int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, con
         STR_CUDA_OK(cudaEventRecord(ctx->copy_ev[1 + nblk], ctx->copy_stream));
     }
     const StackFeed feed = {nblk, (int)per, ctx->copy_ev + 1};
-    int rc = stack_prefill_impl(ctx, d, in_dev, out_dev, pos_dev, idx_dev, nullptr, nullptr, ws,
+    int rc = stack_prefill_impl(ctx, d, nullptr, in_dev, out_dev, pos_dev, idx_dev, nullptr, nullptr, ws,
                                 workspace_bytes - (size_t)(ws - (char *)workspace), stream, &feed);
     if (rc != STR_OK) return rc;
     STR_CUDA_OK(cudaMemcpyAsync(hidden_out_host, out_dev, Rout * d->D * e, cudaMemcpyDeviceToHost, st));

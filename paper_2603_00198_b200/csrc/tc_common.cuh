@@ -67,6 +67,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return true;
 }
 
+// Has an earlier CTA of this launch (or an earlier launch) recorded an error?  Thread 0 reads the status word and
+// the block agrees on the answer, so that a CTA leaves whole or not at all: warps that stayed behind would run
+// warp-collective tcgen05 instructions and barriers with roles missing.
+__device__ __forceinline__ bool cta_should_leave(const int *status) {
+    return __syncthreads_or(threadIdx.x == 0 && *(volatile const int *)status != 0) != 0;
+}
+
 // ---- TMA ------------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)m) : "memory");
@@ -154,6 +161,84 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
         : "memory");
 }
+// ---- several K-slices of one product in ONE instruction block ---------------------------------
+// Measured on B200 (one issuing warp next to arithmetic warps on its scheduler): a product written as a
+// loop of single tcgen05.mma statements, or issued from an `if (lane == 0)` region, costs 100-400 clocks
+// per instruction once the scheduler has other ready warps, because every instruction in between is a
+// chance to lose the issue slot.  The same K-slices written as one straight-line block inside a region
+// entered through elect_one() (which the compiler knows to be single-threaded) issue at the tensor pipe's
+// own rate (about 50 clocks for N = 64, 64 for N = 128) whatever the other warps do.  So issuer roles
+// enter elect_one() ONCE, stay in it for their whole loop, and issue each product with these helpers.
+// `Step` gives the descriptor / tensor-memory address advance of K-slice ks as a compile-time constant.
+struct StepKMajor2x64 {   // K-major operand stored as two 64-column halves 16 KB apart (128-byte swizzle), 16-byte units
+    static __host__ __device__ constexpr uint32_t at(int ks) { return (uint32_t)(ks >> 2) * 1024u + (uint32_t)(ks & 3) * 2u; }
+};
+struct StepKMajor64 {     // K-major operand, one 64-column tile: 32 bytes per K-slice
+    static __host__ __device__ constexpr uint32_t at(int ks) { return (uint32_t)ks * 2u; }
+};
+struct StepMNMajor {      // MN-major operand: 16 K-rows x 128 bytes = 2 KB per K-slice
+    static __host__ __device__ constexpr uint32_t at(int ks) { return (uint32_t)ks * 128u; }
+};
+struct StepTmem8 {        // bf16 A operand in tensor memory, K-slices in consecutive groups of 8 columns
+    static __host__ __device__ constexpr uint32_t at(int ks) { return (uint32_t)ks * 8u; }
+};
+struct StepTmem16 {       // bf16 A operand in tensor memory, K-slice ks in the first 8 of columns [16 ks, 16 ks + 16)
+    static __host__ __device__ constexpr uint32_t at(int ks) { return (uint32_t)ks * 16u; }
+};
+
+#define STR_MMA_TAIL_SS(n, ia, ib)                                                        \
+    "add.s64 a, %1, %" #ia ";\n\tadd.s64 b, %2, %" #ib ";\n\t"                            \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
+#define STR_MMA_TAIL_TS(n, ia, ib)                                                        \
+    "add.u32 at, %1, %" #ia ";\n\tadd.s64 b, %2, %" #ib ";\n\t"                           \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], b, %3, pt;\n\t"
+
+// Eight K-slices, both operands in shared memory.  The first slice accumulates iff acc_first.
+template <class SA, class SB>
+__device__ __forceinline__ void mma8_ss(uint32_t d_tmem, uint64_t a0, uint64_t b0, uint32_t idesc, bool acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred pf, pt;\n\t.reg .b64 a, b;\n\t"
+        "setp.ne.b32 pf, %4, 0;\n\tsetp.eq.u32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n\t"
+        STR_MMA_TAIL_SS(1, 5, 6) STR_MMA_TAIL_SS(2, 7, 8) STR_MMA_TAIL_SS(3, 9, 10) STR_MMA_TAIL_SS(4, 11, 12)
+        STR_MMA_TAIL_SS(5, 13, 14) STR_MMA_TAIL_SS(6, 15, 16) STR_MMA_TAIL_SS(7, 17, 18)
+        "}"
+        ::"r"(d_tmem), "l"(a0), "l"(b0), "r"(idesc), "r"((uint32_t)acc_first),
+          "n"(SA::at(1)), "n"(SB::at(1)), "n"(SA::at(2)), "n"(SB::at(2)), "n"(SA::at(3)), "n"(SB::at(3)), "n"(SA::at(4)), "n"(SB::at(4)),
+          "n"(SA::at(5)), "n"(SB::at(5)), "n"(SA::at(6)), "n"(SB::at(6)), "n"(SA::at(7)), "n"(SB::at(7))
+        : "memory");
+}
+// Eight K-slices, A (bf16) in tensor memory, B in shared memory.
+template <class SA, class SB>
+__device__ __forceinline__ void mma8_ts(uint32_t d_tmem, uint32_t a_tmem0, uint64_t b0, uint32_t idesc, bool acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred pf, pt;\n\t.reg .b64 b;\n\t.reg .b32 at;\n\t"
+        "setp.ne.b32 pf, %4, 0;\n\tsetp.eq.u32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pf;\n\t"
+        STR_MMA_TAIL_TS(1, 5, 6) STR_MMA_TAIL_TS(2, 7, 8) STR_MMA_TAIL_TS(3, 9, 10) STR_MMA_TAIL_TS(4, 11, 12)
+        STR_MMA_TAIL_TS(5, 13, 14) STR_MMA_TAIL_TS(6, 15, 16) STR_MMA_TAIL_TS(7, 17, 18)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem0), "l"(b0), "r"(idesc), "r"((uint32_t)acc_first),
+          "n"(SA::at(1)), "n"(SB::at(1)), "n"(SA::at(2)), "n"(SB::at(2)), "n"(SA::at(3)), "n"(SB::at(3)), "n"(SA::at(4)), "n"(SB::at(4)),
+          "n"(SA::at(5)), "n"(SB::at(5)), "n"(SA::at(6)), "n"(SB::at(6)), "n"(SA::at(7)), "n"(SB::at(7))
+        : "memory");
+}
+// Four K-slices (one 64-column stage), both operands in shared memory.
+template <class SA, class SB>
+__device__ __forceinline__ void mma4_ss(uint32_t d_tmem, uint64_t a0, uint64_t b0, uint32_t idesc, bool acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred pf, pt;\n\t.reg .b64 a, b;\n\t"
+        "setp.ne.b32 pf, %4, 0;\n\tsetp.eq.u32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n\t"
+        STR_MMA_TAIL_SS(1, 5, 6) STR_MMA_TAIL_SS(2, 7, 8) STR_MMA_TAIL_SS(3, 9, 10)
+        "}"
+        ::"r"(d_tmem), "l"(a0), "l"(b0), "r"(idesc), "r"((uint32_t)acc_first),
+          "n"(SA::at(1)), "n"(SB::at(1)), "n"(SA::at(2)), "n"(SB::at(2)), "n"(SA::at(3)), "n"(SB::at(3))
+        : "memory");
+}
+#undef STR_MMA_TAIL_SS
+#undef STR_MMA_TAIL_TS
+
 // Arrive on an mbarrier when all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void mma_commit(uint64_t *bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -217,6 +302,13 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// log2(x) on the special-function unit (log2(0) = -inf).
+__device__ __forceinline__ float lg2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
