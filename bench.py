@@ -62,18 +62,10 @@ def workload(args):
     return cfg
 
 
-def ffn_keep_counts(pattern, K, n_vis):
-    """FFN layers never reduce: a cut that the schedule places on one is taken by the next Mamba / attention layer."""
-    out, n_cur = [], n_vis
-    for kind, k in zip(pattern, K):
-        n_cur = n_cur if kind == "F" else min(k, n_cur)
-        out.append(n_cur)
-    return out
-
-
 # ------------------------------------------------------------------ algorithmic work per category
 def work_model(cfg, keep_counts):
-    """Algorithmic flops / bytes of one step, per kernel category (formulas in the design doc)."""
+    """Algorithmic flops / bytes of one step, per kernel category: 2 M N K per product and one read + one write of
+    every operand for the GEMMs, the causal chunked count for the scan, the score / select / gather byte counts."""
     ms, at = cfg["mamba"], cfg["attn"]
     D, M, Bz = ms["D"], cfg["n_text"], cfg["batch"]
     H, p, n, G, Q = ms["H"], ms["p"], ms["n"], ms["G"], ms["Q"]
@@ -110,9 +102,11 @@ def work_model(cfg, keep_counts):
                 w["attn_score"]["bytes"] += 2 * Bz * n_cur * 2.0 * Hkv * d
         if K < n_cur:
             w["topk"]["bytes"] += Bz * (4.0 * n_cur + 4.0 * K)
-            w["compact"]["bytes"] += Bz * 2.0 * (K + M) * (2 * D + 8)
+            w["compact"]["bytes"] += Bz * 2.0 * (K + M) * (2 * D + 8)       # residual rows, positions, index map
             if kind == "A":
                 w["compact"]["bytes"] += Bz * 2.0 * (K + M) * 2 * Hq * d     # the survivors' attention outputs
+            else:
+                w["compact"]["bytes"] += Bz * 2.0 * (K + M) * 2 * D          # the survivors' normed rows (input of the z projection)
             n_cur = K
     return w
 
@@ -126,13 +120,13 @@ class ClockSampler:
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index):
+    def __init__(self, gpu_index, interval_ms=100):
         self.path = tempfile.mktemp(suffix=".csv")
         self.proc = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", str(int(interval_ms))], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -178,11 +172,28 @@ def oracle_sample_tokens_per_s(cfg, n_vis_s, n_text_s, seed):
     from paper_2603_00198_b200 import inputs
     layers = inputs.stack_params(seed, cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"], ffn_dim=cfg.get("ffn_dim", 0))
     h0 = inputs.hidden_inputs(seed, n_vis_s + n_text_s, cfg["mamba"]["D"], cfg["dtype"])[0]
-    K = ffn_keep_counts(cfg["pattern"], oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0), n_vis_s)
+    K = oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0, cfg["pattern"])
     t0 = time.perf_counter()
     oracle.stack_prefill(h0, n_text_s, layers, K, oracle.round_to_bf16)
     sec = time.perf_counter() - t0
     return (n_vis_s + n_text_s) / sec, sec, layers
+
+
+def oracle_whole_config(name):
+    """The oracle on one whole single-layer configuration (C0: tiny fp32 Mamba-2 layer, C1: 8B-class Mamba-2 layer),
+    inputs and weights as the configuration states them.  Returns seconds and tokens/s."""
+    import oracle
+    from paper_2603_00198_b200 import inputs
+    cfg = inputs.CONFIGS[name]
+    layers = inputs.stack_params(cfg["seed"], "M", cfg["shape"], cfg["shape"], cfg["dtype"])
+    T = cfg["n_vis"] + cfg["n_text"]
+    h0 = inputs.hidden_inputs(cfg["seed"], T, cfg["shape"]["D"], cfg["dtype"])[0]
+    K = oracle.schedule_keep_counts([cfg["keep_bp"]], cfg["n_vis"], 0)
+    rnd = oracle.round_to_bf16 if cfg["dtype"] == "bf16" else oracle._identity
+    t0 = time.perf_counter()
+    oracle.stack_prefill(h0, cfg["n_text"], layers, K, rnd)
+    sec = time.perf_counter() - t0
+    return {"seconds": sec, "tokens_per_s": T / sec, "tokens": T}
 
 
 def run_reference(args):
@@ -198,7 +209,7 @@ def run_reference(args):
     n_vis_s = args.ref_tokens - n_text_s
     layers = inputs.stack_params(cfg["seed"], cfg["pattern"], cfg["mamba"], cfg["attn"], cfg["dtype"], ffn_dim=cfg.get("ffn_dim", 0))
     h0 = inputs.hidden_inputs(cfg["seed"], n_vis_s + n_text_s, cfg["mamba"]["D"], cfg["dtype"])[0]
-    K = ffn_keep_counts(cfg["pattern"], oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0), n_vis_s)
+    K = oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis_s, 0, cfg["pattern"])
 
     def step():
         oracle.stack_prefill(h0, n_text_s, layers, K, oracle.round_to_bf16)
@@ -256,8 +267,7 @@ def run_ours(args):
     cfg = workload(args)
     Bz, n_vis, M, D = cfg["batch"], cfg["n_vis"], cfg["n_text"], cfg["mamba"]["D"]
     T0 = n_vis + M
-    K = binding.str_schedule_keep_counts(cfg["alpha_bp"], n_vis, cfg["min_keep"])
-    K = ffn_keep_counts(cfg["pattern"], K, n_vis)
+    K = binding.str_schedule_keep_counts_layers(cfg["alpha_bp"], cfg["pattern"], n_vis, cfg["min_keep"])
 
     ctx = binding.Context(local)
     # weights: seeded on the host, one replica per rank (the path does not shard: replicas only)
@@ -284,6 +294,7 @@ def run_ours(args):
     barrier()
     sampler = ClockSampler(local) if rank == 0 else None
     l0 = ctx.launch_count()
+    tc0, fb0 = ctx.path_counts()
     ctx.profile_enable(True)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -296,8 +307,12 @@ def run_ours(args):
     ctx.profile_enable(False)
     prof = ctx.profile_collect()
     launches = ctx.launch_count() - l0
+    tc1, fb1 = ctx.path_counts()
     clocks = sampler.stop() if sampler else None
     ctx.check_status()
+    # the headline number is a tensor-core number: no call of the timed region may have taken an fp32-FMA fallback
+    if fb1 != fb0:
+        raise SystemExit("bench: %d calls of the timed region fell back to the fp32-FMA kernels" % (fb1 - fb0))
 
     # ---- end to end through the host-buffer entry point (H2D + stack + D2H inside the timed region)
     for _ in range(max(1, min(args.warmup, 2))):
@@ -360,7 +375,20 @@ def run_ours(args):
         val, sec, _ = oracle_sample_tokens_per_s(cfg, args.ref_tokens - n_text_s, n_text_s, cfg["seed"])
         cpu = {"value": val, "unit": UNIT, "cores": os.cpu_count() or 1, "kind": "oracle",
                "sample": "fp64 oracle stack_prefill, full layer shapes and schedule, %d visual + %d text tokens, %.1f s"
-                         % (args.ref_tokens - n_text_s, n_text_s, sec)}
+                         % (args.ref_tokens - n_text_s, n_text_s, sec),
+               "whole_configs": {name: oracle_whole_config(name) for name in ("C0", "C1")}}
+
+    # ---- the exported hot-path calls alone, at the configurations' shapes (outside the timed region; rank 0, N=1)
+    alone = None
+    if world == 1 and not args.no_kernels_alone:
+        del out, pos, idx
+        alone = []
+        for name, nv, bp in KERNELS_ALONE:
+            r = micro_case(ctx, pk, name, Bz=1, n_vis=nv, final_bp=bp, steps=5, warmup=3, min_seconds=0.5, gpu_index=local)
+            alone.append({"kernel": name, "n_vis": nv, "ms": r["ms"], "bound": r["roofline"]["bound"],
+                          "achieved": r["roofline"]["achieved"], "unit": r["roofline"]["unit"], "frac": r["roofline"]["frac"],
+                          "gbs": r["gbs"], "tflops": r["tflops"], "launches_timed": r["launches_timed"], "clocks": r["clocks"]})
+            torch.cuda.empty_cache()
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -378,6 +406,8 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h_pin.numel() * 2),
                 "d2h_bytes_per_step": int(out_pin.numel() * 2 + idx_pin.numel() * 4), "matches_device_run": same},
         "gpu_launches": int(launches), "clocks": clocks, "kernels": kernels,
+        "paths": {"tensor_core_calls": int(tc1 - tc0), "fallback_calls": int(fb1 - fb0)},
+        "kernels_alone": alone,
     }
     print(json.dumps(line))
     if world > 1:
@@ -386,21 +416,20 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------ single-kernel microbenchmarks
-def run_micro(args):
-    """--micro NAME: times one entry point of the hot path alone (CUDA events, L2 flushed between launches)
-    on seeded device-side inputs of the C1/C2 layer shapes and prints one JSON line with its roofline."""
+def micro_case(ctx, pk, name, Bz=1, n_vis=32768, final_bp=5000, attn_denominator="visual", steps=5, warmup=3,
+               min_seconds=0.0, gpu_index=0):
+    """Times one entry point of the hot path alone (CUDA events on the launching stream, L2 flushed between launches)
+    on seeded device-side inputs of the C1 / C2 layer shapes.  Returns a dict with its roofline and the SM clocks
+    sampled while it ran (launches are repeated for at least `min_seconds` so that the sampler sees the GPU under
+    load)."""
     import torch
     from paper_2603_00198_b200 import binding, inputs
-    torch.cuda.set_device(0)
     torch.manual_seed(1234)
-    ctx = binding.Context(0)
-    pk = peaks()
     ms_, at_ = inputs.MAMBA_8B, inputs.ATTN_8B
-    Bz, n_vis, M = args.batch, (args.n_vis or 32768), 128
+    M = 128
     T = n_vis + M
-    dev = "cuda:0"
+    dev = "cuda:%d" % gpu_index
     bf = torch.bfloat16
-    name = args.micro
     flops = nbytes = 0.0
     bound = "hbm"
     if name == "ssd":
@@ -437,7 +466,7 @@ def run_micro(args):
         Hq, Hkv, d = at_["Hq"], at_["Hkv"], at_["d"]
         q = torch.randn(Bz, T, Hq, d, device=dev).to(bf)
         k = torch.randn(Bz, T, Hkv, d, device=dev).to(bf)
-        fn = lambda: binding.str_attn_importance(ctx, q, k, n_vis, M, 1.0 / np.sqrt(d), denominator=args.attn_denominator)
+        fn = lambda: binding.str_attn_importance(ctx, q, k, n_vis, M, 1.0 / np.sqrt(d), denominator=attn_denominator)
         flops = 2 * Bz * n_vis * 2.0 * M * d * Hq
         nbytes = 2 * Bz * n_vis * 2.0 * Hkv * d
         bound = "tensor"
@@ -451,13 +480,13 @@ def run_micro(args):
         nbytes = Bz * T * 2.0 * (2 * Hq * d + 2 * Hkv * d)
         bound = "tensor"
     elif name == "topk":
-        K = max(1, n_vis * (args.final_bp or 5000) // 10000)
+        K = max(1, n_vis * (final_bp or 5000) // 10000)
         sc = torch.rand(Bz, n_vis, device=dev)
         fn = lambda: binding.str_topk_select(ctx, sc, K)
         nbytes = Bz * (4.0 * n_vis + 4.0 * K)
     elif name == "compact":
         D = ms_["D"]
-        K = max(1, n_vis * (args.final_bp or 5000) // 10000)
+        K = max(1, n_vis * (final_bp or 5000) // 10000)
         hid = torch.randn(Bz, T, D, device=dev).to(bf)
         pos = torch.arange(T, device=dev, dtype=torch.int32).repeat(Bz, 1).contiguous()
         kept = torch.sort(torch.rand(Bz, n_vis, device=dev).argsort(dim=1)[:, :K], dim=1).values.to(torch.int32).contiguous()
@@ -475,12 +504,14 @@ def run_micro(args):
     else:
         raise SystemExit("unknown --micro " + name)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    for _ in range(max(3, args.warmup)):
+    for _ in range(max(3, warmup)):
         fn()
     ctx.check_status()
     torch.cuda.synchronize()
+    sampler = ClockSampler(gpu_index, interval_ms=50)
     times = []
-    for _ in range(args.steps):
+    t_begin = time.perf_counter()
+    while len(times) < steps or time.perf_counter() - t_begin < min_seconds:
         flush.zero_()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -488,17 +519,34 @@ def run_micro(args):
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
+    clocks = sampler.stop()
     ctx.check_status()
     ms = float(np.median(times))
     if bound == "tensor":
         ach, peak, unit = flops / (ms * 1e-3) / 1e12, pk["bf16_tflops"], "TFLOP/s"
     else:
         ach, peak, unit = nbytes / (ms * 1e-3) / 1e9, pk["hbm_gbs"], "GB/s"
-    print(json.dumps({"micro": name, "batch": Bz, "n_vis": n_vis, "n_text": M, "ms": ms, "ms_min": float(min(times)),
-                      "steps": args.steps, "l2": "256 MB buffer written between launches",
-                      "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                                   "peak_source": pk["source"] + " (burst figure: kernel timed alone)"},
-                      "gbs": nbytes / (ms * 1e-3) / 1e9, "tflops": flops / (ms * 1e-3) / 1e12 if flops else None}))
+    return {"micro": name, "batch": Bz, "n_vis": n_vis, "n_text": M, "ms": ms, "ms_min": float(min(times)),
+            "launches_timed": len(times), "l2": "256 MB buffer written between launches",
+            "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                         "peak_source": pk["source"] + " (burst figure: kernel timed alone)"},
+            "gbs": nbytes / (ms * 1e-3) / 1e9, "tflops": flops / (ms * 1e-3) / 1e12 if flops else None, "clocks": clocks}
+
+
+# The exported hot-path calls at the shapes the benchmark configurations give them, timed alone after the headline run.
+KERNELS_ALONE = [("ssd", 4096, 0), ("ssd", 32768, 0), ("mamba_score", 32768, 0), ("attn_score", 16384, 0),
+                 ("topk", 32768, 5000), ("compact", 32768, 5000)]
+
+
+def run_micro(args):
+    """--micro NAME: one entry point alone; prints one JSON line with its roofline and clock record."""
+    import torch
+    from paper_2603_00198_b200 import binding
+    torch.cuda.set_device(0)
+    ctx = binding.Context(0)
+    res = micro_case(ctx, peaks(), args.micro, Bz=args.batch, n_vis=args.n_vis or 32768, final_bp=args.final_bp,
+                     attn_denominator=args.attn_denominator, steps=args.steps, warmup=args.warmup, min_seconds=args.micro_seconds)
+    print(json.dumps(res))
 
 
 def main():
@@ -520,6 +568,8 @@ def main():
     ap.add_argument("--attn-denominator", default="visual", choices=["visual", "causal_row"],
                     help="normaliser of the attention-layer importance: visual keys only (the paper's formula) or the causal row")
     ap.add_argument("--x0", type=float, default=0.11, help="midpoint of the sigmoid schedule (0.11 / 0.24 / 0.41)")
+    ap.add_argument("--micro-seconds", type=float, default=0.6, help="repeat a --micro launch for at least this long (clock sampling)")
+    ap.add_argument("--no-kernels-alone", action="store_true", help="skip the per-kernel timings after the headline run")
     ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | mamba_dyn_score | attn_score | attn_fwd | "
                                                 "topk | compact | gemm")
     args = ap.parse_args()

@@ -40,7 +40,9 @@ enum { STR_F32 = 0, STR_BF16 = 1 };
 typedef struct str_ctx str_ctx;
 
 /* Context: device id, SM count, tensor-map encoder, device status word.  str_create allocates
- * a few bytes of device memory and may synchronise; str_destroy frees them. */
+ * a few bytes of device memory and may synchronise; str_destroy frees them.  str_create fails with
+ * STR_ERR_CUDA when the driver offers no tensor-map encoder: without it no tensor-core kernel can run
+ * and every call would silently take the much slower fp32-FMA kernels. */
 int str_create(int device, str_ctx **out);
 int str_destroy(str_ctx *ctx);
 const char *str_strerror(int code);
@@ -124,12 +126,16 @@ int str_attn_importance_ex(str_ctx *ctx, const str_attn_score_shape *s, int n_vi
 /* (2b, allocation-free variant)  The paper has no counterpart for this call; it exists for callers
  * that cannot allocate device memory (a plug-in inside a host with a fixed memory pool, a real-time
  * loop that must stay off the allocator, code that is handed raw pointers and owns no allocator).
- * Same inputs, outputs and result as str_attn_importance, but the per-(sequence, head, query) row
- * maxima and sums live in a fixed array inside the library image, so no workspace is passed and the
- * call performs no allocation of any kind.
+ * Same inputs and outputs as str_attn_importance, but the per-(sequence, head, query) row maxima and
+ * sums live in a fixed array inside the library image, so no workspace is passed and the call itself
+ * allocates nothing.  It always runs the plain fp32-FMA kernels (never the tensor-core path), so for
+ * bf16 inputs with head dimension 128 its scores agree with str_attn_importance to the score tolerance
+ * (1e-3 relative), not bit for bit, and it is slower at large shapes.
  *   Limit: Bz * Hq * n_text <= STR_ATTN_STATIC_MAX_ROWS, else STR_ERR_WORKSPACE_TOO_SMALL is
  *   returned and nothing is launched.  The array (2 * STR_ATTN_STATIC_MAX_ROWS floats = 512 KiB) is
- *   resident on every GPU that loads the library until the process exits.
+ *   resident on every GPU that loads the library until the process exits; it becomes resident when
+ *   the driver loads the library's device code, which with lazy module loading may be during the
+ *   first call.
  *   The first call on a device looks up the array's device address (one runtime query, no
  *   allocation); make that first call before starting any stream capture.
  *   All calls share the array and it keeps the previous call's contents; each call overwrites the
@@ -173,9 +179,21 @@ int str_compact(str_ctx *ctx, int Bz, int T_in, int n_vis, int n_text, int k, in
  * points of the ORIGINAL visual count n0; K_out[l] = min(n_cur, max(min_keep, floor(alpha n0)))
  * is the visual count after layer l.  Layer l reduces iff K_out[l] < its incoming count. */
 int str_schedule_keep_counts(const int *alpha_bp, int L, int n0, int min_keep, int *K_out);
+/* Same for a stack whose layer kinds (STR_LAYER_*, host array [L]) are known: FFN layers never reduce, so a cut the
+ * schedule places on an FFN layer is taken by the next Mamba / attention layer (K_out of an FFN layer equals its
+ * incoming count).  The paper's all-layer schedules cut at Mamba and attention layers only. */
+int str_schedule_keep_counts_layers(const int *alpha_bp, const int *layer_kinds, int L, int n0, int min_keep, int *K_out);
 /* Sigmoid retention alpha_l = a_end + (a_start - a_end) * sigmoid(k (x0 - l/L)), in basis points
  * (rounded to nearest), l = 0..L-1.  Host only. */
 int str_sigmoid_schedule_bp(int L, double k, double x0, double a_start, double a_end, int *alpha_bp_out);
+
+/* (3') Density of an importance vector (Section 2, the sparsity analysis: "tokens needed for 80% of the importance
+ * mass"): per row, the smallest k such that the k largest scores sum to at least mass_fraction of the row's total.
+ * A diagnostic of how concentrated a layer's scores are; the mass-threshold dual of the rank threshold of (3).
+ *   scores device [Bz,n_vis] fp32, all >= 0; mass_fraction in (0,1]; count_out device [Bz] int32 (0 for a row
+ *   whose scores are all zero).  Sums are taken in fp64.  No workspace. */
+int str_score_density(str_ctx *ctx, int Bz, int n_vis, const float *scores, float mass_fraction,
+                      int32_t *count_out, void *stream);
 
 /* ------------------------------------------------------------------------------------------
  * Block glue.  The paper gives only the recurrence and the scores; these are the standard
@@ -315,6 +333,14 @@ int str_profile_collect(str_ctx *ctx, double *ms_by_category, long long *calls_b
 
 /* Number of kernels this library has launched on this context since creation (host counter). */
 long long str_launch_count(const str_ctx *ctx);
+/* How many entry-point calls on this context ran a tensor-core (tcgen05) kernel and how many fell back to the plain
+ * fp32-FMA kernel of the same entry point (shapes or dtypes the tensor-core kernels do not tile, or
+ * STR_FORCE_SIMT=1 in the environment).  Counted for the scan, the three scores, the GEMM and the attention forward. */
+int str_path_counts(const str_ctx *ctx, long long *tensor_core_calls, long long *fallback_calls);
+/* Self-test of the bounded device-side waits: launches one CTA that waits on a barrier nobody signals, gives up
+ * after probe_limit probes (1 .. 2^20), records STR_ERR_TIMEOUT in the status word and returns normally.  The next
+ * str_check_status reports the timeout once and clears it.  No tensor memory, no copies: safe at any time. */
+int str_selftest_wait_timeout(str_ctx *ctx, unsigned int probe_limit, void *stream);
 
 #ifdef __cplusplus
 }

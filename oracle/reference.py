@@ -18,9 +18,11 @@ Pin status (tests/test_oracle_*.py, all CPU):
   compact                pinned  (bit-exact gather, index-map composition)
   step_schedule / mean_retention / schedule_keep_counts
                          pinned  (the paper's printed compression percentages)
+  score_density          pinned  (closed forms: uniform, one-hot, two-level vectors; brute force)
   sigmoid_schedule       parity unpinned: the printed percentages of the sigmoid rows are
                          not reproduced to the printed digit by any indexing of the formula
-  rmsnorm, causal_conv1d_silu, rope, attention_forward, attention_rows, mamba2_block, attn_block, stack_prefill
+  rmsnorm, causal_conv1d_silu, rope, attention_forward, attention_rows, mamba2_block, attn_block, attn_block_projections,
+  attn_block_rows, stack_prefill
                          parity unpinned by the paper (it does not define the block around the
                          recurrence); pinned only to textbook definitions, library routines
                          and brute force on tiny inputs
@@ -297,19 +299,36 @@ def mean_retention(alpha_bp):
     return sum(alpha_bp) / len(alpha_bp) / 100.0
 
 
-def schedule_keep_counts(alpha_bp, n0, min_keep):
+def schedule_keep_counts(alpha_bp, n0, min_keep, kinds=None):
     """Visual tokens kept AFTER each layer: K_l = min(n_cur, max(min_keep, floor(alpha_l n0))).
 
     alpha is a fraction of the ORIGINAL visual count n0 (pinned by the printed compression
-    percentages); integer arithmetic in basis points; the count never grows.
+    percentages); integer arithmetic in basis points; the count never grows.  With ``kinds`` (a
+    sequence of "M" / "A" / "F" per layer) FFN layers never reduce: the paper's all-layer schedules
+    cut at Mamba and attention layers, so a cut that falls on an FFN layer is taken by the next
+    Mamba / attention layer.
     """
     out, n_cur = [], int(n0)
-    for a in alpha_bp:
+    for l, a in enumerate(alpha_bp):
         k = (int(a) * int(n0)) // 10000
         k = min(n_cur, max(int(min_keep), k))
+        if kinds is not None and kinds[l] == "F":
+            k = n_cur
         out.append(k)
         n_cur = k
     return out
+
+
+def score_density(scores, mass_fraction):
+    """The sparsity statistic of Section 2 ("tokens needed for 80% of the importance mass"): the smallest k such
+    that the k largest scores sum to at least ``mass_fraction`` of the total.  Full sort, fp64 cumulative sum.
+    Returns 0 for an all-zero vector."""
+    s = np.sort(_f64(scores))[::-1]
+    csum = np.cumsum(s)
+    total = csum[-1] if len(csum) else 0.0            # the total is the last running sum: the full vector always suffices
+    if not total > 0.0:
+        return 0
+    return min(len(s), int(np.searchsorted(csum, float(mass_fraction) * total, side="left")) + 1)
 
 
 # ----------------------------------------------------------------------------
@@ -434,6 +453,35 @@ def attn_block(u, positions, prm, rnd=_identity):
     o = rnd(attention_forward(q, k, v, scale))
     out = rnd(u + o.reshape(T, Hq * d) @ _f64(prm["W_o"]))
     return out, dict(q=q, k=k, v=v, o=o, scale=scale)
+
+
+def attn_block_projections(u, positions, prm, rnd=_identity):
+    """The first half of attn_block: q, k (after the rotary embedding) and v of every row.  Returns dict(q, k, v, scale)."""
+    Hq, Hkv, d = prm["Hq"], prm["Hkv"], prm["d"]
+    u = _f64(u)
+    T = u.shape[0]
+    normed = rnd(rmsnorm(u))
+    qkv = rnd(normed @ _f64(prm["W_qkv"]))
+    q = qkv[:, :Hq * d].reshape(T, Hq, d)
+    k = qkv[:, Hq * d:(Hq + Hkv) * d].reshape(T, Hkv, d)
+    v = qkv[:, (Hq + Hkv) * d:].reshape(T, Hkv, d)
+    q = rnd(rope(q, positions, prm["theta"]))
+    k = rnd(rope(k, positions, prm["theta"]))
+    return dict(q=q, k=k, v=v, scale=1.0 / np.sqrt(d))
+
+
+def attn_block_rows(u, positions, prm, rows, rnd=_identity, mid=None):
+    """attn_block for a sequence too long to evaluate every row on the CPU: q, k, v are computed for every row (or
+    taken from ``mid`` = attn_block_projections of the same input), the attention output and the layer output only
+    for ``rows``.  Returns (layer output rows [len(rows), D], mid)."""
+    Hq, d = prm["Hq"], prm["d"]
+    u = _f64(u)
+    if mid is None:
+        mid = attn_block_projections(u, positions, prm, rnd)
+    rows = [int(r) for r in rows]
+    o = rnd(attention_rows(mid["q"], mid["k"], mid["v"], mid["scale"], rows))
+    out = rnd(u[rows] + o.reshape(len(rows), Hq * d) @ _f64(prm["W_o"]))
+    return out, mid
 
 
 def ffn_block(u, prm, rnd=_identity):

@@ -62,7 +62,8 @@ class StackIO(ctypes.Structure):
 PROF_CATEGORIES = ["gemm", "ssd_scan", "mamba_score", "attn_score", "topk", "compact", "attn_fwd", "elementwise"]
 
 EXPORTS = [
-    "str_create", "str_destroy", "str_strerror", "str_check_status", "str_launch_count",
+    "str_create", "str_destroy", "str_strerror", "str_check_status", "str_launch_count", "str_path_counts",
+    "str_selftest_wait_timeout", "str_score_density", "str_schedule_keep_counts_layers",
     "str_profile_enable", "str_profile_collect",
     "str_mamba2_prefill_workspace_size", "str_mamba2_prefill",
     "str_mamba_importance_workspace_size", "str_mamba_importance",
@@ -160,6 +161,15 @@ class Context:
 
     def launch_count(self):
         return int(lib().str_launch_count(self._h))
+
+    def path_counts(self):
+        """(calls that ran a tensor-core kernel, calls that fell back to the fp32-FMA kernel)."""
+        tc, fb = ctypes.c_longlong(), ctypes.c_longlong()
+        _check(lib().str_path_counts(self._h, ctypes.byref(tc), ctypes.byref(fb)), "str_path_counts")
+        return int(tc.value), int(fb.value)
+
+    def selftest_wait_timeout(self, probe_limit=1000):
+        _check(lib().str_selftest_wait_timeout(self._h, ctypes.c_uint(probe_limit), _stream()), "str_selftest_wait_timeout")
 
     def profile_enable(self, on=True):
         _check(lib().str_profile_enable(self._h, c_int(1 if on else 0)), "str_profile_enable")
@@ -279,6 +289,29 @@ def str_schedule_keep_counts(alpha_bp, n0, min_keep):
     out = (c_int * L)()
     _check(lib().str_schedule_keep_counts(a, c_int(L), c_int(n0), c_int(min_keep), out), "str_schedule_keep_counts")
     return list(out)
+
+
+LAYER_KIND = {"M": STR_LAYER_MAMBA, "A": STR_LAYER_ATTN, "F": STR_LAYER_FFN}
+
+
+def str_schedule_keep_counts_layers(alpha_bp, pattern, n0, min_keep):
+    """Keep counts for a stack whose layer kinds are given as a string of M / A / F: FFN layers never reduce."""
+    L = len(alpha_bp)
+    assert len(pattern) == L
+    a = (c_int * L)(*[int(v) for v in alpha_bp])
+    kinds = (c_int * L)(*[LAYER_KIND[c] for c in pattern])
+    out = (c_int * L)()
+    _check(lib().str_schedule_keep_counts_layers(a, kinds, c_int(L), c_int(n0), c_int(min_keep), out),
+           "str_schedule_keep_counts_layers")
+    return list(out)
+
+
+def str_score_density(ctx, scores, mass_fraction):
+    Bz, n_vis = scores.shape
+    out = torch.empty((Bz,), dtype=torch.int32, device=scores.device)
+    _check(lib().str_score_density(ctx.handle, c_int(Bz), c_int(n_vis), _p(scores), c_float(mass_fraction), _p(out), _stream()),
+           "str_score_density")
+    return out
 
 
 def str_sigmoid_schedule_bp(L, k, x0, a_start, a_end):
@@ -447,10 +480,10 @@ def str_stack_prefill(stack, hidden_in, want_trace=False):
     return out, pos, idx, trace
 
 
-def str_stack_prefill_ex(stack, hidden_in, positions_in=None, idx_map_in=None, want_handoff=False):
+def str_stack_prefill_ex(stack, hidden_in, positions_in=None, idx_map_in=None, want_handoff=False, want_trace=False):
     """str_stack_prefill with the optional inputs (original token ids of the incoming rows) and, with
     ``want_handoff``, the decoder hand-off outputs: the final state of every Mamba layer and the keys, values and
-    positions of the rows leaving every attention layer.  Returns a dict."""
+    positions of the rows leaving every attention layer.  Returns a dict (``trace`` as in str_stack_prefill)."""
     ctx = stack.ctx
     T_out = stack.K_last + stack.n_text
     out = torch.empty((stack.Bz, T_out, stack.D), dtype=stack.tdt, device=stack.dev)
@@ -470,11 +503,23 @@ def str_stack_prefill_ex(stack, hidden_in, positions_in=None, idx_map_in=None, w
             v_all = torch.empty_like(k_all)
             p_all = torch.empty((sum(rows_a),), dtype=torch.int32, device=stack.dev)
     io = StackIO(_p(positions_in), _p(idx_map_in), _p(fs_all), _p(k_all), _p(v_all), _p(p_all))
+    kept_tr = score_tr = None
+    if want_trace and stack.trace_layout:
+        kept_tr = torch.empty(sum(stack.Bz * K for _, _, K in stack.trace_layout), dtype=torch.int32, device=stack.dev)
+        score_tr = torch.empty(sum(stack.Bz * n for _, n, _ in stack.trace_layout), dtype=torch.float32, device=stack.dev)
     ws = ctx.workspace(stack.ws_bytes)
     _check(lib().str_stack_prefill_ex(ctx.handle, ctypes.byref(stack.desc), ctypes.byref(io), _p(hidden_in), _p(out), _p(pos),
-                                      _p(idx), _p(None), _p(None), _p(ws), c_size_t(ws.numel()), _stream()),
+                                      _p(idx), _p(kept_tr), _p(score_tr), _p(ws), c_size_t(ws.numel()), _stream()),
            "str_stack_prefill_ex")
     res = dict(hidden=out, positions=pos, idx_map=idx)
+    if want_trace:
+        trace, ko, so = [], 0, 0
+        for l, n_in, K in stack.trace_layout:
+            trace.append(dict(layer=l, n_in=n_in, kept=kept_tr[ko:ko + stack.Bz * K].view(stack.Bz, K),
+                              scores=score_tr[so:so + stack.Bz * n_in].view(stack.Bz, n_in)))
+            ko += stack.Bz * K
+            so += stack.Bz * n_in
+        res["trace"] = trace
     if want_handoff:
         mi, ro = 0, 0
         for l, k in enumerate(kinds):

@@ -31,9 +31,9 @@ extern "C" int str_mamba2_prefill(str_ctx *ctx, const str_ssd_shape *s, const vo
     if (workspace_bytes < str_mamba2_prefill_workspace_size(s)) return STR_ERR_WORKSPACE_TOO_SMALL;
     if (s->T == 0) return STR_OK;
     if (!str_force_simt() && ctx->encode_tiled && str_ssd_tc_supported(s, x, B, C, y, D, init_state))
-        return str_ssd_tc(ctx, s, x, dt, A, B, C, y, final_state, (cudaStream_t)stream);
+        return ++ctx->tc_calls, str_ssd_tc(ctx, s, x, dt, A, B, C, y, final_state, (cudaStream_t)stream);
     if (!str_ssd_simt_supported(s)) return STR_ERR_UNSUPPORTED_SHAPE;
-    return str_ssd_simt(ctx, s, x, dt, A, B, C, D, init_state, y, final_state, (cudaStream_t)stream);
+    return ++ctx->fallback_calls, str_ssd_simt(ctx, s, x, dt, A, B, C, D, init_state, y, final_state, (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------- (2a) Mamba importance
@@ -54,8 +54,8 @@ extern "C" int str_mamba_importance(str_ctx *ctx, const str_ssm_score_shape *s, 
     if (n_vis == 0) return STR_OK;
     if (!scores_out) return STR_ERR_INVALID_ARG;
     if (!str_force_simt() && ctx->encode_tiled && str_mamba_importance_tc_supported(s, n_vis, n_text, B, C))
-        return str_mamba_importance_tc(ctx, s, n_vis, n_text, B, C, dt, scores_out, (cudaStream_t)stream);
-    return str_mamba_importance_simt(ctx, s, n_vis, n_text, B, C, dt, scores_out, (cudaStream_t)stream);
+        return ++ctx->tc_calls, str_mamba_importance_tc(ctx, s, n_vis, n_text, B, C, dt, scores_out, (cudaStream_t)stream);
+    return ++ctx->fallback_calls, str_mamba_importance_simt(ctx, s, n_vis, n_text, B, C, dt, scores_out, (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------- (2a') Mamba importance with the cumulative decay
@@ -93,6 +93,7 @@ extern "C" int str_mamba_importance_dynamic(str_ctx *ctx, const str_ssm_score_sh
     uint8_t *U = (uint8_t *)workspace + str_mamba_dyn_part_bytes(s, n_vis), *V = U + u_bytes;
     int rc = str_mamba_dyn_weights(ctx, s, n_vis, n_text, n_pad, dt, A, part, U, V, tc, (cudaStream_t)stream);
     if (rc != STR_OK) return rc;
+    ++(tc ? ctx->tc_calls : ctx->fallback_calls);
     if (tc) return str_mamba_dyn_importance_tc(ctx, s, n_vis, n_text, B, C, U, V, scores_out, (cudaStream_t)stream);
     return str_mamba_dyn_importance_simt(ctx, s, n_vis, n_text, B, C, (const float *)U, (const float *)V, scores_out,
                                          (cudaStream_t)stream);
@@ -120,8 +121,9 @@ extern "C" int str_attn_importance_ex(str_ctx *ctx, const str_attn_score_shape *
     if (workspace_bytes < str_attn_importance_workspace_size(s, n_vis, n_text)) return STR_ERR_WORKSPACE_TOO_SMALL;
     const bool causal_row = denominator == STR_ATTN_DENOM_CAUSAL_ROW;
     if (!str_force_simt() && ctx->encode_tiled && str_attn_importance_tc_supported(s, n_vis, n_text, q, k))
-        return str_attn_importance_tc(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, (float *)workspace, causal_row,
-                                      (cudaStream_t)stream);
+        return ++ctx->tc_calls, str_attn_importance_tc(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, (float *)workspace,
+                                                       causal_row, (cudaStream_t)stream);
+    ++ctx->fallback_calls;
     float *row_max = (float *)workspace;
     float *row_sum = row_max + (size_t)s->Bz * s->Hq * n_text;
     return str_attn_importance_simt(ctx, s, n_vis, n_text, q, k, softmax_scale, scores_out, row_max, row_sum, causal_row,
@@ -145,8 +147,8 @@ extern "C" int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void
     if (!ctx || !a || !w || !out || M < 0 || N <= 0 || K <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
     if (M == 0) return STR_OK;
     if (!str_force_simt() && ctx->encode_tiled && str_gemm_tc_supported(dtype, M, N, K, a, w, residual, out))
-        return str_gemm_tc(ctx, M, N, K, a, w, residual, out, (cudaStream_t)stream);
-    return str_gemm_simt(ctx, dtype, M, N, K, a, w, residual, out, (cudaStream_t)stream);
+        return ++ctx->tc_calls, str_gemm_tc(ctx, M, N, K, a, w, residual, out, (cudaStream_t)stream);
+    return ++ctx->fallback_calls, str_gemm_simt(ctx, dtype, M, N, K, a, w, residual, out, (cudaStream_t)stream);
 }
 
 extern "C" size_t str_attn_prefill_workspace_size(const str_attn_shape *) { return 0; }
@@ -161,6 +163,6 @@ extern "C" int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const voi
         !STR_DTYPE_OK(s->dtype))
         return STR_ERR_INVALID_ARG;
     if (!str_force_simt() && ctx->encode_tiled && str_attn_prefill_tc_supported(s, q, k, v, o))
-        return str_attn_prefill_tc(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
-    return str_attn_prefill_simt(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
+        return ++ctx->tc_calls, str_attn_prefill_tc(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
+    return ++ctx->fallback_calls, str_attn_prefill_simt(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
 }

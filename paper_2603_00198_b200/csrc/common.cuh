@@ -22,6 +22,8 @@ struct str_ctx {
     int *status_dev;          // device status word: 0 or the first STR_ERR_* a kernel recorded
     void *encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), or nullptr
     long long launches;       // host-side count of kernels launched through this context
+    long long tc_calls;       // entry-point calls that took a tensor-core (tcgen05) kernel
+    long long fallback_calls; // entry-point calls that took the plain fp32-FMA kernel of the same entry point
     size_t smem_attr[8];      // dynamic shared memory already opted into on this device, per tensor-core kernel
     cudaStream_t copy_stream; // host-buffer entry point: input chunks are copied on this stream while the caller's
     cudaEvent_t copy_ev[8];   // stream computes; [0] orders the copies after the caller's earlier work, [1..] = chunk landed

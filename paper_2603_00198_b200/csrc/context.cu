@@ -14,6 +14,8 @@ extern "C" int str_create(int device, str_ctx **out) {
     if (!c) return STR_ERR_CUDA;
     c->device = device;
     c->launches = 0;
+    c->tc_calls = 0;
+    c->fallback_calls = 0;
     c->prof_on = false;
     for (size_t &v : c->smem_attr) v = 0;
     c->copy_stream = nullptr;
@@ -31,6 +33,13 @@ extern "C" int str_create(int device, str_ctx **out) {
         qres == cudaDriverEntryPointSuccess)
         c->encode_tiled = fn;
     (void)cudaGetLastError();
+    if (!c->encode_tiled) {
+        // Without the tensor-map encoder no tensor-core kernel can be launched.  Every call would quietly take the
+        // fp32-FMA kernels, many times slower: refuse to create the context instead.
+        cudaFree(c->status_dev);
+        delete c;
+        return STR_ERR_CUDA;
+    }
     *out = c;
     return STR_OK;
 }
@@ -96,6 +105,13 @@ extern "C" int str_profile_collect(str_ctx *ctx, double *ms_by_category, long lo
 
 extern "C" long long str_launch_count(const str_ctx *ctx) { return ctx ? ctx->launches : -1; }
 
+extern "C" int str_path_counts(const str_ctx *ctx, long long *tensor_core_calls, long long *fallback_calls) {
+    if (!ctx || !tensor_core_calls || !fallback_calls) return STR_ERR_INVALID_ARG;
+    *tensor_core_calls = ctx->tc_calls;
+    *fallback_calls = ctx->fallback_calls;
+    return STR_OK;
+}
+
 // Section 3.2 / appendix schedules: alpha is a fraction of the original visual count.
 extern "C" int str_schedule_keep_counts(const int *alpha_bp, int L, int n0, int min_keep, int *K_out) {
     if (!alpha_bp || !K_out || L < 0 || n0 < 0 || min_keep < 0) return STR_ERR_INVALID_ARG;
@@ -107,6 +123,23 @@ extern "C" int str_schedule_keep_counts(const int *alpha_bp, int L, int n0, int 
         if (k > n_cur) k = n_cur;
         K_out[l] = (int)k;
         n_cur = k;
+    }
+    return STR_OK;
+}
+
+// Same with the layer kinds known: FFN layers only transform the rows they are given, so a cut that the schedule
+// places on one is taken by the next Mamba / attention layer (the paper's all-layer schedules cut at those).
+extern "C" int str_schedule_keep_counts_layers(const int *alpha_bp, const int *layer_kinds, int L, int n0, int min_keep,
+                                               int *K_out) {
+    if (!layer_kinds) return STR_ERR_INVALID_ARG;
+    int rc = str_schedule_keep_counts(alpha_bp, L, n0, min_keep, K_out);
+    if (rc != STR_OK) return rc;
+    int n_cur = n0;
+    for (int l = 0; l < L; ++l) {
+        if (layer_kinds[l] != STR_LAYER_MAMBA && layer_kinds[l] != STR_LAYER_ATTN && layer_kinds[l] != STR_LAYER_FFN)
+            return STR_ERR_INVALID_ARG;
+        if (layer_kinds[l] != STR_LAYER_FFN && K_out[l] < n_cur) n_cur = K_out[l];
+        K_out[l] = n_cur;
     }
     return STR_OK;
 }

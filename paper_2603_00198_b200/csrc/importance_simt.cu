@@ -7,6 +7,8 @@
 #include <float.h>
 
 #include "common.cuh"
+#include <atomic>
+
 #include "dispatch.cuh"
 
 namespace {
@@ -262,7 +264,9 @@ static __device__ __align__(256) float g_attn_static_rowstats[2 * STR_ATTN_STATI
 
 namespace {
 constexpr int kMaxDevices = 64;
-float *g_rowstats_dev_ptr[kMaxDevices] = {};   // device address of the array, per device (host cache)
+// device address of the array, per device (host cache; contexts on several host threads may race to fill an entry,
+// and every one of them stores the same value)
+std::atomic<float *> g_rowstats_dev_ptr[kMaxDevices];
 }  // namespace
 
 extern "C" int str_attn_importance_static(str_ctx *ctx, const str_attn_score_shape *s, int n_vis, int n_text,
@@ -278,7 +282,7 @@ extern "C" int str_attn_importance_static(str_ctx *ctx, const str_attn_score_sha
     if (n_vis == 0) return STR_OK;
     if (!scores_out) return STR_ERR_INVALID_ARG;
     if (ctx->device < 0 || ctx->device >= kMaxDevices) return STR_ERR_INVALID_ARG;
-    float *base = g_rowstats_dev_ptr[ctx->device];
+    float *base = g_rowstats_dev_ptr[ctx->device].load(std::memory_order_acquire);
     if (!base) {
         // One-time set-up per device: in host code the array's name is only a stand-in, so ask the
         // runtime for its device address, with the context's device current.
@@ -288,9 +292,12 @@ extern "C" int str_attn_importance_static(str_ctx *ctx, const str_attn_score_sha
         void *sym = nullptr;
         const cudaError_t e = cudaGetSymbolAddress(&sym, g_attn_static_rowstats);
         if (prev != ctx->device) cudaSetDevice(prev);
-        if (e != cudaSuccess || !sym) return STR_ERR_CUDA;
+        if (e != cudaSuccess || !sym) {
+            (void)cudaGetLastError();             // do not leave the runtime's sticky error for an unrelated later call
+            return STR_ERR_CUDA;
+        }
         base = (float *)sym;
-        g_rowstats_dev_ptr[ctx->device] = base;
+        g_rowstats_dev_ptr[ctx->device].store(base, std::memory_order_release);
     }
     // Both halves are fully rewritten by the first pass before the second pass reads them, so nothing
     // left over from an earlier call is ever used and nothing needs clearing.

@@ -101,3 +101,54 @@ def test_compact_rejects_bad_arguments(ctx):
     with pytest.raises(binding.StrError):       # row not a multiple of 16 bytes
         binding.str_compact(ctx, dev(inputs.hidden_inputs(23, 10, 3, "f32")), None, None,
                             torch.zeros((1, 2), dtype=torch.int32, device="cuda"), 2)
+
+
+@pytest.mark.parametrize("kind", ["uniform", "heavy", "ties", "equal", "ascending"])
+@pytest.mark.parametrize("n", [1, 100, 4096, 32768, 100003])
+def test_score_density_matches_the_full_sort(ctx, kind, n):
+    """Tokens needed for a share of the importance mass (the paper's sparsity statistic), against sort + cumulative sum."""
+    s = inputs.score_vectors(44, n, kind, batch=3)
+    s[2] = 0.0                                                      # one all-zero row
+    for frac in (0.8, 0.5, 1.0):
+        got = binding.str_score_density(ctx, dev(s), frac).cpu().numpy()
+        for b in range(3):
+            want = oracle.score_density(s[b], np.float32(frac))
+            if kind in ("ties", "equal"):
+                # many equal scores at the threshold: the count of copies still needed is a quotient on the GPU and a
+                # running sum in the oracle, which may round differently exactly at a boundary
+                assert abs(int(got[b]) - want) <= 1, (kind, n, frac, b)
+            else:
+                assert int(got[b]) == want, (kind, n, frac, b)
+    hot = np.zeros((1, max(n, 2)), dtype=np.float32)
+    hot[0, n // 2] = 2.5
+    assert int(binding.str_score_density(ctx, dev(hot), 0.8).cpu().numpy()[0]) == 1
+
+
+def test_bounded_wait_gives_up_and_the_status_word_reports_it_once(ctx):
+    """Every pipelined kernel of the library waits on its barriers with a probe limit and, on giving up, records
+    STR_ERR_TIMEOUT in the context's status word.  The self-test kernel makes such a wait run out (a barrier that
+    nobody signals): the next status check reports the timeout, the one after it is clean, and the context works."""
+    ctx.check_status()
+    ctx.selftest_wait_timeout(1000)
+    with pytest.raises(binding.StrError) as e:
+        ctx.check_status()
+    assert e.value.code == -5
+    ctx.check_status()                                              # cleared by the read
+    s = inputs.score_vectors(45, 5000, "uniform")
+    kept = binding.str_topk_select(ctx, dev(s), 1250).cpu().numpy()[0]
+    assert np.array_equal(kept, oracle.topk_select(s[0], 1250))
+    ctx.check_status()
+
+
+def test_path_counters_tell_tensor_core_from_fallback_calls(ctx):
+    """A shape the tensor-core scan tiles and one it does not: the context counts which path each call took."""
+    tc0, fb0 = ctx.path_counts()
+    d = inputs.ssd_inputs(46, 300, 4, 64, 128, 2, "bf16")
+    binding.str_mamba2_prefill(ctx, dev(d["x"], "bf16"), dev(d["dt"]), dev(d["A"]), dev(d["B"], "bf16"), dev(d["C"], "bf16"))
+    tc1, fb1 = ctx.path_counts()
+    assert (tc1 - tc0, fb1 - fb0) == (1, 0)
+    d = inputs.ssd_inputs(46, 300, 4, 16, 32, 2, "f32")
+    binding.str_mamba2_prefill(ctx, dev(d["x"]), dev(d["dt"]), dev(d["A"]), dev(d["B"]), dev(d["C"]))
+    tc2, fb2 = ctx.path_counts()
+    assert (tc2 - tc1, fb2 - fb1) == (0, 1)
+    ctx.check_status()

@@ -138,3 +138,36 @@ def test_stack_with_ffn_layers_keeps_the_row_set():
     np.testing.assert_allclose(oracle.ffn_block(h1[rows], layers[1][1]), oracle.ffn_block(h1, layers[1][1])[rows], rtol=1e-13)
     with pytest.raises(AssertionError):
         oracle.stack_prefill(h0, M, layers, [12, 6, 6, 6])          # an FFN layer may not reduce
+
+
+def test_attn_block_rows_and_resumed_stack_agree_with_the_whole_computation():
+    """Two conveniences of the oracle used by the large GPU parity tests: the attention block evaluated for a few
+    rows only, and a stack continued from a reduced context (carried ids passed in) with its trace of layer
+    inputs.  Both must reproduce the plain whole-sequence run."""
+    from paper_2603_00198_b200 import inputs
+    ms = dict(D=32, H=4, p=8, n=8, G=2, Q=16, conv=4)
+    at = dict(D=32, Hq=4, Hkv=2, d=8, theta=1.0e6)
+    layers = inputs.stack_params(15, "MAMA", ms, at, "f32")
+    n_vis, M = 40, 6
+    h0 = inputs.hidden_inputs(15, n_vis + M, 32, "f32")[0]
+    pos = np.arange(n_vis + M) * 3 + 1                          # arbitrary ascending positions
+    full, mid = oracle.attn_block(h0, pos, layers[1][1])
+    rows = [0, 5, 17, n_vis + M - 1]
+    part, mid_r = oracle.attn_block_rows(h0, pos, layers[1][1], rows)
+    np.testing.assert_allclose(part, full[rows], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(mid_r["k"], mid["k"], rtol=0, atol=0)
+    # whole run with a trace of layer inputs; layers 2.. re-run from the stored input of layer 2 give the same result
+    K = [n_vis, 20, 20, 10]
+    out, opos, oidx, trace = oracle.stack_prefill(h0, M, layers, K, keep_inputs=True)
+    rec = trace[2]
+    assert rec["n_in"] == 20 and rec["hidden_in"].shape == (20 + M, 32)
+    out2, pos2, idx2, trace2 = oracle.stack_prefill(rec["hidden_in"], M, layers[2:], K[2:], positions=rec["positions_in"],
+                                                    idx_map=rec["idx_map_in"])
+    np.testing.assert_array_equal(out2, out)
+    np.testing.assert_array_equal(idx2, oidx)
+    np.testing.assert_array_equal(pos2, opos)
+    # hand-off records: a Mamba layer's final state is the recurrence's, an attention layer's keys are those of the
+    # rows that leave it, with their original positions
+    assert trace[0]["final_state"].shape == (4, 8, 8) and trace[1]["k"].shape == (20 + M, 2, 8)
+    np.testing.assert_array_equal(trace[1]["kv_positions"], trace[2]["positions_in"])
+    np.testing.assert_array_equal(trace[3]["kv_positions"], opos)

@@ -101,3 +101,50 @@ def test_sigmoid_schedule_shape():
     assert np.all(np.diff(a) < 0) and a[0] > 0.99 and abs(a[-1] - 0.125) < 1e-4
     mid = oracle.sigmoid_schedule(100, 20.0, 0.5, 1.0, 0.125)[50]
     np.testing.assert_allclose(mid, 0.125 + 0.875 * 0.5, rtol=1e-12)
+
+
+def test_score_density_closed_forms_and_brute_force():
+    """The sparsity statistic (Section 2: tokens needed for a given share of the importance mass)."""
+    # uniform vector: ceil(frac n) tokens (values a power of two so that every partial sum is exact)
+    for n, frac, want in ((10, 0.8, 8), (10, 0.5, 5), (1000, 0.801, 801), (7, 1.0, 7)):
+        assert oracle.score_density(np.full(n, 0.25), frac) == want
+    # all mass on one token; nothing at all
+    onehot = np.zeros(50); onehot[17] = 3.0
+    assert oracle.score_density(onehot, 0.8) == 1 and oracle.score_density(onehot, 1.0) == 1
+    assert oracle.score_density(np.zeros(9), 0.8) == 0
+    # two levels: h heavy tokens of weight 8 and l light tokens of weight 1 -> mass 8h + l
+    h, l = 4, 32                                           # total 64; 80% = 51.2 -> 4 heavy (32) + 20 light
+    v = np.concatenate([np.ones(l), np.full(h, 8.0)])
+    assert oracle.score_density(v, 0.8) == 24 and oracle.score_density(v, 0.5) == 4 and oracle.score_density(v, 0.51) == 5
+    # order of the input does not matter; brute force over prefixes of the sorted vector
+    r = np.random.default_rng(12)
+    for _ in range(20):
+        s = r.exponential(size=r.integers(1, 40))
+        frac = r.uniform(0.05, 1.0)
+        srt = sorted(s, reverse=True)
+        want = next(k for k in range(1, len(s) + 1) if sum(srt[:k]) >= frac * sum(srt) - 1e-15)
+        assert oracle.score_density(r.permutation(s), frac) == want
+    # a heavy-tailed vector is denser than a flat one (the paper's 10.9% against 30.6% contrast, in kind)
+    flat = r.uniform(0.5, 1.0, size=4096)
+    peaky = flat * 1e-2
+    peaky[r.choice(4096, size=400, replace=False)] += r.exponential(1.0, size=400)
+    assert oracle.score_density(peaky, 0.8) < 0.2 * 4096 < oracle.score_density(flat, 0.8)
+
+
+def test_ffn_layers_never_reduce_in_the_schedule():
+    """With layer kinds given, a cut that the schedule places on an FFN layer moves to the next Mamba / attention layer."""
+    alpha = [10000, 5000, 5000, 2500, 2500, 1000]
+    plain = oracle.schedule_keep_counts(alpha, 1000, 0)
+    assert plain == [1000, 500, 500, 250, 250, 100]
+    assert oracle.schedule_keep_counts(alpha, 1000, 0, "MAMAMA") == plain              # no FFN layer: unchanged
+    got = oracle.schedule_keep_counts(alpha, 1000, 0, "MFAFMF")
+    assert got == [1000, 1000, 500, 500, 250, 250]
+    # an FFN layer's count equals its incoming count; every other layer takes the schedule's own value
+    n_cur = 1000
+    for kind, k, p in zip("MFAFMF", got, plain):
+        assert k == (n_cur if kind == "F" else min(n_cur, p))
+        n_cur = k
+    # the library's helper is the same rule
+    from paper_2603_00198_b200 import binding
+    for pattern in ("MFAFMF", "FFMAMA", "MAMAMA", "AFAFAF"):
+        assert binding.str_schedule_keep_counts_layers(alpha, pattern, 1000, 16) == oracle.schedule_keep_counts(alpha, 1000, 16, pattern)
