@@ -306,6 +306,23 @@ def run_ours(args):
     ms_total = ev0.elapsed_time(ev1)
     ctx.profile_enable(False)
     prof = ctx.profile_collect()
+    ms_graph = None
+    if args.graph:
+        # the same step captured once into a CUDA graph and replayed: the stack call only enqueues kernels and
+        # device-to-device copies on the caller's stream, so it can be captured after a warm-up call
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            g_out, g_pos, g_idx = binding.str_stack_prefill(stack, h_dev)
+        gr.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(args.steps):
+            gr.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        ms_graph = g0.elapsed_time(g1) / args.steps
+        assert bool((g_out == out).all()) and bool((g_idx == idx).all())
     launches = ctx.launch_count() - l0
     tc1, fb1 = ctx.path_counts()
     clocks = sampler.stop() if sampler else None
@@ -407,6 +424,7 @@ def run_ours(args):
                 "d2h_bytes_per_step": int(out_pin.numel() * 2 + idx_pin.numel() * 4), "matches_device_run": same},
         "gpu_launches": int(launches), "clocks": clocks, "kernels": kernels,
         "paths": {"tensor_core_calls": int(tc1 - tc0), "fallback_calls": int(fb1 - fb0)},
+        "ms_per_step_cuda_graph": ms_graph,
         "kernels_alone": alone,
     }
     print(json.dumps(line))
@@ -569,6 +587,7 @@ def main():
                     help="normaliser of the attention-layer importance: visual keys only (the paper's formula) or the causal row")
     ap.add_argument("--x0", type=float, default=0.11, help="midpoint of the sigmoid schedule (0.11 / 0.24 / 0.41)")
     ap.add_argument("--micro-seconds", type=float, default=0.6, help="repeat a --micro launch for at least this long (clock sampling)")
+    ap.add_argument("--graph", action="store_true", help="also time the step replayed from a CUDA graph")
     ap.add_argument("--no-kernels-alone", action="store_true", help="skip the per-kernel timings after the headline run")
     ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | mamba_dyn_score | attn_score | attn_fwd | "
                                                 "topk | compact | gemm")

@@ -245,6 +245,16 @@ int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const void *q, const
                      const void *v, float softmax_scale, void *o, void *workspace,
                      size_t workspace_bytes, void *stream);
 
+/* The same attention for a gathered subset of the query rows (a layer that has selected its survivors before the
+ * attention only needs their outputs; every incoming key and value is still attended to).  q_rows, o_rows device
+ * [Bz,n_rows,Hq,d]; row_pos device [Bz,n_rows] int32, strictly ascending: the index of each query row in the key
+ * sequence (row r attends to keys 0 .. row_pos[r]); NULL means rows 0 .. n_rows-1 with n_rows == T.  k, v device
+ * [Bz,T,Hkv,d].  A row's output does not depend on which other rows are passed with it: it is bit-identical to the
+ * row str_attn_prefill computes. */
+int str_attn_prefill_rows(str_ctx *ctx, const str_attn_shape *s, int n_rows, const void *q_rows, const int32_t *row_pos,
+                          const void *k, const void *v, float softmax_scale, void *o_rows, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * Whole stack: token-reduced prefill with a per-layer keep schedule (Sections 3.1-3.2).
  * Layer l's mixer runs on the incoming tokens, its own importance score ranks the incoming

@@ -72,7 +72,7 @@ EXPORTS = [
     "str_topk_select_workspace_size", "str_topk_select", "str_compact",
     "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
     "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_relu_squared", "str_mamba_conv_split", "str_gated_rmsnorm",
-    "str_rope_split", "str_attn_prefill_workspace_size", "str_attn_prefill",
+    "str_rope_split", "str_attn_prefill_workspace_size", "str_attn_prefill", "str_attn_prefill_rows",
     "str_stack_workspace_size", "str_stack_prefill", "str_stack_prefill_ex", "str_stack_host_workspace_size",
     "str_stack_prefill_host",
 ]
@@ -389,6 +389,19 @@ def str_attn_prefill(ctx, q, k, v, softmax_scale):
     ws = ctx.workspace(nb)
     _check(lib().str_attn_prefill(ctx.handle, ctypes.byref(s), _p(q), _p(k), _p(v), c_float(softmax_scale), _p(o),
                                   _p(ws), c_size_t(ws.numel()), _stream()), "str_attn_prefill")
+    return o
+
+
+def str_attn_prefill_rows(ctx, q_rows, row_pos, k, v, softmax_scale):
+    """Attention outputs of a gathered subset of query rows: q_rows [Bz,n_rows,Hq,d], row_pos [Bz,n_rows] int32."""
+    Bz, n_rows, Hq, d = q_rows.shape
+    T, Hkv = k.shape[1], k.shape[2]
+    s = AttnShape(Bz, T, Hq, Hkv, d, _dt(q_rows))
+    o = torch.empty_like(q_rows)
+    ws = ctx.workspace(256)
+    _check(lib().str_attn_prefill_rows(ctx.handle, ctypes.byref(s), c_int(n_rows), _p(q_rows), _p(row_pos), _p(k), _p(v),
+                                       c_float(softmax_scale), _p(o), _p(ws), c_size_t(ws.numel()), _stream()),
+           "str_attn_prefill_rows")
     return o
 
 

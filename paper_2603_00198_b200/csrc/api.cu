@@ -153,16 +153,24 @@ extern "C" int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void
 
 extern "C" size_t str_attn_prefill_workspace_size(const str_attn_shape *) { return 0; }
 
+extern "C" int str_attn_prefill_rows(str_ctx *ctx, const str_attn_shape *s, int n_rows, const void *q_rows,
+                                     const int32_t *row_pos, const void *k, const void *v, float softmax_scale,
+                                     void *o_rows, void *workspace, size_t workspace_bytes, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ATTN_FWD, stream);
+    (void)workspace; (void)workspace_bytes;
+    if (!ctx || !s || !q_rows || !k || !v || !o_rows) return STR_ERR_INVALID_ARG;
+    if (s->Bz <= 0 || s->T <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Hq % s->Hkv != 0 || s->d <= 0 || n_rows < 0 ||
+        !STR_DTYPE_OK(s->dtype) || (!row_pos && n_rows != s->T))
+        return STR_ERR_INVALID_ARG;
+    if (n_rows == 0) return STR_OK;
+    if (!str_force_simt() && ctx->encode_tiled && str_attn_prefill_tc_supported(s, q_rows, k, v, o_rows))
+        return ++ctx->tc_calls, str_attn_prefill_tc(ctx, s, n_rows, q_rows, row_pos, k, v, softmax_scale, o_rows, (cudaStream_t)stream);
+    return ++ctx->fallback_calls, str_attn_prefill_simt(ctx, s, n_rows, q_rows, row_pos, k, v, softmax_scale, o_rows, (cudaStream_t)stream);
+}
+
 extern "C" int str_attn_prefill(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v,
                                 float softmax_scale, void *o, void *workspace, size_t workspace_bytes,
                                 void *stream) {
-    StrProfScope prof_scope(ctx, STR_CAT_ATTN_FWD, stream);
-    (void)workspace; (void)workspace_bytes;
-    if (!ctx || !s || !q || !k || !v || !o) return STR_ERR_INVALID_ARG;
-    if (s->Bz <= 0 || s->T <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Hq % s->Hkv != 0 || s->d <= 0 ||
-        !STR_DTYPE_OK(s->dtype))
-        return STR_ERR_INVALID_ARG;
-    if (!str_force_simt() && ctx->encode_tiled && str_attn_prefill_tc_supported(s, q, k, v, o))
-        return ++ctx->tc_calls, str_attn_prefill_tc(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
-    return ++ctx->fallback_calls, str_attn_prefill_simt(ctx, s, q, k, v, softmax_scale, o, (cudaStream_t)stream);
+    if (!s) return STR_ERR_INVALID_ARG;
+    return str_attn_prefill_rows(ctx, s, s->T, q, nullptr, k, v, softmax_scale, o, workspace, workspace_bytes, stream);
 }

@@ -16,6 +16,11 @@
 // Tensor memory (512 columns): S_0 | S_1 | O_0 | O_1, 128 columns each.
 // Warps: 0-3 softmax of tile 0, 4-7 softmax of tile 1 (warp w may touch TMEM lanes 32 (w % 4)...),
 // 8 TMA producer (Q once, then a 2-slot ring for K and one for V), 9 MMA issuer.
+// Query rows may be a gathered subset of the sequence (a layer that has already selected its survivors only needs
+// their outputs): row r then carries its index t_r in the key sequence (ascending), attends to keys <= t_r, and a
+// query tile walks the key tiles up to the one holding its last row's index.  Everything that decides a row's
+// arithmetic (its mask, when its running maximum is raised) depends on that row alone, so a row's output does not
+// depend on which other rows share its tile: gathered and ungathered calls give bit-identical rows.
 // Every mbarrier wait is bounded; a give-up records STR_ERR_TIMEOUT and the CTA tears down.
 #include "dispatch.cuh"
 #include "tc_common.cuh"
@@ -37,8 +42,8 @@ constexpr float RESCALE_THRESHOLD = 8.0f;          // in log2 units
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                   const __grid_constant__ CUtensorMap tmap_v, int Tlen, int Hq, int Hkv, float scale_log2,
-                   __nv_bfloat16 *__restrict__ out, int *status) {
+                   const __grid_constant__ CUtensorMap tmap_v, int Tq, int Tk, int Hq, int Hkv, float scale_log2,
+                   const int32_t *__restrict__ row_pos, __nv_bfloat16 *__restrict__ out, int *status) {
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = (uint64_t *)(smem + OFF_MISC);
     uint32_t *tmem_slot = (uint32_t *)(bars + B_COUNT);
@@ -48,8 +53,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     const int pair = (int)gridDim.x - 1 - (int)blockIdx.x;        // longest rows first
     const int h = blockIdx.y, b = blockIdx.z, kv = h / (Hq / Hkv);
     const int r0 = pair * 2 * BQ;
-    const int n0 = r0 / BKV + 1;                                  // key tiles of query tile 0
-    const int n1 = (r0 + BQ < Tlen) ? n0 + 1 : n0;                // key tiles of query tile 1
+    // index in the key sequence of query row r of this sequence (rows beyond the end take the last row's)
+    const int32_t *rp = row_pos ? row_pos + (size_t)b * Tq : nullptr;
+    auto key_index = [&](int r) -> int { r = min(r, Tq - 1); return rp ? min(max(__ldg(rp + r), 0), Tk - 1) : r; };
+    const int n0 = key_index(r0 + BQ - 1) / BKV + 1;                                  // key tiles of query tile 0
+    const int n1 = (r0 + BQ < Tq) ? max(n0, key_index(r0 + 2 * BQ - 1) / BKV + 1) : n0;  // key tiles of query tile 1
 
     if ((tc::smem_u32(smem) & 1023u) != 0) {
         if (threadIdx.x == 0) atomicCAS(status, 0, STR_ERR_CUDA);
@@ -180,7 +188,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const uint32_t tS = tmem + lane_base + TM_S + (uint32_t)i * 128;
         const uint32_t tO = tmem + lane_base + TM_O + (uint32_t)i * 128;
         const int ni = i == 0 ? n0 : n1;
-        const int jd = r0 / BKV + i;                            // the diagonal key tile of this query tile
+        const int t_row = key_index(r0 + i * BQ + row);         // this row attends to keys 0 .. t_row
         float m = MASKED, l = 0.f;
         bool ok = true;
         for (int j = 0; j < ni; ++j) {
@@ -190,12 +198,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 #pragma unroll
             for (int c = 0; c < 4; ++c) tc::tmem_ld32(tS + c * 32, v[c]);
             tc::tmem_ld_wait();
-            if (j == jd) {
+            if (__any_sync(0xffffffffu, j * BKV + BKV - 1 > t_row)) {      // some row of this warp ends inside (or before) this tile
+                const int lim = t_row - j * BKV;                            // keys of this tile beyond lim are masked
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
-                        if (c * 32 + e > row) v[c][e] = __float_as_uint(MASKED);
+                        if (c * 32 + e > lim) v[c][e] = __float_as_uint(MASKED);
             }
             float tmax = MASKED;
 #pragma unroll
@@ -203,13 +212,15 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 #pragma unroll
                 for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(v[c][e]));
             const float m_new = fmaxf(m, tmax);
+            // a row raises its maximum only when it has grown by more than the threshold: a decision of the row alone
+            const bool grow = (m_new - m) * scale_log2 > RESCALE_THRESHOLD;
             if (j == 0) {
                 m = m_new;
-            } else if (__any_sync(0xffffffffu, (m_new - m) * scale_log2 > RESCALE_THRESHOLD)) {
-                // S_j complete implies the previous P V product of this tile is complete: O is stable
-                const float f = tc::ex2((m - m_new) * scale_log2);
-                l *= f;
-                m = m_new;
+            } else if (__any_sync(0xffffffffu, grow)) {
+                // S_j complete implies the previous P V product of this tile is complete: O is stable.  The whole warp
+                // runs the (warp-collective) accumulator update; rows that keep their maximum multiply by exactly 1.
+                const float f = grow ? tc::ex2((m - m_new) * scale_log2) : 1.0f;
+                if (grow) { l *= f; m = m_new; }
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -247,13 +258,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             tc::tc_fence_after();
             const int t = r0 + i * BQ + row;
             const float inv = 1.0f / l;
-            __nv_bfloat16 *dst = out + (((size_t)b * Tlen + t) * Hq + h) * HD;
+            __nv_bfloat16 *dst = out + (((size_t)b * Tq + t) * Hq + h) * HD;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
                 tc::tmem_ld32(tO + c * 32, o);
                 tc::tmem_ld_wait();
-                if (t < Tlen) {
+                if (t < Tq) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         uint4 w;
@@ -281,19 +292,19 @@ bool str_attn_prefill_tc_supported(const str_attn_shape *s, const void *q, const
     return (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15) == 0;
 }
 
-int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v, float scale,
-                        void *o, cudaStream_t st) {
+int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, int n_rows, const void *q, const int32_t *row_pos, const void *k,
+                        const void *v, float scale, void *o, cudaStream_t st) {
     if (SMEM_BYTES > (size_t)ctx->max_smem_optin) return STR_ERR_UNSUPPORTED_SHAPE;
     CUtensorMap tq, tk, tv;
-    int rc = str_make_tmap_3d_bf16_sw128(ctx, &tq, q, (uint64_t)s->Hq * HD, (uint64_t)s->T, (uint64_t)s->Bz, BQ);
+    int rc = str_make_tmap_3d_bf16_sw128(ctx, &tq, q, (uint64_t)s->Hq * HD, (uint64_t)n_rows, (uint64_t)s->Bz, BQ);
     if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tk, k, (uint64_t)s->Hkv * HD, (uint64_t)s->T, (uint64_t)s->Bz, BKV);
     if (rc == STR_OK) rc = str_make_tmap_3d_bf16_sw128(ctx, &tv, v, (uint64_t)s->Hkv * HD, (uint64_t)s->T, (uint64_t)s->Bz, BKV);
     if (rc != STR_OK) return rc;
     rc = str_ensure_smem(ctx, STR_SMEM_ATTN_FWD, attn_fwd_tc_kernel, SMEM_BYTES);
     if (rc != STR_OK) return rc;
-    dim3 grid(ceil_div(s->T, 2 * BQ), s->Hq, s->Bz);
-    attn_fwd_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, s->T, s->Hq, s->Hkv,
-                                                             scale * 1.4426950408889634f, (__nv_bfloat16 *)o,
+    dim3 grid(ceil_div(n_rows, 2 * BQ), s->Hq, s->Bz);
+    attn_fwd_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, n_rows, s->T, s->Hq, s->Hkv,
+                                                             scale * 1.4426950408889634f, row_pos, (__nv_bfloat16 *)o,
                                                              ctx->status_dev);
     return str_launch_ok(ctx);
 }

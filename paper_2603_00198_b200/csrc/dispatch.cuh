@@ -16,8 +16,10 @@ int str_ssd_simt(str_ctx *ctx, const str_ssd_shape *s, const void *x, const floa
 bool str_ssd_simt_supported(const str_ssd_shape *s);
 int str_gemm_simt(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w,
                   const void *residual, void *out, cudaStream_t st);
-int str_attn_prefill_simt(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v,
-                          float scale, void *o, cudaStream_t st);
+// n_rows query rows per sequence; row_pos (device [Bz,n_rows], ascending) gives each row's index in the key sequence,
+// nullptr = rows 0 .. n_rows-1 (then n_rows == s->T).
+int str_attn_prefill_simt(str_ctx *ctx, const str_attn_shape *s, int n_rows, const void *q, const int32_t *row_pos,
+                          const void *k, const void *v, float scale, void *o, cudaStream_t st);
 bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const void *w, const void *residual,
                            const void *out);
 int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
@@ -28,8 +30,8 @@ bool str_ssd_tc_supported(const str_ssd_shape *s, const void *x, const void *B, 
 int str_ssd_tc(str_ctx *ctx, const str_ssd_shape *s, const void *x, const float *dt, const float *A, const void *B,
                const void *C, void *y, float *final_state, cudaStream_t st);
 bool str_attn_prefill_tc_supported(const str_attn_shape *s, const void *q, const void *k, const void *v, const void *o);
-int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, const void *q, const void *k, const void *v, float scale,
-                        void *o, cudaStream_t st);
+int str_attn_prefill_tc(str_ctx *ctx, const str_attn_shape *s, int n_rows, const void *q, const int32_t *row_pos, const void *k,
+                        const void *v, float scale, void *o, cudaStream_t st);
 bool str_mamba_importance_tc_supported(const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C);
 int str_mamba_importance_tc(str_ctx *ctx, const str_ssm_score_shape *s, int n_vis, int n_text, const void *B, const void *C,
                             const float *dt, float *scores, cudaStream_t st);

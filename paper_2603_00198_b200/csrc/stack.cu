@@ -13,8 +13,17 @@ __global__ void iota_rows_kernel(int rows, int T, int32_t *a, int32_t *b) {
     if (i < rows) { a[i] = i % T; b[i] = i % T; }
 }
 
+// Index in the incoming sequence of every row that survives a cut: the kept visual rows, then the text rows.
+__global__ void survivor_rows_kernel(int Bz, int n_vis, int n_text, int k, const int32_t *__restrict__ kept,
+                                     int32_t *__restrict__ rows_out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Bz * (k + n_text)) return;
+    const int b = i / (k + n_text), j = i % (k + n_text);
+    rows_out[i] = j < k ? kept[(size_t)b * k + j] : n_vis + (j - k);
+}
+
 struct Regions {
-    size_t hidden[2], normed, proj, bufA, bufB, bufC, bufY, dt, pos[2], idx[2], scores, kept, sub, total;
+    size_t hidden[2], normed, proj, bufA, bufB, bufC, bufY, dt, pos[2], idx[2], scores, kept, rowpos, sub, total;
     size_t sub_bytes;
 };
 
@@ -80,6 +89,7 @@ Regions plan(const str_stack_desc *d) {
     for (int i = 0; i < 2; ++i) { r.pos[i] = take(R * 4); r.idx[i] = take(R * 4); }
     r.scores = take((size_t)d->Bz * imax(d->n_vis, 1) * 4);
     r.kept = take((size_t)d->Bz * imax(d->n_vis, 1) * 4);
+    r.rowpos = take(R * 4);
     size_t sub = 0;
     if (has_m) {
         str_ssd_shape s = {d->Bz, (int)T0, d->H, d->p, d->n, d->G, d->Q, d->dtype};
@@ -248,21 +258,27 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
                                    bufC, stream));
             str_attn_shape as = {Bz, T, d->Hq, d->Hkv, d->d, dtype};
             const float scale = 1.0f / sqrtf((float)d->d);
-            STR_TRY(str_attn_prefill(ctx, &as, bufA, bufB, bufC, scale, bufY, sub, r.sub_bytes, stream));
             if (want_score && n_cur > 0) {
                 str_attn_score_shape ss = {Bz, T, d->Hq, d->Hkv, d->d, dtype};
                 STR_TRY(str_attn_importance_ex(ctx, &ss, n_cur, M, bufA, bufB, scale, d->attn_score_denominator, scores, sub,
                                                r.sub_bytes, stream));
             }
             if (reduce) {
+                // The score needs the text queries and the keys only, so the layer selects first and runs the attention
+                // for the surviving query rows alone, against every incoming key and value.
                 STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));
                 STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, cur, pos[psel], idx[psel], kept, normed, pdst, idst,
                                     stream));
-                // the attention outputs of the survivors (q is no longer needed: its buffer takes them)
-                STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, qd, dtype, bufY, nullptr, nullptr, kept, bufA, nullptr, nullptr,
+                // the survivors' queries go to the projection buffer (its q | k | v content has been split out)
+                STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, qd, dtype, bufA, nullptr, nullptr, kept, proj, nullptr, nullptr,
                                     stream));
-                STR_TRY(str_gemm(ctx, dtype, rows_out, D, qd, bufA, L.w_out, normed, dst, sub, r.sub_bytes, stream));
+                int32_t *rowpos = (int32_t *)(ws + r.rowpos);
+                survivor_rows_kernel<<<ceil_div(rows_out, 256), 256, 0, st>>>(Bz, n_cur, M, K, kept, rowpos);
+                STR_TRY(str_launch_ok(ctx));
+                STR_TRY(str_attn_prefill_rows(ctx, &as, K + M, proj, rowpos, bufB, bufC, scale, bufY, sub, r.sub_bytes, stream));
+                STR_TRY(str_gemm(ctx, dtype, rows_out, D, qd, bufY, L.w_out, normed, dst, sub, r.sub_bytes, stream));
             } else {
+                STR_TRY(str_attn_prefill(ctx, &as, bufA, bufB, bufC, scale, bufY, sub, r.sub_bytes, stream));
                 STR_TRY(str_gemm(ctx, dtype, rows, D, qd, bufY, L.w_out, cur, dst, sub, r.sub_bytes, stream));
             }
             // hand-off to a decoder: keys, values and positions of the rows that leave the layer

@@ -136,3 +136,30 @@ def test_relu_squared(ctx, dtype, n):
     assert max_rel_err(host(binding.str_relu_squared(ctx, x)), ref) <= TOL[dtype]
     binding.str_relu_squared(ctx, x, inplace=True)
     assert max_rel_err(host(x), ref) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype,Bz,T,Hq,Hkv,d,keep", [("bf16", 2, 1500, 4, 2, 128, 0.25), ("bf16", 1, 700, 8, 2, 128, 0.1),
+                                                      ("f32", 1, 333, 4, 4, 32, 0.3), ("bf16", 2, 450, 4, 2, 64, 0.5)])
+def test_attention_for_a_gathered_subset_of_query_rows(ctx, dtype, Bz, T, Hq, Hkv, d, keep):
+    """A layer that selects before its attention only needs the surviving rows' outputs: computed for a gathered
+    subset (ascending indices into the key sequence) they equal the oracle's rows and are bit-identical to the rows
+    of the full call, whatever other rows share their tile."""
+    import torch
+    g = inputs.rng(31, T)
+    q = inputs.to_grid(g.standard_normal((Bz, T, Hq, d), dtype=np.float32), dtype)
+    k = inputs.to_grid(g.standard_normal((Bz, T, Hkv, d), dtype=np.float32) * 1.5, dtype)
+    v = inputs.to_grid(g.standard_normal((Bz, T, Hkv, d), dtype=np.float32), dtype)
+    n_text = 20
+    n_keep = int((T - n_text) * keep)
+    rows = np.stack([np.concatenate([np.sort(g.choice(T - n_text, size=n_keep, replace=False)), np.arange(T - n_text, T)])
+                     for _ in range(Bz)]).astype(np.int32)
+    scale = 1.0 / np.sqrt(d)
+    full = binding.str_attn_prefill(ctx, dev(q, dtype), dev(k, dtype), dev(v, dtype), scale)
+    qr = np.stack([q[b][rows[b]] for b in range(Bz)])
+    part = binding.str_attn_prefill_rows(ctx, dev(qr, dtype), dev(rows), dev(k, dtype), dev(v, dtype), scale)
+    ctx.check_status()
+    for b in range(Bz):
+        assert bool((part[b] == full[b][torch.from_numpy(rows[b]).long().cuda()]).all())
+        sample = [0, 1, n_keep // 2, n_keep - 1, n_keep, n_keep + n_text - 1]
+        ref = oracle.attention_rows(q[b], k[b], v[b], scale, [int(rows[b][j]) for j in sample])
+        assert max_rel_err(host(part)[b][sample], ref) <= (2e-2 if dtype == "bf16" else 2e-4)

@@ -29,7 +29,9 @@ def _rnd(dtype):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("kind,shape", [("M", MS), ("A", AS), ("M", inputs.MAMBA_TINY)])
+@pytest.mark.parametrize("kind,shape", [("M", MS), ("A", AS), ("M", inputs.MAMBA_TINY),
+                                        ("M", dict(D=512, H=8, p=64, n=128, G=2, Q=128, conv=4)),
+                                        ("A", dict(D=512, Hq=4, Hkv=2, d=128, theta=1.0e6))])
 def test_single_layer_with_reduction(ctx, dtype, kind, shape):
     n_vis, M = 1000, 24
     layers = inputs.stack_params(61, kind, shape, shape, dtype)
@@ -150,6 +152,27 @@ def test_all_layer_sigmoid_schedule(ctx):
 
 
 MS_TC = dict(D=512, H=8, p=64, n=128, G=2, Q=128, conv=4)      # shapes the tensor-core kernels tile
+AS_TC = dict(D=512, Hq=4, Hkv=2, d=128, theta=1.0e6)
+
+
+@pytest.mark.parametrize("pattern", ["MAM", "MMA", "AMA"])
+@pytest.mark.parametrize("ms,at", [(MS, AS), (MS_TC, AS_TC)])
+def test_select_before_the_mixer_epilogue_leaves_survivors_bit_identical(ctx, pattern, ms, at):
+    """A reducing layer selects before its epilogue: a Mamba layer gates / norms / projects only the survivors, an
+    attention layer runs its attention for the surviving query rows only.  The rows that survive a cut at the last
+    layer are bit-identical to the same rows of the unreduced run, for either layer kind, on the tensor-core shapes
+    as well as on the fallback shapes."""
+    n_vis, M, Bz = 700, 20, 2
+    layers = inputs.stack_params(70, pattern, ms, at, "bf16")
+    h0 = inputs.hidden_inputs(70, n_vis + M, ms["D"], "bf16", batch=Bz)
+    full = binding.Stack(ctx, layers, "bf16", Bz, n_vis, M, [n_vis] * 3, Q=ms["Q"])
+    out, pos, idx = binding.str_stack_prefill(full, dev(h0, "bf16"))
+    cut = binding.Stack(ctx, layers, "bf16", Bz, n_vis, M, [n_vis, n_vis, n_vis // 3], Q=ms["Q"])
+    out2, pos2, idx2 = binding.str_stack_prefill(cut, dev(h0, "bf16"))
+    ctx.check_status()
+    assert out2.shape == (Bz, n_vis // 3 + M, ms["D"])
+    for b in range(Bz):
+        assert bool((out2[b] == out[b][idx2[b].long()]).all())
 
 
 @pytest.mark.parametrize("dtype,shape", [("f32", MS), ("bf16", MS), ("bf16", MS_TC)])
