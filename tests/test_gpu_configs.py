@@ -19,12 +19,11 @@ import torch
 
 import oracle
 from paper_2603_00198_b200 import binding, inputs
-from util_gpu import assert_kept_matches, dev, host
+from util_gpu import SCORE_TOL, assert_kept_matches, check_layer, dev, host
 
 pytestmark = pytest.mark.gpu
 MS, AT = inputs.MAMBA_8B, inputs.ATTN_8B
 RND = oracle.round_to_bf16
-SCORE_TOL = 5e-3
 
 
 @pytest.fixture(scope="module")
@@ -33,38 +32,6 @@ def ctx():
     yield c
     c.check_status()
     c.close()
-
-
-def _row_err(got, ref):
-    """max over rows of max|got - ref|, relative to max|ref| of the tensor."""
-    return float(np.abs(got - ref).max() / np.abs(ref).max())
-
-
-def _check_layer(ctx, layer, Bz, n_in, M, K, hid_in, pos_in, idx_in, ref_out, ref_idx, rec, Q=0):
-    """One layer on the GPU, fed `hid_in` [Bz, n_in+M, D] with its carried ids; compared with the oracle's output of
-    the same layer (`ref_out`, `ref_idx` per sequence) and, when it reduces, with the oracle's scores and selection."""
-    st = binding.Stack(ctx, [layer], "bf16", Bz, n_in, M, [K], Q=Q)
-    res = binding.str_stack_prefill_ex(st, dev(hid_in, "bf16"), positions_in=dev(pos_in), idx_map_in=dev(idx_in), want_trace=True)
-    ctx.check_status()
-    out, gidx = host(res["hidden"]), res["idx_map"].cpu().numpy()
-    assert np.array_equal(res["positions"].cpu().numpy(), gidx)
-    worst = 0.0
-    for b in range(Bz):
-        gi = gidx[b]
-        assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], idx_in[b][-M:])
-        if K < n_in:
-            s_gpu, kept = res["trace"][0]["scores"][b].cpu().numpy(), res["trace"][0]["kept"][b].cpu().numpy()
-            s_ref = rec[b]["scores"]
-            assert np.abs(s_gpu / s_ref - 1).max() <= SCORE_TOL
-            assert_kept_matches(kept, rec[b]["kept"], s_ref, tol=SCORE_TOL)
-            assert np.array_equal(gi[:K], idx_in[b][kept])            # ids bit-exact given the selection
-        else:
-            assert np.array_equal(gi, idx_in[b])
-        common, a, c = np.intersect1d(gi, ref_idx[b], return_indices=True)
-        assert len(common) >= 0.98 * len(ref_idx[b])
-        worst = max(worst, _row_err(out[b][a], ref_out[b][c]))
-    assert worst <= 2e-2, worst
-    return worst
 
 
 def test_c1_mamba_layer_at_full_width(ctx):
@@ -76,7 +43,7 @@ def test_c1_mamba_layer_at_full_width(ctx):
     h0 = inputs.hidden_inputs(cfg["seed"], n_vis + M, MS["D"], "bf16")
     ref, rpos, ridx, trace = oracle.stack_prefill(h0[0], M, layers, K, RND)
     ids = np.arange(n_vis + M, dtype=np.int32)[None]
-    _check_layer(ctx, layers[0], 1, n_vis, M, K[0], h0, ids, ids, [ref], [ridx], [trace[0]], Q=MS["Q"])
+    check_layer(ctx, layers[0], 1, n_vis, M, K[0], h0, ids, ids, [ref], [ridx], [trace[0]], Q=MS["Q"])
 
 
 def test_c2_attention_layer_at_full_width_whole_output(ctx):
@@ -86,7 +53,7 @@ def test_c2_attention_layer_at_full_width_whole_output(ctx):
     K = [n_vis // 4]
     ref, rpos, ridx, trace = oracle.stack_prefill(h0[0], M, layers, K, RND)
     ids = np.arange(n_vis + M, dtype=np.int32)[None]
-    _check_layer(ctx, layers[0], 1, n_vis, M, K[0], h0, ids, ids, [ref], [ridx], [trace[0]])
+    check_layer(ctx, layers[0], 1, n_vis, M, K[0], h0, ids, ids, [ref], [ridx], [trace[0]])
     assert abs(trace[0]["scores"].sum() - 1.0) < 1e-9
 
 
@@ -146,7 +113,7 @@ def test_c3_layer_pattern_teacher_forced_at_full_width(ctx, c3_layers, Bz, n_vis
         hid = np.stack([r["hidden_in"] for r in recs]).astype(np.float32)
         pos = np.stack([r["positions_in"] for r in recs])
         ids = np.stack([r["idx_map_in"] for r in recs])
-        worst.append(_check_layer(ctx, layers[l], Bz, n_in, M, K[l], hid, pos, ids, [x[0] for x in nxt], [x[1] for x in nxt],
+        worst.append(check_layer(ctx, layers[l], Bz, n_in, M, K[l], hid, pos, ids, [x[0] for x in nxt], [x[1] for x in nxt],
                                   recs, Q=MS["Q"]))
     print("max row error per layer:", " ".join("%.1e" % w for w in worst))
     # The same stack free-running on the GPU.  Its output is, bit for bit, the composition of the single-layer calls

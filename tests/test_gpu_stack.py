@@ -259,3 +259,39 @@ def test_single_ffn_layer_teacher_forced(ctx):
     out, pos, idx = binding.str_stack_prefill(st, dev(h0, "bf16"))
     ref = oracle.ffn_block(h0[0], layers[0][1], oracle.round_to_bf16)
     assert max_rel_err(host(out)[0], ref) <= 2e-2
+
+
+def test_transformer_stack_reducing_at_every_attention_layer_batch_8(ctx):
+    """The second workload of the paper's appendix "Models": a pure Transformer (attention + FFN blocks) under the
+    all-layer sigmoid schedule, so that every attention layer scores, selects and compacts (FFN layers pass the rows
+    on), at batch 8 and on tensor-core shapes.  Teacher-forced per layer: each GPU layer gets the oracle's input of
+    that layer, so the maximum row error is asserted in every layer; the free-running GPU stack is then shown to be
+    exactly the composition of those layers."""
+    from util_gpu import check_layer
+    Bz, n_vis, M = 8, 900, 28
+    pattern = "AFAFAFAF"
+    layers = inputs.stack_params(71, pattern, None, AS_TC, "bf16", ffn_dim=1024)
+    alpha = binding.str_sigmoid_schedule_bp(len(pattern), 20.0, 0.24, 1.0, 0.125)
+    K = binding.str_schedule_keep_counts_layers(alpha, pattern, n_vis, 16)
+    assert K == oracle.schedule_keep_counts(alpha, n_vis, 16, pattern)
+    cuts = [l for l, (a, b) in enumerate(zip([n_vis] + K, K)) if b < a]
+    assert cuts == [0, 2, 4, 6]                                   # every attention layer reduces, no FFN layer does
+    h0 = inputs.hidden_inputs(71, n_vis + M, AS_TC["D"], "bf16", batch=Bz)
+    runs = [oracle.stack_prefill(h0[b], M, layers, K, oracle.round_to_bf16, keep_inputs=True) for b in range(Bz)]
+    for l in range(len(layers)):
+        recs = [runs[b][3][l] for b in range(Bz)]
+        nxt = [(runs[b][3][l + 1]["hidden_in"], runs[b][3][l + 1]["idx_map_in"]) if l + 1 < len(layers)
+               else (runs[b][0], runs[b][2]) for b in range(Bz)]
+        check_layer(ctx, layers[l], Bz, recs[0]["n_in"], M, K[l], np.stack([r["hidden_in"] for r in recs]).astype(np.float32),
+                    np.stack([r["positions_in"] for r in recs]), np.stack([r["idx_map_in"] for r in recs]),
+                    [x[0] for x in nxt], [x[1] for x in nxt], recs)
+    st = binding.Stack(ctx, layers, "bf16", Bz, n_vis, M, K)
+    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, "bf16"), want_trace=True)
+    ctx.check_status()
+    assert [t["layer"] for t in tr] == cuts and out.shape == (Bz, K[-1] + M, AS_TC["D"])
+    h, p_, i_, n_cur = dev(h0, "bf16"), None, None, n_vis
+    for l in range(len(layers)):
+        one = binding.Stack(ctx, [layers[l]], "bf16", Bz, n_cur, M, [K[l]])
+        res = binding.str_stack_prefill_ex(one, h, positions_in=p_, idx_map_in=i_)
+        h, p_, i_, n_cur = res["hidden"], res["positions"], res["idx_map"], K[l]
+    assert bool((h == out).all()) and bool((i_ == idx).all())
