@@ -25,7 +25,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # Measured DRAM traffic / algorithmic bytes of one launch, from the ncu captures summarised under profiles/
 # (smaller cases of the same kernels; traffic grows in proportion to the algorithmic bytes).  A kernel that
 # has changed since its capture is left out (traffic is then reported as null).
-NCU_TRAFFIC_RATIO = {"gemm": 472.9 / 343.2, "ssd_scan": 115.8 / 157.9, "mamba_score": 86.7 / 84.0, "compact": 226.6 / 270.7}
+NCU_TRAFFIC_RATIO = {"gemm": 464.1 / 343.2, "ssd_scan": 115.1 / 157.9, "mamba_score": 86.7 / 84.0, "compact": 226.6 / 270.7}
 
 
 def peaks():
@@ -586,7 +586,7 @@ def main():
     ap.add_argument("--attn-denominator", default="visual", choices=["visual", "causal_row"],
                     help="normaliser of the attention-layer importance: visual keys only (the paper's formula) or the causal row")
     ap.add_argument("--x0", type=float, default=0.11, help="midpoint of the sigmoid schedule (0.11 / 0.24 / 0.41)")
-    ap.add_argument("--micro-seconds", type=float, default=0.6, help="repeat a --micro launch for at least this long (clock sampling)")
+    ap.add_argument("--micro-seconds", type=float, default=0.0, help="repeat a --micro launch for at least this long, so that the clock sampler sees the GPU under load")
     ap.add_argument("--graph", action="store_true", help="also time the step replayed from a CUDA graph")
     ap.add_argument("--no-kernels-alone", action="store_true", help="skip the per-kernel timings after the headline run")
     ap.add_argument("--micro", default="", help="time one kernel alone: ssd | mamba_score | mamba_dyn_score | attn_score | attn_fwd | "
