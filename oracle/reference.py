@@ -420,7 +420,7 @@ def mamba2_block(u, prm, rnd=_identity):
     d_inner = H * p
     u = _f64(u)
     T = u.shape[0]
-    normed = rnd(rmsnorm(u))
+    normed = rmsnorm(u)                        # not stored by the GPU path (the norm is fused into the projection)
     zxbcdt = rnd(normed @ _f64(prm["W_in"]))
     z = zxbcdt[:, :d_inner]
     xBC = zxbcdt[:, d_inner:2 * d_inner + 2 * G * n]
@@ -442,7 +442,7 @@ def attn_block(u, positions, prm, rnd=_identity):
     Hq, Hkv, d = prm["Hq"], prm["Hkv"], prm["d"]
     u = _f64(u)
     T = u.shape[0]
-    normed = rnd(rmsnorm(u))
+    normed = rmsnorm(u)                        # not stored by the GPU path (the norm is fused into the projection)
     qkv = rnd(normed @ _f64(prm["W_qkv"]))
     q = qkv[:, :Hq * d].reshape(T, Hq, d)
     k = qkv[:, Hq * d:(Hq + Hkv) * d].reshape(T, Hkv, d)
@@ -460,7 +460,7 @@ def attn_block_projections(u, positions, prm, rnd=_identity):
     Hq, Hkv, d = prm["Hq"], prm["Hkv"], prm["d"]
     u = _f64(u)
     T = u.shape[0]
-    normed = rnd(rmsnorm(u))
+    normed = rmsnorm(u)                        # not stored by the GPU path (the norm is fused into the projection)
     qkv = rnd(normed @ _f64(prm["W_qkv"]))
     q = qkv[:, :Hq * d].reshape(T, Hq, d)
     k = qkv[:, Hq * d:(Hq + Hkv) * d].reshape(T, Hkv, d)
@@ -490,7 +490,7 @@ def ffn_block(u, prm, rnd=_identity):
     The paper names FFN (MLP) blocks as the third block type of its hybrid (appendix "Models") and says nothing
     about their inside; the squared-ReLU, ungated form is the one of the hybrid family it cites."""
     u = _f64(u)
-    normed = rnd(rmsnorm(u))
+    normed = rmsnorm(u)                        # not stored by the GPU path (the norm is fused into the projection)
     up = rnd(normed @ _f64(prm["W_up"]))
     act = rnd(np.maximum(up, 0.0) ** 2)
     return rnd(u + act @ _f64(prm["W_down"]))

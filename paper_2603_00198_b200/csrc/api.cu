@@ -140,15 +140,21 @@ extern "C" int str_attn_importance(str_ctx *ctx, const str_attn_score_shape *s, 
 // ---------------------------------------------------------------- glue: GEMM, attention forward
 extern "C" size_t str_gemm_workspace_size(int, int, int, int) { return 0; }
 
-extern "C" int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w,
-                        const void *residual, void *out, void *workspace, size_t workspace_bytes, void *stream) {
+int str_gemm_fused(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
+                   const StrRowNorm &rn, void *stream) {
     StrProfScope prof_scope(ctx, STR_CAT_GEMM, stream);
-    (void)workspace; (void)workspace_bytes;
     if (!ctx || !a || !w || !out || M < 0 || N <= 0 || K <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
     if (M == 0) return STR_OK;
     if (!str_force_simt() && ctx->encode_tiled && str_gemm_tc_supported(dtype, M, N, K, a, w, residual, out))
-        return ++ctx->tc_calls, str_gemm_tc(ctx, M, N, K, a, w, residual, out, (cudaStream_t)stream);
-    return ++ctx->fallback_calls, str_gemm_simt(ctx, dtype, M, N, K, a, w, residual, out, (cudaStream_t)stream);
+        return ++ctx->tc_calls, str_gemm_tc(ctx, M, N, K, a, w, residual, out, rn, (cudaStream_t)stream);
+    return ++ctx->fallback_calls, str_gemm_simt(ctx, dtype, M, N, K, a, w, residual, out, rn, (cudaStream_t)stream);
+}
+
+extern "C" int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w,
+                        const void *residual, void *out, void *workspace, size_t workspace_bytes, void *stream) {
+    (void)workspace; (void)workspace_bytes;
+    const StrRowNorm none = {nullptr, 0, 0.f, 0.f, nullptr};
+    return str_gemm_fused(ctx, dtype, M, N, K, a, w, residual, out, none, stream);
 }
 
 extern "C" size_t str_attn_prefill_workspace_size(const str_attn_shape *) { return 0; }

@@ -14,8 +14,27 @@ int str_ssd_simt(str_ctx *ctx, const str_ssd_shape *s, const void *x, const floa
                  const void *B, const void *C, const float *D, const float *init_state, void *y,
                  float *final_state, cudaStream_t st);
 bool str_ssd_simt_supported(const str_ssd_shape *s);
+// RMSNorm fused into a projection.  A pre-norm block computes RMSNorm(h) W^T; with unit norm weight the norm is a
+// per-row scalar, so (h / rms) W^T = (h W^T) / rms: the GEMM runs on h itself and its epilogue scales row r by
+// rsqrt(sum_j ss_in[r, j] * inv_dim + eps).  ss_in holds partial sums of squares of the stored values of row r of A,
+// nt_in per row, written by the kernel that produced A: a GEMM given ss_out writes, per output row, one partial per
+// STR_SS_BLOCK output columns ([M, ceil(N / STR_SS_BLOCK)] floats).  Partials are summed in index order, so the result
+// does not depend on the order in which tiles finish.  All-null = plain GEMM.
+#define STR_SS_BLOCK 256
+struct StrRowNorm {
+    const float *ss_in;
+    int nt_in;
+    float inv_dim, eps;
+    float *ss_out;
+};
+static inline int str_ss_blocks(int N) { return (N + STR_SS_BLOCK - 1) / STR_SS_BLOCK; }
+int str_gemm_fused(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
+                   const StrRowNorm &rn, void *stream);
+// Partial sums of squares of the rows of a [rows, D] matrix in the layout above (for a matrix no GEMM of this
+// library produced: the stack's input).
+int str_row_sumsq(str_ctx *ctx, int dtype, int rows, int D, const void *in, float *ss_out, void *stream);
 int str_gemm_simt(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, const void *w,
-                  const void *residual, void *out, cudaStream_t st);
+                  const void *residual, void *out, const StrRowNorm &rn, cudaStream_t st);
 // n_rows query rows per sequence; row_pos (device [Bz,n_rows], ascending) gives each row's index in the key sequence,
 // nullptr = rows 0 .. n_rows-1 (then n_rows == s->T).
 int str_attn_prefill_simt(str_ctx *ctx, const str_attn_shape *s, int n_rows, const void *q, const int32_t *row_pos,
@@ -23,7 +42,7 @@ int str_attn_prefill_simt(str_ctx *ctx, const str_attn_shape *s, int n_rows, con
 bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const void *w, const void *residual,
                            const void *out);
 int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
-                cudaStream_t st);
+                const StrRowNorm &rn, cudaStream_t st);
 bool str_force_simt();
 bool str_ssd_tc_supported(const str_ssd_shape *s, const void *x, const void *B, const void *C, const void *y,
                           const float *D, const float *init_state);

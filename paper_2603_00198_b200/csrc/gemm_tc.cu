@@ -10,6 +10,9 @@
 //              residual, narrow to bf16, 16-byte stores.  Runs concurrently with the next tile's
 //              main loop thanks to the double-buffered accumulator.
 // Tiles are walked in bands of 8 column tiles so that a band of W stays in L2 while A streams.
+// The epilogue can fuse the RMSNorm that surrounds the projections of a pre-norm block: it scales the accumulator
+// row by 1/rms of the A row (from partial sums of squares left by the kernel that wrote A), and it leaves the
+// partial sums of squares of its own output rows, one per 256-column tile, for the next projection.
 // Every mbarrier wait is bounded; on give-up the kernel records STR_ERR_TIMEOUT and tears down.
 #include "dispatch.cuh"
 #include "tc_common.cuh"
@@ -33,7 +36,7 @@ __device__ __forceinline__ TileCoord tile_coord(int t, int tiles_m, int tiles_n)
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w, int M, int N,
-               int K, const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ out, int *status) {
+               int K, const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ out, StrRowNorm rn, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
@@ -126,6 +129,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int row = tc_.m * BM + quad * 32 + lane;
             const int col0 = tc_.n * BN;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN;
+            // fused RMSNorm of the A rows: 1/rms from the partial sums of squares the producer of A left behind, summed
+            // in index order (deterministic), applied to the accumulator row
+            float scale = 1.0f;
+            if (rn.ss_in && row < M) {
+                float t = 0.f;
+                for (int j = 0; j < rn.nt_in; ++j) t += __ldg(rn.ss_in + (size_t)row * rn.nt_in + j);
+                scale = rsqrtf(t * rn.inv_dim + rn.eps);
+            }
+            float ss = 0.f;                              // sum of squares of this row's stored outputs in this tile
 #pragma unroll 1
             for (int c = 0; c < BN; c += 32) {
                 uint32_t v[32];
@@ -139,7 +151,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         if (g * 8 < valid) {
                             float f[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]);
+                            for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]) * scale;
                             if (residual) {
                                 const uint4 r = *reinterpret_cast<const uint4 *>(residual + off + g * 8);
                                 const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
@@ -155,10 +167,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                             o.z = tc::pack_bf16x2(f[4], f[5]);
                             o.w = tc::pack_bf16x2(f[6], f[7]);
                             *reinterpret_cast<uint4 *>(out + off + g * 8) = o;
+                            if (rn.ss_out) {
+                                const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const float lo = __uint_as_float(ow[j] << 16), hi = __uint_as_float(ow[j] & 0xFFFF0000u);
+                                    ss = fmaf(lo, lo, ss);
+                                    ss = fmaf(hi, hi, ss);
+                                }
+                            }
                         }
                     }
                 }
             }
+            if (rn.ss_out && row < M) rn.ss_out[(size_t)row * tiles_n + tc_.n] = ss;
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(acc_empty + acc);
@@ -180,7 +202,7 @@ bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const 
 }
 
 int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
-                cudaStream_t st) {
+                const StrRowNorm &rn, cudaStream_t st) {
     CUtensorMap ta, tw;
     int rc = str_make_tmap_2d_bf16(ctx, &ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != STR_OK) return rc;
@@ -191,6 +213,6 @@ int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w,
     const int tiles = ceil_div(M, BM) * ceil_div(N, BN);
     const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tw, M, N, K, (const __nv_bfloat16 *)residual,
-                                                         (__nv_bfloat16 *)out, ctx->status_dev);
+                                                         (__nv_bfloat16 *)out, rn, ctx->status_dev);
     return str_launch_ok(ctx);
 }

@@ -22,8 +22,19 @@ __global__ void survivor_rows_kernel(int Bz, int n_vis, int n_text, int k, const
     rows_out[i] = j < k ? kept[(size_t)b * k + j] : n_vis + (j - k);
 }
 
+// Rows of a small fp32 side array (the partial sums of squares of the hidden rows) for the rows that survive a cut.
+__global__ void gather_rows_f32_kernel(int Bz, int T_in, int n_vis, int n_text, int k, int width, const int32_t *__restrict__ kept,
+                                       const float *__restrict__ in, float *__restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Bz * (k + n_text) * width) return;
+    const int c = i % width, r = i / width;
+    const int b = r / (k + n_text), j = r % (k + n_text);
+    const int src = j < k ? kept[(size_t)b * k + j] : n_vis + (j - k);
+    out[i] = in[((size_t)b * T_in + src) * width + c];
+}
+
 struct Regions {
-    size_t hidden[2], normed, proj, bufA, bufB, bufC, bufY, dt, pos[2], idx[2], scores, kept, rowpos, sub, total;
+    size_t hidden[2], normed, proj, bufA, bufB, bufC, bufY, dt, pos[2], idx[2], scores, kept, rowpos, ss[3], sub, total;
     size_t sub_bytes;
 };
 
@@ -90,6 +101,7 @@ Regions plan(const str_stack_desc *d) {
     r.scores = take((size_t)d->Bz * imax(d->n_vis, 1) * 4);
     r.kept = take((size_t)d->Bz * imax(d->n_vis, 1) * 4);
     r.rowpos = take(R * 4);
+    for (int i = 0; i < 3; ++i) r.ss[i] = take(R * str_ss_blocks(d->D) * sizeof(float));
     size_t sub = 0;
     if (has_m) {
         str_ssd_shape s = {d->Bz, (int)T0, d->H, d->p, d->n, d->G, d->Q, d->dtype};
@@ -169,6 +181,16 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
     const void *cur = hidden_in;
     int hsel = 0;      // next free hidden buffer
     int psel = 0;      // current positions / idx buffer
+    // The RMSNorm in front of every layer is fused into the layer's first projection: the projection runs on the hidden
+    // rows themselves and scales its output rows by 1/rms, taken from partial sums of squares that the previous layer's
+    // last projection left behind (for the stack's input: from one pass over it).  `normed` is only a scratch buffer
+    // for the survivors' residual rows now.
+    const int ntD = str_ss_blocks(D);
+    const float inv_D = 1.0f / (float)D;
+    float *ssb[3] = {(float *)(ws + r.ss[0]), (float *)(ws + r.ss[1]), (float *)(ws + r.ss[2])};
+    const float *cur_ss = ssb[0];
+    int ssel = 1;      // next free buffer of partial sums
+    if (!feed) STR_TRY(str_row_sumsq(ctx, dtype, Bz * (n_cur + M), D, hidden_in, ssb[0], stream));
     size_t kept_off = 0, score_off = 0;
 
     for (int l = 0; l < d->n_layers; ++l) {
@@ -182,20 +204,30 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
         int32_t *kept = (reduce && kept_trace) ? kept_trace + kept_off : kept_int;
         void *mix_out = (last && !reduce) ? hidden_out : hid[hsel];
 
-        // RMSNorm of the layer input and the layer's first projection [rows x N] = normed W^T into `proj`
+        // the layer's first projection with the RMSNorm of the layer input fused in: [rows x N] = RMSNorm(cur) W^T into `proj`
         auto norm_and_project = [&](int N, const void *w) -> int {
             const bool fed = feed && l == 0;
             const int step = fed ? feed->rows_per_chunk : rows;
             const size_t esz = dtype_size(dtype);
             for (int j = 0, r0 = 0; r0 < rows; ++j, r0 += step) {
                 const int nr = rows - r0 < step ? rows - r0 : step;
-                if (fed) STR_CUDA_OK(cudaStreamWaitEvent(st, feed->ready[j], 0));
-                STR_TRY(str_rmsnorm(ctx, dtype, nr, D, d->norm_eps, (const char *)cur + (size_t)r0 * D * esz,
-                                    (char *)normed + (size_t)r0 * D * esz, stream));
-                STR_TRY(str_gemm(ctx, dtype, nr, N, D, (const char *)normed + (size_t)r0 * D * esz, w, nullptr,
-                                 (char *)proj + (size_t)r0 * N * esz, sub, r.sub_bytes, stream));
+                float *ss_blk = ssb[0] + (size_t)r0 * ntD;
+                if (fed) {
+                    STR_CUDA_OK(cudaStreamWaitEvent(st, feed->ready[j], 0));
+                    STR_TRY(str_row_sumsq(ctx, dtype, nr, D, (const char *)cur + (size_t)r0 * D * esz, ss_blk, stream));
+                }
+                const StrRowNorm rn = {cur_ss + (size_t)r0 * ntD, ntD, inv_D, d->norm_eps, nullptr};
+                STR_TRY(str_gemm_fused(ctx, dtype, nr, N, D, (const char *)cur + (size_t)r0 * D * esz, w, nullptr,
+                                       (char *)proj + (size_t)r0 * N * esz, rn, stream));
             }
             return STR_OK;
+        };
+        // the layer's last projection adds the residual and leaves the partial sums of squares of its output rows for
+        // the next layer's fused norm
+        float *next_ss = last ? nullptr : ssb[ssel];
+        auto project_out = [&](int nrows, int K_in, const void *a, const void *w, const void *residual, void *out_rows) -> int {
+            const StrRowNorm rn = {nullptr, 0, 0.f, 0.f, next_ss};
+            return str_gemm_fused(ctx, dtype, nrows, D, K_in, a, w, residual, out_rows, rn, stream);
         };
         // A reducing layer selects BEFORE the mixer's epilogue: the score only needs the projections, so the rows
         // about to be dropped skip the gate / norm / output projection (their inputs still feed the scan state
@@ -229,28 +261,29 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
             }
             if (reduce) {
                 STR_TRY(str_topk_select(ctx, Bz, n_cur, K, scores, kept, sub, r.sub_bytes, stream));
-                // z of the survivors: their normed rows are gathered into the layer's output buffer (free until the
-                // output projection writes it), projected with the first d_inner weight rows into the projection
-                // buffer (its [x B C | dt] content was consumed by the conv)
-                STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, normed, nullptr, nullptr, kept, dst, nullptr, nullptr,
-                                    stream));
-                STR_TRY(str_gemm(ctx, dtype, rows_out, d_inner, D, dst, L.w_in, nullptr, proj, sub, r.sub_bytes, stream));
-                // residual rows, positions and the index map of the survivors (normed is free now)
+                // hidden rows (the residual), positions and the index map of the survivors, and their sums of squares
                 STR_TRY(str_compact(ctx, Bz, T, n_cur, M, K, D, dtype, cur, pos[psel], idx[psel], kept, normed, pdst, idst,
                                     stream));
+                float *ss_kept = ssb[2];
+                gather_rows_f32_kernel<<<ceil_div(rows_out * ntD, 256), 256, 0, st>>>(Bz, T, n_cur, M, K, ntD, kept, cur_ss, ss_kept);
+                STR_TRY(str_launch_ok(ctx));
+                // z of the survivors: the same gathered hidden rows, projected with the first d_inner weight rows (and
+                // the fused norm) into the projection buffer, whose [x B C | dt] content was consumed by the conv
+                const StrRowNorm rnz = {ss_kept, ntD, inv_D, d->norm_eps, nullptr};
+                STR_TRY(str_gemm_fused(ctx, dtype, rows_out, d_inner, D, normed, L.w_in, nullptr, proj, rnz, stream));
                 STR_TRY(str_gated_rmsnorm_gather(ctx, dtype, Bz, T, n_cur, M, K, d_inner, d_inner, d->norm_eps, bufY, proj, true,
                                                  kept, bufA, stream));
-                STR_TRY(str_gemm(ctx, dtype, rows_out, D, d_inner, bufA, L.w_out, normed, dst, sub, r.sub_bytes, stream));
+                STR_TRY(project_out(rows_out, d_inner, bufA, L.w_out, normed, dst));
             } else {
                 STR_TRY(str_gated_rmsnorm(ctx, dtype, rows, d_inner, dip, d->norm_eps, bufY, proj, bufA, stream));
-                STR_TRY(str_gemm(ctx, dtype, rows, D, d_inner, bufA, L.w_out, cur, dst, sub, r.sub_bytes, stream));
+                STR_TRY(project_out(rows, d_inner, bufA, L.w_out, cur, dst));
             }
         } else if (L.kind == STR_LAYER_FFN) {
             // h <- h + W_down relu(W_up RMSNorm(h))^2; the activation runs in place on the up-projection
             const int F = d->ffn_dim;
             STR_TRY(norm_and_project(F, L.w_in));
             STR_TRY(str_relu_squared(ctx, dtype, (size_t)rows * F, proj, proj, stream));
-            STR_TRY(str_gemm(ctx, dtype, rows, D, F, proj, L.w_out, cur, dst, sub, r.sub_bytes, stream));
+            STR_TRY(project_out(rows, F, proj, L.w_out, cur, dst));
         } else {
             const int qd = d->Hq * d->d, kd = d->Hkv * d->d;
             STR_TRY(norm_and_project(qd + 2 * kd, L.w_in));
@@ -276,10 +309,10 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
                 survivor_rows_kernel<<<ceil_div(rows_out, 256), 256, 0, st>>>(Bz, n_cur, M, K, kept, rowpos);
                 STR_TRY(str_launch_ok(ctx));
                 STR_TRY(str_attn_prefill_rows(ctx, &as, K + M, proj, rowpos, bufB, bufC, scale, bufY, sub, r.sub_bytes, stream));
-                STR_TRY(str_gemm(ctx, dtype, rows_out, D, qd, bufY, L.w_out, normed, dst, sub, r.sub_bytes, stream));
+                STR_TRY(project_out(rows_out, qd, bufY, L.w_out, normed, dst));
             } else {
                 STR_TRY(str_attn_prefill(ctx, &as, bufA, bufB, bufC, scale, bufY, sub, r.sub_bytes, stream));
-                STR_TRY(str_gemm(ctx, dtype, rows, D, qd, bufY, L.w_out, cur, dst, sub, r.sub_bytes, stream));
+                STR_TRY(project_out(rows, qd, bufY, L.w_out, cur, dst));
             }
             // hand-off to a decoder: keys, values and positions of the rows that leave the layer
             if (k_out || v_out || kvpos_out) {
@@ -299,6 +332,7 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
             }
         }
         cur = dst;
+        if (next_ss) { cur_ss = next_ss; ssel = (next_ss == ssb[0]) ? 1 : 0; }
         if (dst == hid[0]) hsel = 1;
         else if (dst == hid[1]) hsel = 0;
         if (reduce) {
