@@ -104,9 +104,7 @@ def work_model(cfg, keep_counts):
             w["topk"]["bytes"] += Bz * (4.0 * n_cur + 4.0 * K)
             w["compact"]["bytes"] += Bz * 2.0 * (K + M) * (2 * D + 8)       # residual rows, positions, index map
             if kind == "A":
-                w["compact"]["bytes"] += Bz * 2.0 * (K + M) * 2 * Hq * d     # the survivors' attention outputs
-            else:
-                w["compact"]["bytes"] += Bz * 2.0 * (K + M) * 2 * D          # the survivors' normed rows (input of the z projection)
+                w["compact"]["bytes"] += Bz * 2.0 * (K + M) * 2 * Hq * d     # the survivors' query rows
             n_cur = K
     return w
 

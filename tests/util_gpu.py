@@ -49,8 +49,8 @@ def assert_kept_matches(kept_gpu, kept_ref, scores_ref, tol=1e-4):
 
 
 # Layer-level score tolerance: both sides round the projections to bf16 at the same points, but fp32 against fp64
-# accumulation flips single bf16 roundings of B, C, q, k elements, which moves a score by up to a few 1e-3.
-SCORE_TOL = 5e-3
+# accumulation flips single bf16 roundings of B, C, q, k elements, which moves a score by about 1e-3 (measured maximum 1.1e-3 at the 8B-class Mamba layer).
+SCORE_TOL = 3e-3
 
 
 def row_err(got, ref):
