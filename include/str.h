@@ -325,7 +325,8 @@ int str_stack_prefill_ex(str_ctx *ctx, const str_stack_desc *d, const str_stack_
  * `stream` before returning.  The device staging area is part of the workspace
  * (str_stack_host_workspace_size).  The input travels in a few row blocks on a copy stream owned
  * by the context (created on the first call), so that the first layer starts on block 0 while the
- * rest is still in flight; a context therefore serves one such call at a time. */
+ * rest is still in flight, and the last layer's output projection is issued in row blocks, each
+ * copied back while the next is computed; a context therefore serves one such call at a time. */
 size_t str_stack_host_workspace_size(const str_stack_desc *d);
 int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, const void *hidden_in_host,
                            void *hidden_out_host, int32_t *idx_map_out_host, void *workspace,

@@ -26,7 +26,8 @@ struct str_ctx {
     long long fallback_calls; // entry-point calls that took the plain fp32-FMA kernel of the same entry point
     size_t smem_attr[8];      // dynamic shared memory already opted into on this device, per tensor-core kernel
     cudaStream_t copy_stream; // host-buffer entry point: input chunks are copied on this stream while the caller's
-    cudaEvent_t copy_ev[8];   // stream computes; [0] orders the copies after the caller's earlier work, [1..] = chunk landed
+    cudaEvent_t copy_ev[24];  // stream computes; [0] orders the copies after the caller's earlier work, [1..8] = input
+                              // chunk landed, [9..16] = output row block computed, [17] = output copies done
     bool prof_on;             // record an event pair per leaf call
     std::vector<str_prof_span> prof_spans;
     std::vector<cudaEvent_t> prof_free;

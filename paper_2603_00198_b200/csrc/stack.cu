@@ -137,7 +137,13 @@ extern "C" size_t str_stack_workspace_size(const str_stack_desc *d) {
 // Input feed of the host-buffer entry point: the hidden states arrive in `chunks` row blocks of `rows_per_chunk`
 // rows, block j being complete once `ready[j]` has fired.  Only the first layer's norm and first projection read
 // the input row by row, so only they are issued per block.
-struct StackFeed { int chunks; int rows_per_chunk; cudaEvent_t *ready; };
+// Output drain: the last layer's output projection is issued in `out_chunks` row blocks; after each block an event is
+// recorded on the caller's stream and the block is copied to the host on `copy_stream`, so that only the last block's
+// copy is exposed.
+struct StackFeed {
+    int chunks; int rows_per_chunk; cudaEvent_t *ready;
+    int out_chunks; cudaEvent_t *out_done; cudaStream_t copy_stream; void *out_host;
+};
 
 #define STR_TRY(call)              \
     do {                           \
@@ -227,7 +233,22 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
         float *next_ss = last ? nullptr : ssb[ssel];
         auto project_out = [&](int nrows, int K_in, const void *a, const void *w, const void *residual, void *out_rows) -> int {
             const StrRowNorm rn = {nullptr, 0, 0.f, 0.f, next_ss};
-            return str_gemm_fused(ctx, dtype, nrows, D, K_in, a, w, residual, out_rows, rn, stream);
+            if (!(last && feed && feed->out_chunks > 1))
+                return str_gemm_fused(ctx, dtype, nrows, D, K_in, a, w, residual, out_rows, rn, stream);
+            // host-buffer call, last layer: row blocks (whole GEMM row tiles), each copied out as soon as it is done
+            const size_t esz = dtype_size(dtype);
+            const int step = (int)align_up((size_t)ceil_div(nrows, feed->out_chunks), 128);
+            for (int j = 0, r0 = 0; r0 < nrows; ++j, r0 += step) {
+                const int nr = nrows - r0 < step ? nrows - r0 : step;
+                STR_TRY(str_gemm_fused(ctx, dtype, nr, D, K_in, (const char *)a + (size_t)r0 * K_in * esz, w,
+                                       (const char *)residual + (size_t)r0 * D * esz, (char *)out_rows + (size_t)r0 * D * esz, rn,
+                                       stream));
+                STR_CUDA_OK(cudaEventRecord(feed->out_done[j], st));
+                STR_CUDA_OK(cudaStreamWaitEvent(feed->copy_stream, feed->out_done[j], 0));
+                STR_CUDA_OK(cudaMemcpyAsync((char *)feed->out_host + (size_t)r0 * D * esz, (const char *)out_rows + (size_t)r0 * D * esz,
+                                            (size_t)nr * D * esz, cudaMemcpyDeviceToHost, feed->copy_stream));
+            }
+            return STR_OK;
         };
         // A reducing layer selects BEFORE the mixer's epilogue: the score only needs the projections, so the rows
         // about to be dropped skip the gate / norm / output projection (their inputs still feed the scan state
@@ -389,10 +410,10 @@ extern "C" int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, con
     // The input is copied in a few row blocks on a stream of the context's own, so that the first layer's norm and
     // projection of block j run while block j+1 is still on its way (pinned host memory makes the copies
     // asynchronous; with pageable memory they simply serialise).  Stream and events are created on first use.
-    constexpr int CHUNKS = 4;
+    constexpr int CHUNKS = 8, OUT_CHUNKS = 4;
     if (!ctx->copy_stream) {
         STR_CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
-        for (int i = 0; i <= CHUNKS; ++i) STR_CUDA_OK(cudaEventCreateWithFlags(&ctx->copy_ev[i], cudaEventDisableTiming));
+        for (int i = 0; i < 18; ++i) STR_CUDA_OK(cudaEventCreateWithFlags(&ctx->copy_ev[i], cudaEventDisableTiming));
     }
     const size_t per = align_up((Rin + CHUNKS - 1) / CHUNKS, 128);          // rows per block: whole GEMM row tiles
     STR_CUDA_OK(cudaEventRecord(ctx->copy_ev[0], st));                       // after whatever the caller queued before
@@ -404,11 +425,13 @@ extern "C" int str_stack_prefill_host(str_ctx *ctx, const str_stack_desc *d, con
                                     cudaMemcpyHostToDevice, ctx->copy_stream));
         STR_CUDA_OK(cudaEventRecord(ctx->copy_ev[1 + nblk], ctx->copy_stream));
     }
-    const StackFeed feed = {nblk, (int)per, ctx->copy_ev + 1};
+    const StackFeed feed = {nblk, (int)per, ctx->copy_ev + 1, OUT_CHUNKS, ctx->copy_ev + 9, ctx->copy_stream, hidden_out_host};
     int rc = stack_prefill_impl(ctx, d, nullptr, in_dev, out_dev, pos_dev, idx_dev, nullptr, nullptr, ws,
                                 workspace_bytes - (size_t)(ws - (char *)workspace), stream, &feed);
     if (rc != STR_OK) return rc;
-    STR_CUDA_OK(cudaMemcpyAsync(hidden_out_host, out_dev, Rout * d->D * e, cudaMemcpyDeviceToHost, st));
+    // the hidden rows have gone out block by block on the copy stream; the caller's stream joins it before returning
+    STR_CUDA_OK(cudaEventRecord(ctx->copy_ev[17], ctx->copy_stream));
+    STR_CUDA_OK(cudaStreamWaitEvent(st, ctx->copy_ev[17], 0));
     if (idx_map_out_host)
         STR_CUDA_OK(cudaMemcpyAsync(idx_map_out_host, idx_dev, Rout * 4, cudaMemcpyDeviceToHost, st));
     STR_CUDA_OK(cudaStreamSynchronize(st));
