@@ -67,3 +67,19 @@ def test_argument_validation_needs_no_gpu(libstr):
     assert libstr.str_relu_squared(None, 1, ctypes.c_size_t(8), None, None, None) == -1
     libstr.str_mamba_importance_dynamic_workspace_size.restype = ctypes.c_size_t
     assert libstr.str_mamba_importance_dynamic_workspace_size(None, 8, 2) == 0
+
+
+def test_newer_entry_points_validate_on_the_host(libstr):
+    c_int, c_float, c_size_t = ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    assert libstr.str_score_density(None, 1, 8, None, c_float(0.8), None, None) == -1
+    assert libstr.str_attn_prefill_rows(None, None, 4, None, None, None, None, c_float(1.0), None, None, c_size_t(0), None) == -1
+    assert libstr.str_stack_prefill_ex(None, None, None, None, None, None, None, None, None, None, c_size_t(0), None) == -1
+    assert libstr.str_selftest_wait_timeout(None, ctypes.c_uint(10), None) == -1
+    tc, fb = ctypes.c_longlong(), ctypes.c_longlong()
+    assert libstr.str_path_counts(None, ctypes.byref(tc), ctypes.byref(fb)) == -1
+    # the schedule helper with layer kinds: unknown kinds and missing arrays are refused
+    a = (c_int * 3)(10000, 5000, 2500)
+    out = (c_int * 3)()
+    assert libstr.str_schedule_keep_counts_layers(a, (c_int * 3)(0, 2, 7), 3, 100, 0, out) == -1
+    assert libstr.str_schedule_keep_counts_layers(a, None, 3, 100, 0, out) == -1
+    assert libstr.str_schedule_keep_counts_layers(a, (c_int * 3)(0, 2, 1), 3, 100, 0, out) == 0 and list(out) == [100, 100, 25]
