@@ -19,7 +19,7 @@ import torch
 
 import oracle
 from paper_2603_00198_b200 import binding, inputs
-from util_gpu import SCORE_TOL, assert_kept_matches, check_layer, dev, host
+from util_gpu import SCORE_TOL, assert_kept_matches, check_layer, check_stack_teacher_forced, dev, host
 
 pytestmark = pytest.mark.gpu
 MS, AT = inputs.MAMBA_8B, inputs.ATTN_8B
@@ -103,38 +103,13 @@ def test_c3_layer_pattern_teacher_forced_at_full_width(ctx, c3_layers, Bz, n_vis
     K = oracle.schedule_keep_counts(cfg["alpha_bp"], n_vis, 0)
     assert K == binding.str_schedule_keep_counts(cfg["alpha_bp"], n_vis, 0) == [n_vis] * 4 + [n_vis // 2] * 4 + [n_vis // 4] * 4
     h0 = inputs.hidden_inputs(seed, n_vis + M, MS["D"], "bf16", batch=Bz)
-    runs = [oracle.stack_prefill(h0[b], M, layers, K, RND, keep_inputs=True) for b in range(Bz)]
-    worst = []
-    for l in range(len(layers)):
-        recs = [runs[b][3][l] for b in range(Bz)]
-        n_in = recs[0]["n_in"]
-        nxt = [(runs[b][3][l + 1]["hidden_in"], runs[b][3][l + 1]["idx_map_in"]) if l + 1 < len(layers)
-               else (runs[b][0], runs[b][2]) for b in range(Bz)]
-        hid = np.stack([r["hidden_in"] for r in recs]).astype(np.float32)
-        pos = np.stack([r["positions_in"] for r in recs])
-        ids = np.stack([r["idx_map_in"] for r in recs])
-        worst.append(check_layer(ctx, layers[l], Bz, n_in, M, K[l], hid, pos, ids, [x[0] for x in nxt], [x[1] for x in nxt],
-                                  recs, Q=MS["Q"]))
+    # Against the oracle's free-running output only the bookkeeping is compared at this width: rounding differences
+    # compound through twelve random-init layers (median row difference 6e-2) and any near-tie swap changes the rows
+    # after it; the per-layer bounds and the composition identity inside the helper are the statement about accuracy.
+    worst, (out, gpos, gidx, tr), runs = check_stack_teacher_forced(ctx, layers, "bf16", Bz, n_vis, M, K, h0, Q=MS["Q"])
     print("max row error per layer:", " ".join("%.1e" % w for w in worst))
-    # The same stack free-running on the GPU.  Its output is, bit for bit, the composition of the single-layer calls
-    # checked above (each fed the previous one's GPU output), so the per-layer bounds are the whole statement about
-    # accuracy; against the oracle's free-running output only the bookkeeping is compared, because rounding differences
-    # compound through twelve random-init layers and any near-tie swap changes the rows after it.
-    st = binding.Stack(ctx, layers, "bf16", Bz, n_vis, M, K, Q=MS["Q"])
-    out, gpos, gidx = binding.str_stack_prefill(st, dev(h0, "bf16"))
-    ctx.check_status()
-    h, p_, i_ = dev(h0, "bf16"), None, None
-    n_cur = n_vis
-    for l in range(len(layers)):
-        one = binding.Stack(ctx, [layers[l]], "bf16", Bz, n_cur, M, [K[l]], Q=MS["Q"])
-        res = binding.str_stack_prefill_ex(one, h, positions_in=p_, idx_map_in=i_)
-        h, p_, i_, n_cur = res["hidden"], res["positions"], res["idx_map"], K[l]
-    ctx.check_status()
-    assert bool((h == out).all()) and bool((i_ == gidx).all()) and bool((p_ == gpos).all())
     for b in range(Bz):
-        gi = gidx[b].cpu().numpy()
-        assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], np.arange(n_vis, n_vis + M))
-        assert len(np.intersect1d(gi, runs[b][2])) >= 0.9 * len(gi)
+        assert len(np.intersect1d(gidx[b].cpu().numpy(), runs[b][2])) >= 0.9 * gidx.shape[1]
     assert bool(torch.isfinite(out.float()).all())
 
 

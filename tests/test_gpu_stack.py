@@ -1,14 +1,16 @@
 """GPU parity for whole layers and the token-reduced stack against the oracle.
 
-Teacher-forced layer tests feed the GPU the oracle's (storage-rounded) layer input, so only one
-layer's arithmetic separates the two.  The free-running stack test lets errors compound.
+Stacks are compared TEACHER-FORCED, layer by layer: GPU layer l is fed the oracle's input of layer l (hidden states
+and carried ids), so exactly one layer's arithmetic separates the two and the layer-level bounds (outputs 2e-2 of the
+maximum, scores 3e-3, selection identical up to near-ties; fp32: 1e-3, 1e-3, 1e-4) are asserted as maxima in every
+layer.  The free-running GPU stack is then shown to be, bit for bit, the composition of those layers.
 """
 import numpy as np
 import pytest
 
 import oracle
 from paper_2603_00198_b200 import binding, inputs
-from util_gpu import assert_kept_matches, dev, host, max_rel_err
+from util_gpu import assert_kept_matches, check_stack_teacher_forced, dev, host, max_rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -74,7 +76,7 @@ def test_hundred_percent_schedule_is_the_unreduced_stack(ctx, dtype):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_progressive_stack_free_running(ctx, dtype):
+def test_progressive_stack(ctx, dtype):
     n_vis, M, Bz = 512, 16, 2
     pattern = "MMAMMA"
     layers = inputs.stack_params(63, pattern, MS, AS, dtype)
@@ -82,26 +84,13 @@ def test_progressive_stack_free_running(ctx, dtype):
     alpha = [10000, 10000, 5000, 5000, 2500, 2500]
     K = binding.str_schedule_keep_counts(alpha, n_vis, 16)
     assert K == oracle.schedule_keep_counts(alpha, n_vis, 16) == [512, 512, 256, 256, 128, 128]
-    st = binding.Stack(ctx, layers, dtype, Bz, n_vis, M, K)
-    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, dtype), want_trace=True)
+    worst, (out, pos, idx, tr), runs = check_stack_teacher_forced(ctx, layers, dtype, Bz, n_vis, M, K, h0)
     assert [t["layer"] for t in tr] == [2, 4] and out.shape == (Bz, 128 + M, 128)
     for b in range(Bz):
-        ref, rpos, ridx, trace = oracle.stack_prefill(h0[b], M, layers, K, _rnd(dtype))
-        gi = idx[b].cpu().numpy()
-        assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], np.arange(n_vis, n_vis + M))
-        assert np.array_equal(pos[b].cpu().numpy(), gi)
-        # first reducing layer (attention, layer index 2): both sides still see the same tokens
-        swaps = assert_kept_matches(tr[0]["kept"][b].cpu().numpy(), trace[2]["kept"], trace[2]["scores"],
-                                    tol=1e-3 if dtype == "f32" else 5e-3)
-        common, a, c = np.intersect1d(gi, ridx, return_indices=True)
-        assert len(common) >= 0.97 * len(ridx)
-        row_err = np.abs(host(out)[b][a] - ref[c]).max(axis=1) / np.abs(ref).max()
-        if swaps == 0 and len(common) == len(ridx):
-            assert row_err.max() <= (5e-2 if dtype == "bf16" else 2e-3)
-        else:
-            # a legitimate near-tie swap changes the conv / state context of the rows after it, so only
-            # the bulk of the rows can be compared once the two runs keep different tokens
-            assert np.median(row_err) <= 2e-2 and (row_err > 5e-2).mean() <= 0.25
+        # the first reducing layer (attention, layer index 2) of the free-running stack still sees nearly the oracle's
+        # tokens: its selection matches up to near-ties
+        assert_kept_matches(tr[0]["kept"][b].cpu().numpy(), runs[b][3][2]["kept"], runs[b][3][2]["scores"],
+                            tol=1e-3 if dtype == "f32" else 5e-3)
 
 
 def test_host_buffer_entry_point_matches_device_entry_point(ctx):
@@ -132,23 +121,11 @@ def test_all_layer_sigmoid_schedule(ctx):
     assert K == oracle.schedule_keep_counts(alpha, n_vis, 16)
     reducing = [l for l, (a, b) in enumerate(zip([n_vis] + K, K)) if b < a]
     assert len(reducing) >= 5 and 2 in reducing                      # Mamba and attention layers both cut
-    st = binding.Stack(ctx, layers, "bf16", 1, n_vis, M, K)
-    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, "bf16"), want_trace=True)
+    worst, (out, pos, idx, tr), runs = check_stack_teacher_forced(ctx, layers, "bf16", 1, n_vis, M, K, h0)
     assert [t["layer"] for t in tr] == reducing and out.shape == (1, K[-1] + M, 128)
-    ref, rpos, ridx, trace = oracle.stack_prefill(h0[0], M, layers, K, oracle.round_to_bf16)
-    gi = idx[0].cpu().numpy()
-    assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], np.arange(n_vis, n_vis + M))
-    # layer 0 sees identical tokens on both sides: its selection must match up to near-ties
-    assert_kept_matches(tr[0]["kept"][0].cpu().numpy(), trace[0]["kept"], trace[0]["scores"], tol=5e-3)
-    # every later selection is the oracle's rule applied to the scores the GPU produced
+    # every selection of the free-running stack is the oracle's rule applied to the scores the GPU produced
     for t in tr:
         assert np.array_equal(t["kept"][0].cpu().numpy(), oracle.topk_select(t["scores"][0].cpu().numpy(), K[t["layer"]]))
-    common, a, c = np.intersect1d(gi, ridx, return_indices=True)
-    assert len(common) >= 0.9 * len(ridx)
-    # six cuts in a row: a near-tie swap at any of them changes the context of every later row, so only the
-    # bulk of the surviving rows is compared, loosely
-    row_err = np.abs(host(out)[0][a] - ref[c]).max(axis=1) / np.abs(ref).max()
-    assert np.median(row_err) <= 5e-2
 
 
 MS_TC = dict(D=512, H=8, p=64, n=128, G=2, Q=128, conv=4)      # shapes the tensor-core kernels tile
@@ -228,23 +205,9 @@ def test_hybrid_stack_with_ffn_layers(ctx, dtype):
     layers = inputs.stack_params(68, pattern, MS, AS, dtype, ffn_dim=320)
     h0 = inputs.hidden_inputs(68, n_vis + M, 128, dtype, batch=Bz)
     K = [512, 512, 256, 256, 128, 128]
-    st = binding.Stack(ctx, layers, dtype, Bz, n_vis, M, K)
-    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, dtype), want_trace=True)
-    ctx.check_status()
+    assert K == binding.str_schedule_keep_counts_layers([10000, 5000, 5000, 2500, 2500, 2500], pattern, n_vis, 16)
+    worst, (out, pos, idx, tr), runs = check_stack_teacher_forced(ctx, layers, dtype, Bz, n_vis, M, K, h0)
     assert [t["layer"] for t in tr] == [2, 4] and out.shape == (Bz, 128 + M, 128)
-    for b in range(Bz):
-        ref, rpos, ridx, trace = oracle.stack_prefill(h0[b], M, layers, K, _rnd(dtype))
-        gi = idx[b].cpu().numpy()
-        assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], np.arange(n_vis, n_vis + M))
-        swaps = assert_kept_matches(tr[0]["kept"][b].cpu().numpy(), trace[2]["kept"], trace[2]["scores"],
-                                    tol=1e-3 if dtype == "f32" else 5e-3)
-        common, a, c = np.intersect1d(gi, ridx, return_indices=True)
-        assert len(common) >= 0.97 * len(ridx)
-        row_err = np.abs(host(out)[b][a] - ref[c]).max(axis=1) / np.abs(ref).max()
-        if swaps == 0 and len(common) == len(ridx):
-            assert row_err.max() <= (5e-2 if dtype == "bf16" else 2e-3)
-        else:
-            assert np.median(row_err) <= 2e-2 and (row_err > 5e-2).mean() <= 0.25
     # a keep count that would make an FFN layer reduce is refused
     with pytest.raises(Exception):
         bad = binding.Stack(ctx, layers, dtype, Bz, n_vis, M, [512, 256, 256, 256, 128, 128])
@@ -264,10 +227,7 @@ def test_single_ffn_layer_teacher_forced(ctx):
 def test_transformer_stack_reducing_at_every_attention_layer_batch_8(ctx):
     """The second workload of the paper's appendix "Models": a pure Transformer (attention + FFN blocks) under the
     all-layer sigmoid schedule, so that every attention layer scores, selects and compacts (FFN layers pass the rows
-    on), at batch 8 and on tensor-core shapes.  Teacher-forced per layer: each GPU layer gets the oracle's input of
-    that layer, so the maximum row error is asserted in every layer; the free-running GPU stack is then shown to be
-    exactly the composition of those layers."""
-    from util_gpu import check_layer
+    on), at batch 8 and on tensor-core shapes."""
     Bz, n_vis, M = 8, 900, 28
     pattern = "AFAFAFAF"
     layers = inputs.stack_params(71, pattern, None, AS_TC, "bf16", ffn_dim=1024)
@@ -277,21 +237,5 @@ def test_transformer_stack_reducing_at_every_attention_layer_batch_8(ctx):
     cuts = [l for l, (a, b) in enumerate(zip([n_vis] + K, K)) if b < a]
     assert cuts == [0, 2, 4, 6]                                   # every attention layer reduces, no FFN layer does
     h0 = inputs.hidden_inputs(71, n_vis + M, AS_TC["D"], "bf16", batch=Bz)
-    runs = [oracle.stack_prefill(h0[b], M, layers, K, oracle.round_to_bf16, keep_inputs=True) for b in range(Bz)]
-    for l in range(len(layers)):
-        recs = [runs[b][3][l] for b in range(Bz)]
-        nxt = [(runs[b][3][l + 1]["hidden_in"], runs[b][3][l + 1]["idx_map_in"]) if l + 1 < len(layers)
-               else (runs[b][0], runs[b][2]) for b in range(Bz)]
-        check_layer(ctx, layers[l], Bz, recs[0]["n_in"], M, K[l], np.stack([r["hidden_in"] for r in recs]).astype(np.float32),
-                    np.stack([r["positions_in"] for r in recs]), np.stack([r["idx_map_in"] for r in recs]),
-                    [x[0] for x in nxt], [x[1] for x in nxt], recs)
-    st = binding.Stack(ctx, layers, "bf16", Bz, n_vis, M, K)
-    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, "bf16"), want_trace=True)
-    ctx.check_status()
+    worst, (out, pos, idx, tr), runs = check_stack_teacher_forced(ctx, layers, "bf16", Bz, n_vis, M, K, h0)
     assert [t["layer"] for t in tr] == cuts and out.shape == (Bz, K[-1] + M, AS_TC["D"])
-    h, p_, i_, n_cur = dev(h0, "bf16"), None, None, n_vis
-    for l in range(len(layers)):
-        one = binding.Stack(ctx, [layers[l]], "bf16", Bz, n_cur, M, [K[l]])
-        res = binding.str_stack_prefill_ex(one, h, positions_in=p_, idx_map_in=i_)
-        h, p_, i_, n_cur = res["hidden"], res["positions"], res["idx_map"], K[l]
-    assert bool((h == out).all()) and bool((i_ == idx).all())

@@ -58,15 +58,21 @@ def row_err(got, ref):
     return float(np.abs(got - ref).max() / np.abs(ref).max())
 
 
-def check_layer(ctx, layer, Bz, n_in, M, K, hid_in, pos_in, idx_in, ref_out, ref_idx, rec, Q=0):
+# Layer-level bounds by storage type: (output max row error, score deviation = swap tolerance).  fp32 storage has no
+# rounding points between the kernels, so the kernel-level bounds apply unchanged.
+LAYER_TOL = {"bf16": (2e-2, SCORE_TOL), "f32": (1e-3, 1e-3)}
+
+
+def check_layer(ctx, layer, Bz, n_in, M, K, hid_in, pos_in, idx_in, ref_out, ref_idx, rec, Q=0, dtype="bf16", **stack_kw):
     """One layer on the GPU, fed `hid_in` [Bz, n_in+M, D] with its carried ids; compared with the oracle's output of
     the same layer (`ref_out`, `ref_idx` per sequence) and, when it reduces, with the oracle's scores and selection."""
     from paper_2603_00198_b200 import binding
-    st = binding.Stack(ctx, [layer], "bf16", Bz, n_in, M, [K], Q=Q)
-    res = binding.str_stack_prefill_ex(st, dev(hid_in, "bf16"), positions_in=dev(pos_in), idx_map_in=dev(idx_in), want_trace=True)
+    out_tol, score_tol = LAYER_TOL[dtype]
+    swap_tol = score_tol if dtype == "bf16" else 1e-4
+    st = binding.Stack(ctx, [layer], dtype, Bz, n_in, M, [K], Q=Q, **stack_kw)
+    res = binding.str_stack_prefill_ex(st, dev(hid_in, dtype), positions_in=dev(pos_in), idx_map_in=dev(idx_in), want_trace=True)
     ctx.check_status()
     out, gidx = host(res["hidden"]), res["idx_map"].cpu().numpy()
-    assert np.array_equal(res["positions"].cpu().numpy(), gidx)
     worst = 0.0
     for b in range(Bz):
         gi = gidx[b]
@@ -74,13 +80,54 @@ def check_layer(ctx, layer, Bz, n_in, M, K, hid_in, pos_in, idx_in, ref_out, ref
         if K < n_in:
             s_gpu, kept = res["trace"][0]["scores"][b].cpu().numpy(), res["trace"][0]["kept"][b].cpu().numpy()
             s_ref = rec[b]["scores"]
-            assert np.abs(s_gpu / s_ref - 1).max() <= SCORE_TOL
-            assert_kept_matches(kept, rec[b]["kept"], s_ref, tol=SCORE_TOL)
+            big = s_ref >= 1e-20 * s_ref.max()          # the Eq. 1 score variant underflows far from the text
+            assert np.abs(s_gpu[big] / s_ref[big] - 1).max() <= score_tol
+            assert_kept_matches(kept, rec[b]["kept"], s_ref, tol=swap_tol)
             assert np.array_equal(gi[:K], idx_in[b][kept])            # ids bit-exact given the selection
         else:
             assert np.array_equal(gi, idx_in[b])
         common, a, c = np.intersect1d(gi, ref_idx[b], return_indices=True)
         assert len(common) >= 0.98 * len(ref_idx[b])
         worst = max(worst, row_err(out[b][a], ref_out[b][c]))
-    assert worst <= 2e-2, worst
+    assert worst <= out_tol, worst
     return worst
+
+
+def check_stack_teacher_forced(ctx, layers, dtype, Bz, n_vis, M, K, h0, Q=0, **kw):
+    """The stack against the oracle, layer by layer: GPU layer l is fed the oracle's input of layer l (hidden states and
+    carried ids), so exactly one layer's arithmetic separates the two and the layer-level bounds are asserted as
+    maxima in every layer.  Then the free-running GPU stack is shown to be, bit for bit, the composition of its layers
+    run one by one.  `kw`: mamba_score / attn_denominator, passed to both sides.  Returns (per-layer worst row error,
+    the free-running outputs (hidden, positions, idx_map, trace), the oracle runs)."""
+    import oracle
+    from paper_2603_00198_b200 import binding
+    rnd = oracle.round_to_bf16 if dtype == "bf16" else oracle._identity
+    okw = {}
+    if "mamba_score" in kw:
+        okw["mamba_score"] = kw["mamba_score"]
+    if "attn_denominator" in kw:
+        okw["attn_denominator"] = kw["attn_denominator"]
+    runs = [oracle.stack_prefill(h0[b], M, layers, K, rnd, keep_inputs=True, **okw) for b in range(Bz)]
+    worst = []
+    for l in range(len(layers)):
+        recs = [runs[b][3][l] for b in range(Bz)]
+        nxt = [(runs[b][3][l + 1]["hidden_in"], runs[b][3][l + 1]["idx_map_in"]) if l + 1 < len(layers)
+               else (runs[b][0], runs[b][2]) for b in range(Bz)]
+        worst.append(check_layer(ctx, layers[l], Bz, recs[0]["n_in"], M, K[l],
+                                 np.stack([r["hidden_in"] for r in recs]).astype(np.float32),
+                                 np.stack([r["positions_in"] for r in recs]), np.stack([r["idx_map_in"] for r in recs]),
+                                 [x[0] for x in nxt], [x[1] for x in nxt], recs, Q=Q, dtype=dtype, **kw))
+    st = binding.Stack(ctx, layers, dtype, Bz, n_vis, M, K, Q=Q, **kw)
+    out, pos, idx, tr = binding.str_stack_prefill(st, dev(h0, dtype), want_trace=True)
+    ctx.check_status()
+    h, p_, i_, n_cur = dev(h0, dtype), None, None, n_vis
+    for l in range(len(layers)):
+        one = binding.Stack(ctx, [layers[l]], dtype, Bz, n_cur, M, [K[l]], Q=Q, **kw)
+        res = binding.str_stack_prefill_ex(one, h, positions_in=p_, idx_map_in=i_)
+        h, p_, i_, n_cur = res["hidden"], res["positions"], res["idx_map"], K[l]
+    ctx.check_status()
+    assert bool((h == out).all()) and bool((i_ == idx).all()) and bool((p_ == pos).all())
+    for b in range(Bz):
+        gi = idx[b].cpu().numpy()
+        assert np.all(np.diff(gi) > 0) and np.array_equal(gi[-M:], np.arange(n_vis, n_vis + M))
+    return worst, (out, pos, idx, tr), runs
