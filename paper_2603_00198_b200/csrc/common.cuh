@@ -25,6 +25,7 @@ struct str_ctx {
     long long tc_calls;       // entry-point calls that took a tensor-core (tcgen05) kernel
     long long fallback_calls; // entry-point calls that took the plain fp32-FMA kernel of the same entry point
     size_t smem_attr[8];      // dynamic shared memory already opted into on this device, per tensor-core kernel
+    int gemm_pairs;           // CTA pairs the GEMM can keep resident (0 = not asked yet, -1 = pairs unavailable)
     cudaStream_t copy_stream; // host-buffer entry point: input chunks are copied on this stream while the caller's
     cudaEvent_t copy_ev[24];  // stream computes; [0] orders the copies after the caller's earlier work, [1..8] = input
                               // chunk landed, [9..16] = output row block computed, [17] = output copies done
@@ -64,7 +65,7 @@ static inline int str_launch_ok(str_ctx *ctx, int n = 1) {
 // Opt a kernel into `bytes` of dynamic shared memory once per context (the attribute belongs to the device the
 // context was created on, so it is tracked per context, not per process).
 enum { STR_SMEM_GEMM = 0, STR_SMEM_SSD, STR_SMEM_ATTN_FWD, STR_SMEM_MAMBA_SCORE, STR_SMEM_ATTN_ROWSTATS, STR_SMEM_ATTN_COLSUM,
-       STR_SMEM_MAMBA_DYN_SCORE };
+       STR_SMEM_MAMBA_DYN_SCORE, STR_SMEM_GEMM_PAIR };
 template <typename F>
 static inline int str_ensure_smem(str_ctx *ctx, int slot, F kernel, size_t bytes) {
     // The attribute belongs to the device's copy of the kernel, not to this context: every context raises it to

@@ -17,6 +17,7 @@ extern "C" int str_create(int device, str_ctx **out) {
     c->tc_calls = 0;
     c->fallback_calls = 0;
     c->prof_on = false;
+    c->gemm_pairs = 0;
     for (size_t &v : c->smem_attr) v = 0;
     c->copy_stream = nullptr;
     for (cudaEvent_t &ev : c->copy_ev) ev = nullptr;

@@ -14,6 +14,8 @@
 // row by 1/rms of the A row (from partial sums of squares left by the kernel that wrote A), and it leaves the
 // partial sums of squares of its own output rows, one per 256-column tile, for the next projection.
 // Every mbarrier wait is bounded; on give-up the kernel records STR_ERR_TIMEOUT and tears down.
+#include <stdlib.h>
+
 #include "dispatch.cuh"
 #include "tc_common.cuh"
 
@@ -32,6 +34,66 @@ __device__ __forceinline__ TileCoord tile_coord(int t, int tiles_m, int tiles_n)
     const int n0 = band * BAND;
     const int width = min(BAND, tiles_n - n0);
     return {r / width, n0 + r % width};
+}
+
+// Epilogue of one accumulator row: this thread owns tensor-memory lane `taddr`'s lane field = output row `row`, columns
+// [256 tile_n, 256 tile_n + 256).  Fused RMSNorm of the A rows: 1/rms from the partial sums of squares the producer
+// of A left behind, summed in index order (deterministic), applied to the accumulator row; then the residual, the
+// narrowing to bf16, 16-byte stores, and the partial sum of squares of the stored values in column order.
+__device__ __forceinline__ void store_rows(uint32_t taddr, int row, int tile_n, int tiles_n, int M, int N,
+                                           const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ out,
+                                           const StrRowNorm &rn) {
+    const int col0 = tile_n * BN;
+    float scale = 1.0f;
+    if (rn.ss_in && row < M) {
+        float t = 0.f;
+        for (int j = 0; j < rn.nt_in; ++j) t += __ldg(rn.ss_in + (size_t)row * rn.nt_in + j);
+        scale = rsqrtf(t * rn.inv_dim + rn.eps);
+    }
+    float ss = 0.f;                              // sum of squares of this row's stored outputs in this tile
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 32) {
+        uint32_t v[32];
+        tc::tmem_ld32(taddr + c, v);
+        tc::tmem_ld_wait();
+        if (row < M && col0 + c < N) {
+            const size_t off = (size_t)row * N + col0 + c;
+            const int valid = min(32, N - (col0 + c));       // multiple of 8 (N % 8 == 0)
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                if (g * 8 < valid) {
+                    float f[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]) * scale;
+                    if (residual) {
+                        const uint4 r = *reinterpret_cast<const uint4 *>(residual + off + g * 8);
+                        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            f[2 * j] += __uint_as_float(rw[j] << 16);
+                            f[2 * j + 1] += __uint_as_float(rw[j] & 0xFFFF0000u);
+                        }
+                    }
+                    uint4 o;
+                    o.x = tc::pack_bf16x2(f[0], f[1]);
+                    o.y = tc::pack_bf16x2(f[2], f[3]);
+                    o.z = tc::pack_bf16x2(f[4], f[5]);
+                    o.w = tc::pack_bf16x2(f[6], f[7]);
+                    *reinterpret_cast<uint4 *>(out + off + g * 8) = o;
+                    if (rn.ss_out) {
+                        const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float lo = __uint_as_float(ow[j] << 16), hi = __uint_as_float(ow[j] & 0xFFFF0000u);
+                            ss = fmaf(lo, lo, ss);
+                            ss = fmaf(hi, hi, ss);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (rn.ss_out && row < M) rn.ss_out[(size_t)row * tiles_n + tile_n] = ss;
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -126,61 +188,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const uint32_t aph = (local >> 1) & 1;
             if (!tc::mbar_wait(acc_full + acc, aph, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
-            const int row = tc_.m * BM + quad * 32 + lane;
-            const int col0 = tc_.n * BN;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN;
-            // fused RMSNorm of the A rows: 1/rms from the partial sums of squares the producer of A left behind, summed
-            // in index order (deterministic), applied to the accumulator row
-            float scale = 1.0f;
-            if (rn.ss_in && row < M) {
-                float t = 0.f;
-                for (int j = 0; j < rn.nt_in; ++j) t += __ldg(rn.ss_in + (size_t)row * rn.nt_in + j);
-                scale = rsqrtf(t * rn.inv_dim + rn.eps);
-            }
-            float ss = 0.f;                              // sum of squares of this row's stored outputs in this tile
-#pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t v[32];
-                tc::tmem_ld32(taddr + c, v);
-                tc::tmem_ld_wait();
-                if (row < M && col0 + c < N) {
-                    const size_t off = (size_t)row * N + col0 + c;
-                    const int valid = min(32, N - (col0 + c));       // multiple of 8 (N % 8 == 0)
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        if (g * 8 < valid) {
-                            float f[8];
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]) * scale;
-                            if (residual) {
-                                const uint4 r = *reinterpret_cast<const uint4 *>(residual + off + g * 8);
-                                const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    f[2 * j] += __uint_as_float(rw[j] << 16);
-                                    f[2 * j + 1] += __uint_as_float(rw[j] & 0xFFFF0000u);
-                                }
-                            }
-                            uint4 o;
-                            o.x = tc::pack_bf16x2(f[0], f[1]);
-                            o.y = tc::pack_bf16x2(f[2], f[3]);
-                            o.z = tc::pack_bf16x2(f[4], f[5]);
-                            o.w = tc::pack_bf16x2(f[6], f[7]);
-                            *reinterpret_cast<uint4 *>(out + off + g * 8) = o;
-                            if (rn.ss_out) {
-                                const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    const float lo = __uint_as_float(ow[j] << 16), hi = __uint_as_float(ow[j] & 0xFFFF0000u);
-                                    ss = fmaf(lo, lo, ss);
-                                    ss = fmaf(hi, hi, ss);
-                                }
-                            }
-                        }
-                    }
-                }
-            }
-            if (rn.ss_out && row < M) rn.ss_out[(size_t)row * tiles_n + tc_.n] = ss;
+            store_rows(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN, tc_.m * BM + quad * 32 + lane,
+                       tc_.n, tiles_n, M, N, residual, out, rn);
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(acc_empty + acc);
@@ -192,6 +201,128 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, 512); }
 }
 
+// ---- the same GEMM on CTA pairs ------------------------------------------------------------------
+// A cluster of two CTAs on neighbouring SMs owns a 256 x 256 output tile and runs it as ONE tcgen05.mma of M = 256
+// per K-slice (cta_group::2), issued by CTA 0.  CTA r stages rows [128 r, 128 r + 128) of the A tile and rows
+// [128 r, 128 r + 128) of the W tile, so an SM moves 8 KB of operands per K-slice through its shared memory instead
+// of 12 KB, and holds rows [128 r, 128 r + 128) of the accumulator in its own tensor memory; its four epilogue warps
+// store them exactly as the lone-CTA kernel does (same arithmetic in the same order: the outputs are bit-identical).
+// Barriers: each CTA has its own `empty` ring (CTA 0's commit arrives on both) and `acc_full` pair (likewise); the
+// `full` ring and the `acc_empty` pair that count are CTA 0's: both producers' copies complete their bytes there,
+// and both CTAs' epilogue warps arrive there.
+constexpr int P_BM = 256, P_STAGES = 6;
+constexpr int P_A_BYTES = 128 * BK * 2, P_W_BYTES = 128 * BK * 2, P_STAGE_BYTES = P_A_BYTES + P_W_BYTES;
+constexpr size_t P_SMEM_BYTES = 1024 /*align slack*/ + (size_t)P_STAGES * P_STAGE_BYTES + 256;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w, int M, int N,
+                    int K, const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ out, StrRowNorm rn,
+                    int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = (uint64_t *)(smem + (size_t)P_STAGES * P_STAGE_BYTES);
+    uint64_t *full = bars, *empty = bars + P_STAGES, *acc_full = bars + 2 * P_STAGES, *acc_empty = bars + 2 * P_STAGES + 2;
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * P_STAGES + 4);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = tc::cluster_cta_rank();
+    const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+    const int tiles_m = (M + P_BM - 1) / P_BM, tiles_n = (N + BN - 1) / BN, tiles = tiles_m * tiles_n;
+    const int k_blocks = (K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P_STAGES; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, 1); }
+        for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, 8); }
+        abort_flag[0] = 0;
+        tc::fence_mbar_init();
+        tc::prefetch_tmap(&tmap_a);
+        tc::prefetch_tmap(&tmap_w);
+    }
+    __syncthreads();
+    tc::cluster_sync_all();                  // both CTAs' barriers exist before anything can signal them
+    if (warp == 1) { tc::tmem_alloc_pair(tmem_slot, 512); tc::tmem_relinquish_pair(); }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::cluster_sync_all();                  // both halves of the accumulator are allocated before the first MMA
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int t = pair; t < tiles && ok; t += pairs) {
+                const TileCoord tc_ = tile_coord(t, tiles_m, tiles_n);
+                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                    const int s = it % P_STAGES;
+                    const uint32_t ph = (it / P_STAGES) & 1;
+                    if (!tc::mbar_wait(empty + s, ph ^ 1, abort_flag)) { ok = false; break; }
+                    if (rank == 0) tc::mbar_arrive_expect_tx(full + s, 2 * P_STAGE_BYTES);
+                    const uint32_t full_cta0 = tc::map_to_cta(full + s, 0);
+                    uint8_t *sa = smem + (size_t)s * P_STAGE_BYTES;
+                    tc::tma_load_2d_pair(sa, &tmap_a, full_cta0, kb * BK, tc_.m * P_BM + (int)rank * 128);
+                    tc::tma_load_2d_pair(sa + P_A_BYTES, &tmap_w, full_cta0, kb * BK, tc_.n * BN + (int)rank * 128);
+                }
+            }
+            // every commit aimed at this CTA's ring has arrived before the CTA may leave
+            for (int back = 0; back < P_STAGES && ok; ++back, ++it)
+                if (!tc::mbar_wait(empty + it % P_STAGES, ((it / P_STAGES) & 1) ^ 1, abort_flag)) ok = false;
+            if (!ok) {
+                atomicCAS(status, 0, STR_ERR_TIMEOUT);
+                for (int i = 0; i < 2000; ++i) __nanosleep(1000);    // copies already issued land before the CTA leaves
+            }
+        }
+    } else if (warp == 1) {
+        if (rank == 0 && tc::elect_one()) {
+            const uint32_t idesc = tc::make_idesc_bf16(P_BM, BN, 0, 0);
+            int it = 0, local = 0;
+            bool ok = true;
+            for (int t = pair; t < tiles && ok; t += pairs, ++local) {
+                const int acc = local & 1;
+                const uint32_t aph = (local >> 1) & 1;
+                if (!tc::mbar_wait(acc_empty + acc, aph ^ 1, abort_flag)) { ok = false; break; }
+                tc::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
+                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                    const int s = it % P_STAGES;
+                    const uint32_t ph = (it / P_STAGES) & 1;
+                    if (!tc::mbar_wait(full + s, ph, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint32_t sa = tc::smem_u32(smem + (size_t)s * P_STAGE_BYTES);
+                    tc::mma4_ss_pair<tc::StepKMajor64, tc::StepKMajor64>(d_tmem, tc::desc_kmajor_sw128(sa, 0),
+                                                                         tc::desc_kmajor_sw128(sa + P_A_BYTES, 0), idesc, kb != 0);
+                    tc::mma_commit_pair(empty + s, 3);
+                }
+                if (ok) tc::mma_commit_pair(acc_full + acc, 3);
+            }
+            if (!ok) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+        }
+        __syncwarp();
+    } else {
+        const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
+        int local = 0;
+        bool ok = true;
+        for (int t = pair; t < tiles && ok; t += pairs, ++local) {
+            const TileCoord tc_ = tile_coord(t, tiles_m, tiles_n);
+            const int acc = local & 1;
+            const uint32_t aph = (local >> 1) & 1;
+            if (!tc::mbar_wait(acc_full + acc, aph, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after();
+            store_rows(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN,
+                       tc_.m * P_BM + (int)rank * 128 + quad * 32 + lane, tc_.n, tiles_n, M, N, residual, out, rn);
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_cta(acc_empty + acc, 0));
+        }
+        if (!ok && lane == 0) atomicCAS(status, 0, STR_ERR_TIMEOUT);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::cluster_sync_all();                  // neither CTA leaves, or frees tensor memory, while the other still works
+    if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc_pair(tmem_base, 512); }
+}
+
 }  // namespace
 
 bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const void *w, const void *residual,
@@ -201,13 +332,50 @@ bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const 
     return (al & 15) == 0;
 }
 
+// How many CTA pairs the device runs at once (one per SM pair that a cluster of two can occupy), found once per
+// context; 0 when clusters of two cannot be launched or STR_GEMM_PAIR=0 asks for the lone-CTA kernel (A/B runs).
+static int str_gemm_pairs(str_ctx *ctx) {
+    if (ctx->gemm_pairs != 0) return ctx->gemm_pairs > 0 ? ctx->gemm_pairs : 0;
+    ctx->gemm_pairs = -1;
+    const char *e = getenv("STR_GEMM_PAIR");
+    if (e && e[0] == '0') return 0;
+    if (str_ensure_smem(ctx, STR_SMEM_GEMM_PAIR, gemm_tc_pair_kernel, P_SMEM_BYTES) != STR_OK) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * ctx->sm_count);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = P_SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, gemm_tc_pair_kernel, &cfg) != cudaSuccess || clusters < 1) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    ctx->gemm_pairs = clusters;
+    return clusters;
+}
+
 int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
                 const StrRowNorm &rn, cudaStream_t st) {
+    // CTA pairs whenever the problem has more than one row tile and the device can co-schedule clusters of two
+    const bool paired = M > BM && str_gemm_pairs(ctx) > 0;
     CUtensorMap ta, tw;
     int rc = str_make_tmap_2d_bf16(ctx, &ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != STR_OK) return rc;
-    rc = str_make_tmap_2d_bf16(ctx, &tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN, BK, CU_TENSOR_MAP_SWIZZLE_128B);
+    rc = str_make_tmap_2d_bf16(ctx, &tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, paired ? 128 : BN, BK, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != STR_OK) return rc;
+    if (paired) {
+        const int tiles = ceil_div(M, P_BM) * ceil_div(N, BN);
+        const int pairs = tiles < ctx->gemm_pairs ? tiles : ctx->gemm_pairs;
+        gemm_tc_pair_kernel<<<2 * pairs, NUM_THREADS, P_SMEM_BYTES, st>>>(ta, tw, M, N, K, (const __nv_bfloat16 *)residual,
+                                                                         (__nv_bfloat16 *)out, rn, ctx->status_dev);
+        return str_launch_ok(ctx);
+    }
     rc = str_ensure_smem(ctx, STR_SMEM_GEMM, gemm_tc_kernel, SMEM_BYTES);
     if (rc != STR_OK) return rc;
     const int tiles = ceil_div(M, BM) * ceil_div(N, BN);

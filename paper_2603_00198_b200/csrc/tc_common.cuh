@@ -245,6 +245,71 @@ __device__ __forceinline__ void mma_commit(uint64_t *bar) {
                  : "memory");
 }
 
+// ---- CTA pairs (cta_group::2) ------------------------------------------------------------------
+// Two CTAs of a cluster of two, on neighbouring SMs, run ONE tcgen05.mma of M = 256: CTA r holds rows
+// [128 r, 128 r + 128) of A, rows [N/2 r, N/2 r + N/2) of B (both at the same shared-memory offsets in the two CTAs)
+// and, in its own tensor memory, rows [128 r, 128 r + 128) of the accumulator.  The instruction is issued by one
+// thread of CTA 0 only.  Each SM then reads half the B operand per K-slice that a lone CTA reads for the same
+// accumulator width.  Tensor memory is allocated and freed by the same warp of BOTH CTAs.
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// All threads of all CTAs of the cluster; orders shared-memory accesses (mbarrier initialisation included) across it.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The shared::cluster address of `p`'s counterpart (same offset) in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(const void *p, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Tile load into this CTA's shared memory whose bytes are counted on an mbarrier that may live in the pair's
+// other CTA (given by its shared::cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(void *smem_dst, const CUtensorMap *m, uint32_t bar_cluster_addr, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"((uint64_t)m), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t *smem_slot, uint32_t ncols) {   // whole warp, same warp in both CTAs
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {      // whole warp, same warp in both CTAs
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// Four K-slices (one 64-column stage) of a pair MMA, both operands in shared memory; issued by ONE thread of CTA 0.
+template <class SA, class SB>
+__device__ __forceinline__ void mma4_ss_pair(uint32_t d_tmem, uint64_t a0, uint64_t b0, uint32_t idesc, bool acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred pf, pt;\n\t.reg .b64 a, b;\n\t"
+        "setp.ne.b32 pf, %4, 0;\n\tsetp.eq.u32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, pf;\n\t"
+        "add.s64 a, %1, %5;\n\tadd.s64 b, %2, %6;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], a, b, %3, pt;\n\t"
+        "add.s64 a, %1, %7;\n\tadd.s64 b, %2, %8;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], a, b, %3, pt;\n\t"
+        "add.s64 a, %1, %9;\n\tadd.s64 b, %2, %10;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], a, b, %3, pt;\n\t"
+        "}"
+        ::"r"(d_tmem), "l"(a0), "l"(b0), "r"(idesc), "r"((uint32_t)acc_first),
+          "n"(SA::at(1)), "n"(SB::at(1)), "n"(SA::at(2)), "n"(SB::at(2)), "n"(SA::at(3)), "n"(SB::at(3))
+        : "memory");
+}
+// Arrive, once all pair MMAs issued so far by this thread have completed, on the mbarrier at this offset in each CTA
+// of `cta_mask` (bit r = CTA r of the cluster).
+__device__ __forceinline__ void mma_commit_pair(uint64_t *bar, uint16_t cta_mask) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(cta_mask)
+                 : "memory");
+}
+
 // TMEM -> registers: 32 lanes x 32-bit, 32 consecutive columns; thread i of the warp reads lane
 // (lane_base + i).  The warp may only touch the lane quadrant 32*(warp_id % 4).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {

@@ -34,6 +34,26 @@ def test_gemm_with_residual(ctx, dtype, M, N, K):
     assert max_rel_err(got, ref + r) <= TOL[dtype]
 
 
+@pytest.mark.parametrize("M,N,K", [(129, 256, 64), (300, 200, 256), (1056, 1184, 256), (257, 136, 8192), (8320, 2304, 1024)])
+def test_gemm_on_cta_pairs_is_bit_identical_to_the_lone_cta_kernel(M, N, K, monkeypatch):
+    """Above 128 rows the GEMM runs on CTA pairs (one 256-row MMA per K-slice across two SMs); a context created with
+    STR_GEMM_PAIR=0 keeps the one-CTA kernel.  Same K order, same epilogue arithmetic: the outputs must be equal bit
+    for bit, with and without the residual, on ragged M, N and K."""
+    g = inputs.rng(57, M + N + K)
+    a = dev(inputs.to_grid(g.standard_normal((M, K), dtype=np.float32), "bf16"), "bf16")
+    w = dev(inputs.to_grid(g.standard_normal((N, K), dtype=np.float32) / np.sqrt(K), "bf16"), "bf16")
+    r = dev(inputs.to_grid(g.standard_normal((M, N), dtype=np.float32), "bf16"), "bf16")
+    outs = []
+    for flag in ("0", "1"):
+        monkeypatch.setenv("STR_GEMM_PAIR", flag)
+        c = binding.Context(0)
+        outs.append((binding.str_gemm(c, a, w), binding.str_gemm(c, a, w, residual=r)))
+        c.check_status()
+        assert c.path_counts() == (2, 0)
+        c.close()
+    assert bool((outs[0][0] == outs[1][0]).all()) and bool((outs[0][1] == outs[1][1]).all())
+
+
 @pytest.mark.parametrize("dtype,rows,D", [("bf16", 100, 4096), ("f32", 33, 256), ("bf16", 5, 40), ("bf16", 9, 8192),
                                           ("bf16", 3, 36)])
 def test_rmsnorm(ctx, dtype, rows, D):
