@@ -223,6 +223,20 @@ int str_mamba_conv_split(str_ctx *ctx, int dtype, int Bz, int T, int H, int p, i
                          const float *dt_bias, void *x_out, void *B_out, void *C_out, float *dt_out,
                          void *stream);
 
+/* The Mamba block's input side in one call: the in-projection followed by the pre-scan step above,
+ * zxbcdt = u * w_in^T with u [Bz*T, D] (rows already normalised) and w_in [2*d_inner + 2*G*n + H, D], then
+ * str_mamba_conv_split on it.  Where the tensor-core GEMM takes the shape (bf16, W = 4, d_inner and G*n
+ * multiples of 32, H a multiple of 8, 16-byte aligned pointers) the conv, SiLU, split and softplus run in the
+ * projection's epilogue, so the [x B C | dt] columns never make a round trip through memory; the results are
+ * bit for bit those of the two separate calls, which is also what runs otherwise.
+ *   zxbcdt  device [Bz*T, 2*d_inner + 2*G*n + H], dtype: on return its first d_inner columns hold the gate z;
+ *           the other columns are scratch.  All other arguments as in str_gemm and str_mamba_conv_split.
+ * Returns STR_ERR_INVALID_ARG on a null pointer or a non-positive size. */
+int str_mamba_in_proj_conv(str_ctx *ctx, int dtype, int Bz, int T, int D, int H, int p, int n, int G, int W,
+                           const void *u, const void *w_in, const float *conv_w, const float *conv_b,
+                           const float *dt_bias, void *zxbcdt, void *x_out, void *B_out, void *C_out,
+                           float *dt_out, void *stream);
+
 /* out[r,:] = RMSNorm( y[r,:] * SiLU(z[r,:]) ) over d_inner columns; z is read in place from the
  * in_proj output (row stride ld_z elements, first d_inner columns). */
 int str_gated_rmsnorm(str_ctx *ctx, int dtype, int rows, int d_inner, int ld_z, float eps,

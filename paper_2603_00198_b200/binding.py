@@ -71,7 +71,8 @@ EXPORTS = [
     "str_attn_importance_workspace_size", "str_attn_importance", "str_attn_importance_ex", "str_attn_importance_static",
     "str_topk_select_workspace_size", "str_topk_select", "str_compact",
     "str_schedule_keep_counts", "str_sigmoid_schedule_bp",
-    "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_relu_squared", "str_mamba_conv_split", "str_gated_rmsnorm",
+    "str_gemm_workspace_size", "str_gemm", "str_rmsnorm", "str_relu_squared", "str_mamba_conv_split", "str_mamba_in_proj_conv",
+    "str_gated_rmsnorm",
     "str_rope_split", "str_attn_prefill_workspace_size", "str_attn_prefill", "str_attn_prefill_rows",
     "str_stack_workspace_size", "str_stack_prefill", "str_stack_prefill_ex", "str_stack_host_workspace_size",
     "str_stack_prefill_host",
@@ -359,6 +360,25 @@ def str_mamba_conv_split(ctx, zxbcdt, conv_w, conv_b, dt_bias, Bz, T, H, p, n, G
                                       c_int(G), c_int(W), _p(zxbcdt), _p(conv_w), _p(conv_b), _p(dt_bias), _p(x),
                                       _p(Bm), _p(Cm), _p(dt), _stream()), "str_mamba_conv_split")
     return x, Bm, Cm, dt
+
+
+def str_mamba_in_proj_conv(ctx, u, w_in, conv_w, conv_b, dt_bias, Bz, T, H, p, n, G):
+    """In-projection of the rows u [Bz*T, D] and the pre-scan step in one call; returns (zxbcdt, x, B, C, dt), of
+    zxbcdt only the first H*p columns (the gate z) are meaningful."""
+    W = conv_w.shape[1]
+    dev, dtp = u.device, u.dtype
+    D = u.shape[1]
+    N = 2 * H * p + 2 * G * n + H
+    assert u.shape[0] == Bz * T and tuple(w_in.shape) == (N, D)
+    zx = torch.empty((Bz * T, N), dtype=dtp, device=dev)
+    x = torch.empty((Bz, T, H, p), dtype=dtp, device=dev)
+    Bm = torch.empty((Bz, T, G, n), dtype=dtp, device=dev)
+    Cm = torch.empty((Bz, T, G, n), dtype=dtp, device=dev)
+    dt = torch.empty((Bz, T, H), dtype=torch.float32, device=dev)
+    _check(lib().str_mamba_in_proj_conv(ctx.handle, c_int(_dt(u)), c_int(Bz), c_int(T), c_int(D), c_int(H), c_int(p), c_int(n),
+                                        c_int(G), c_int(W), _p(u), _p(w_in), _p(conv_w), _p(conv_b), _p(dt_bias), _p(zx), _p(x),
+                                        _p(Bm), _p(Cm), _p(dt), _stream()), "str_mamba_in_proj_conv")
+    return zx, x, Bm, Cm, dt
 
 
 def str_gated_rmsnorm(ctx, y, zxbcdt, d_inner, eps=1e-5):

@@ -146,7 +146,7 @@ int str_gemm_fused(str_ctx *ctx, int dtype, int M, int N, int K, const void *a, 
     if (!ctx || !a || !w || !out || M < 0 || N <= 0 || K <= 0 || !STR_DTYPE_OK(dtype)) return STR_ERR_INVALID_ARG;
     if (M == 0) return STR_OK;
     if (!str_force_simt() && ctx->encode_tiled && str_gemm_tc_supported(dtype, M, N, K, a, w, residual, out))
-        return ++ctx->tc_calls, str_gemm_tc(ctx, M, N, K, a, w, residual, out, rn, (cudaStream_t)stream);
+        return ++ctx->tc_calls, str_gemm_tc(ctx, M, N, K, a, w, residual, out, rn, StrConvEpilogue{}, (cudaStream_t)stream);
     return ++ctx->fallback_calls, str_gemm_simt(ctx, dtype, M, N, K, a, w, residual, out, rn, (cudaStream_t)stream);
 }
 
@@ -155,6 +155,33 @@ extern "C" int str_gemm(str_ctx *ctx, int dtype, int M, int N, int K, const void
     (void)workspace; (void)workspace_bytes;
     const StrRowNorm none = {nullptr, 0, 0.f, 0.f, nullptr};
     return str_gemm_fused(ctx, dtype, M, N, K, a, w, residual, out, none, stream);
+}
+
+extern "C" int str_mamba_in_proj_conv(str_ctx *ctx, int dtype, int Bz, int T, int D, int H, int p, int n, int G, int W,
+                                      const void *u, const void *w_in, const float *conv_w, const float *conv_b,
+                                      const float *dt_bias, void *zxbcdt, void *x_out, void *B_out, void *C_out,
+                                      float *dt_out, void *stream) {
+    if (!ctx || !u || !w_in || !conv_w || !conv_b || !dt_bias || !zxbcdt || !x_out || !B_out || !C_out || !dt_out || Bz <= 0 ||
+        T <= 0 || D <= 0 || H <= 0 || p <= 0 || n <= 0 || G <= 0 || W <= 0 || !STR_DTYPE_OK(dtype))
+        return STR_ERR_INVALID_ARG;
+    if ((long long)Bz * T > 2147483647LL) return STR_ERR_UNSUPPORTED_SHAPE;
+    const int rows = Bz * T, d_inner = H * p, gn = G * n, N = 2 * d_inner + 2 * gn + H;
+    const StrRowNorm none = {nullptr, 0, 0.f, 0.f, nullptr};
+    const StrConvEpilogue cv = {W == 4 ? T : 0, 0, d_inner, d_inner, gn, H, conv_w, conv_b, dt_bias, (__nv_bfloat16 *)x_out,
+                                (__nv_bfloat16 *)B_out, (__nv_bfloat16 *)C_out, dt_out};
+    if (!str_force_simt() && ctx->encode_tiled && str_gemm_conv_supported(dtype, rows, N, D, u, w_in, zxbcdt, cv)) {
+        {
+            StrProfScope prof_scope(ctx, STR_CAT_GEMM, stream);
+            ++ctx->tc_calls;
+            const int rc = str_gemm_tc(ctx, rows, N, D, u, w_in, nullptr, zxbcdt, none, cv, (cudaStream_t)stream);
+            if (rc != STR_OK) return rc;
+        }
+        return str_mamba_conv_edge_rows(ctx, Bz, T, N, cv, zxbcdt, stream);
+    }
+    const int rc = str_gemm_fused(ctx, dtype, rows, N, D, u, w_in, nullptr, zxbcdt, none, stream);
+    if (rc != STR_OK) return rc;
+    return str_mamba_conv_split(ctx, dtype, Bz, T, H, p, n, G, W, zxbcdt, conv_w, conv_b, dt_bias, x_out, B_out, C_out, dt_out,
+                                stream);
 }
 
 extern "C" size_t str_attn_prefill_workspace_size(const str_attn_shape *) { return 0; }

@@ -41,8 +41,28 @@ int str_attn_prefill_simt(str_ctx *ctx, const str_attn_shape *s, int n_rows, con
                           const void *k, const void *v, float scale, void *o, cudaStream_t st);
 bool str_gemm_tc_supported(int dtype, int M, int N, int K, const void *a, const void *w, const void *residual,
                            const void *out);
+// The Mamba block's pre-scan step fused into the in-projection's epilogue.  The projection's output row is
+// [z (zoff columns) | x (d_inner) | B (gn) | C (gn) | dt (H)].  With T != 0 the epilogue, instead of storing the
+// x/B/C columns, applies the causal depthwise conv of width 4 along the rows (the three earlier rows of a warp's 32
+// consecutive rows come from its neighbouring lanes), SiLU, and stores into the split x/B/C tensors; the dt columns
+// become softplus(dt + dt_bias) in fp32.  Rows whose earlier rows belong to another warp (row % 32 < 3) are left to
+// str_mamba_conv_edge_rows: for them and for the last three rows of every 32 the epilogue stores the projection
+// itself, as the unfused GEMM would.  The arithmetic on every element is that of str_mamba_conv_split on the stored
+// bf16 projection, so both routes give the same bits.  Column segments must start on multiples of 32.
+struct StrConvEpilogue {
+    int T;                       // rows per sequence; 0 = plain GEMM epilogue
+    int row_base;                // index of the call's first row among the Bz * T rows (multiple of 32)
+    int zoff, d_inner, gn, H;
+    const float *conv_w, *conv_b, *dt_bias;
+    __nv_bfloat16 *x_out, *B_out, *C_out;    // whole tensors (row 0 = first row of the first sequence)
+    float *dt_out;
+};
+bool str_gemm_conv_supported(int dtype, int M, int N, int K, const void *a, const void *w, const void *out,
+                             const StrConvEpilogue &cv);
 int str_gemm_tc(str_ctx *ctx, int M, int N, int K, const void *a, const void *w, const void *residual, void *out,
-                const StrRowNorm &rn, cudaStream_t st);
+                const StrRowNorm &rn, const StrConvEpilogue &cv, cudaStream_t st);
+// Conv / SiLU / split of the rows the fused epilogue leaves out (row % 32 < 3), from the stored projection rows.
+int str_mamba_conv_edge_rows(str_ctx *ctx, int Bz, int T, int ld, const StrConvEpilogue &cv, const void *zxbcdt, void *stream);
 bool str_force_simt();
 bool str_ssd_tc_supported(const str_ssd_shape *s, const void *x, const void *B, const void *C, const void *y,
                           const float *D, const float *init_state);

@@ -1,7 +1,7 @@
 // Element-wise / row-wise block glue around the mixers: RMSNorm, the Mamba-2 pre-scan step
 // (causal depthwise conv + SiLU + split + softplus), gated RMSNorm, and RoPE + q/k/v split.
 // All HBM-bound; each activation is read once and written once.
-#include "common.cuh"
+#include "dispatch.cuh"
 
 namespace {
 
@@ -134,12 +134,6 @@ __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
 }
 // SiLU for results that are stored as bf16: exp2 and reciprocal on the special-function unit (relative
 // error about 2^-21, far below the 2^-9 of the storage rounding) instead of the exact exp and division.
-__device__ __forceinline__ float silu_fast(float v) {
-    float e, r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-1.4426950408889634f * v));
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
-    return v * r;
-}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -306,6 +300,67 @@ mamba_conv_split_bf16_vec_kernel(int Tlen, int H, int p, int n, int G, int zoff,
             }
             if (tb + u < t1)
                 *reinterpret_cast<uint2 *>(dst + (row0 + tb + u) * dst_ld) = make_uint2(pack2(o[0], o[1]), pack2(o[2], o[3]));
+        }
+    }
+}
+
+// The rows a fused in-projection epilogue (StrConvEpilogue) leaves out: rows r with r % 32 < 3, whose earlier rows
+// sit in another warp of that epilogue.  The projection of rows r-3 .. r is in `zxbcdt` (the epilogue stores it for
+// the first and the last three rows of every 32).  One thread: 8 channels (taps and bias held in registers) of
+// EDGE_GROUPS consecutive 32-row groups, the arithmetic of mamba_conv_split_bf16_vec_kernel.
+constexpr int EDGE_GROUPS = 8;
+__global__ void __launch_bounds__(256)
+mamba_conv_edge_rows_kernel(int rows, int Tlen, int ld, int zoff, int d_inner, int gn, const __nv_bfloat16 *__restrict__ zxbcdt,
+                            const float *__restrict__ conv_w, const float *__restrict__ conv_b,
+                            __nv_bfloat16 *__restrict__ x_out, __nv_bfloat16 *__restrict__ B_out,
+                            __nv_bfloat16 *__restrict__ C_out) {
+    const int c0 = (blockIdx.y * blockDim.x + threadIdx.x) * 8;
+    if (c0 >= d_inner + 2 * gn) return;
+    float4 w[8];
+    float bias[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        w[j] = __ldg(reinterpret_cast<const float4 *>(conv_w) + c0 + j);
+        bias[j] = __ldg(conv_b + c0 + j);
+    }
+    __nv_bfloat16 *dst;
+    int dst_ld;
+    if (c0 < d_inner) { dst = x_out + c0; dst_ld = d_inner; }
+    else if (c0 < d_inner + gn) { dst = B_out + (c0 - d_inner); dst_ld = gn; }
+    else { dst = C_out + (c0 - d_inner - gn); dst_ld = gn; }
+    const __nv_bfloat16 *src = zxbcdt + zoff + c0;
+    const int groups = (rows + 31) / 32;
+#pragma unroll 2
+    for (int gi = 0; gi < EDGE_GROUPS; ++gi) {
+        const int grp = blockIdx.x * EDGE_GROUPS + gi;
+        if (grp >= groups) break;
+        const int r0 = grp * 32;
+        uint4 raw[6];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) {
+            const int r = r0 - 3 + i;
+            raw[i] = (r >= 0 && r < rows) ? __ldg(reinterpret_cast<const uint4 *>(src + (size_t)r * ld)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        float h[6][8];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) unpack8(raw[i], h[i]);
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            const int r = r0 + k;
+            if (r < rows) {
+                const int t_in = r % Tlen;
+                float o[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float acc = bias[j];
+                    acc = fmaf(w[j].x, t_in >= 3 ? h[k][j] : 0.f, acc);
+                    acc = fmaf(w[j].y, t_in >= 2 ? h[k + 1][j] : 0.f, acc);
+                    acc = fmaf(w[j].z, t_in >= 1 ? h[k + 2][j] : 0.f, acc);
+                    acc = fmaf(w[j].w, h[k + 3][j], acc);
+                    o[j] = silu_fast(acc);
+                }
+                *reinterpret_cast<uint4 *>(dst + (size_t)r * dst_ld) = pack8(o);
+            }
         }
     }
 }
@@ -494,6 +549,17 @@ int str_mamba_conv_split_rows(str_ctx *ctx, int dtype, int Bz, int T, int H, int
         mamba_conv_split_kernel<float><<<grid, 256, 0, st>>>(T, H, p, n, G, W, zoff, (const float *)zxbcdt, conv_w, conv_b,
                                                             dt_bias, (float *)x_out, (float *)B_out, (float *)C_out,
                                                             dt_out);
+    return str_launch_ok(ctx);
+}
+
+int str_mamba_conv_edge_rows(str_ctx *ctx, int Bz, int T, int ld, const StrConvEpilogue &cv, const void *zxbcdt, void *stream) {
+    StrProfScope prof_scope(ctx, STR_CAT_ELEMENTWISE, stream);
+    const long long rows = (long long)Bz * T;
+    if (rows <= 0 || rows > 2147483647LL) return STR_ERR_INVALID_ARG;
+    dim3 grid(ceil_div(ceil_div((int)rows, 32), EDGE_GROUPS), ceil_div((cv.d_inner + 2 * cv.gn) / 8, 256));
+    mamba_conv_edge_rows_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((int)rows, T, ld, cv.zoff, cv.d_inner, cv.gn,
+                                                                       (const __nv_bfloat16 *)zxbcdt, cv.conv_w, cv.conv_b,
+                                                                       cv.x_out, cv.B_out, cv.C_out);
     return str_launch_ok(ctx);
 }
 

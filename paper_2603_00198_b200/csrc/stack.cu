@@ -4,7 +4,16 @@
 // schedule does not depend on the input).
 #include <string.h>
 
+#include <stdlib.h>
+
 #include "dispatch.cuh"
+
+// Debug switch: STR_CONV_FUSE=0 keeps the pre-scan step in its own kernel (A/B runs of the fused epilogue).
+static bool str_conv_fusion_on() {
+    static int v = -1;
+    if (v < 0) { const char *e = getenv("STR_CONV_FUSE"); v = (e && e[0] == '0') ? 0 : 1; }
+    return v == 1;
+}
 
 namespace {
 
@@ -211,10 +220,15 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
         void *mix_out = (last && !reduce) ? hidden_out : hid[hsel];
 
         // the layer's first projection with the RMSNorm of the layer input fused in: [rows x N] = RMSNorm(cur) W^T into `proj`
-        auto norm_and_project = [&](int N, const void *w) -> int {
+        // With `conv` (a Mamba layer) the projection's epilogue also runs the pre-scan step when the shapes allow;
+        // *conv_fused tells the caller which of the two follow-up kernels is due.
+        auto norm_and_project = [&](int N, const void *w, const StrConvEpilogue *conv = nullptr, bool *conv_fused = nullptr) -> int {
             const bool fed = feed && l == 0;
             const int step = fed ? feed->rows_per_chunk : rows;
             const size_t esz = dtype_size(dtype);
+            const bool fuse = conv && !str_force_simt() && str_conv_fusion_on() && step % 32 == 0 &&
+                              str_gemm_conv_supported(dtype, rows < step ? rows : step, N, D, cur, w, proj, *conv);
+            if (conv_fused) *conv_fused = fuse;
             for (int j = 0, r0 = 0; r0 < rows; ++j, r0 += step) {
                 const int nr = rows - r0 < step ? rows - r0 : step;
                 float *ss_blk = ssb[0] + (size_t)r0 * ntD;
@@ -223,6 +237,15 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
                     STR_TRY(str_row_sumsq(ctx, dtype, nr, D, (const char *)cur + (size_t)r0 * D * esz, ss_blk, stream));
                 }
                 const StrRowNorm rn = {cur_ss + (size_t)r0 * ntD, ntD, inv_D, d->norm_eps, nullptr};
+                if (fuse) {
+                    StrProfScope prof_scope(ctx, STR_CAT_GEMM, stream);
+                    StrConvEpilogue cv = *conv;
+                    cv.row_base = r0;
+                    ++ctx->tc_calls;
+                    STR_TRY(str_gemm_tc(ctx, nr, N, D, (const char *)cur + (size_t)r0 * D * esz, w, nullptr,
+                                        (char *)proj + (size_t)r0 * N * esz, rn, cv, st));
+                    continue;
+                }
                 STR_TRY(str_gemm_fused(ctx, dtype, nr, N, D, (const char *)cur + (size_t)r0 * D * esz, w, nullptr,
                                        (char *)proj + (size_t)r0 * N * esz, rn, stream));
             }
@@ -259,16 +282,23 @@ static int stack_prefill_impl(str_ctx *ctx, const str_stack_desc *d, const str_s
         const int rows_out = reduce ? Bz * (K + M) : rows;
         if (L.kind == STR_LAYER_MAMBA) {
             const int d_inner = d->H * d->p, gn = d->G * d->n, dip = 2 * d_inner + 2 * gn + d->H;
+            // conv + SiLU + split + softplus(dt) ride in the in-projection's epilogue when the kernel supports the shape
+            StrConvEpilogue conv = {d->conv_width == 4 ? T : 0, 0, reduce ? 0 : d_inner, d_inner, gn, d->H, L.conv_w, L.conv_b,
+                                    L.dt_bias, (__nv_bfloat16 *)bufA, (__nv_bfloat16 *)bufB, (__nv_bfloat16 *)bufC, dt};
+            bool conv_fused = false;
             if (reduce) {
                 // the gate z is only needed for the rows that survive: project [x B C | dt] for every row now (the
                 // weight rows after the first d_inner) and z for the kept rows after the selection
                 const char *w_rest = (const char *)L.w_in + (size_t)d_inner * D * dtype_size(dtype);
-                STR_TRY(norm_and_project(dip - d_inner, w_rest));
+                STR_TRY(norm_and_project(dip - d_inner, w_rest, &conv, &conv_fused));
             } else {
-                STR_TRY(norm_and_project(dip, L.w_in));
+                STR_TRY(norm_and_project(dip, L.w_in, &conv, &conv_fused));
             }
-            STR_TRY(str_mamba_conv_split_rows(ctx, dtype, Bz, T, d->H, d->p, d->n, d->G, d->conv_width, !reduce, proj,
-                                              L.conv_w, L.conv_b, L.dt_bias, bufA, bufB, bufC, dt, stream));
+            if (conv_fused)
+                STR_TRY(str_mamba_conv_edge_rows(ctx, Bz, T, conv.zoff + d_inner + 2 * gn + d->H, conv, proj, stream));
+            else
+                STR_TRY(str_mamba_conv_split_rows(ctx, dtype, Bz, T, d->H, d->p, d->n, d->G, d->conv_width, !reduce, proj,
+                                                  L.conv_w, L.conv_b, L.dt_bias, bufA, bufB, bufC, dt, stream));
             str_ssd_shape s = {Bz, T, d->H, d->p, d->n, d->G, d->Q, dtype};
             STR_TRY(str_mamba2_prefill(ctx, &s, bufA, dt, L.A, bufB, bufC, nullptr, nullptr, bufY, fs_out, sub,
                                        r.sub_bytes, stream));

@@ -75,6 +75,7 @@ def test_newer_entry_points_validate_on_the_host(libstr):
     assert libstr.str_attn_prefill_rows(None, None, 4, None, None, None, None, c_float(1.0), None, None, c_size_t(0), None) == -1
     assert libstr.str_stack_prefill_ex(None, None, None, None, None, None, None, None, None, None, c_size_t(0), None) == -1
     assert libstr.str_selftest_wait_timeout(None, ctypes.c_uint(10), None) == -1
+    assert libstr.str_mamba_in_proj_conv(None, 1, 1, 8, 64, 8, 32, 32, 1, 4, *([None] * 11)) == -1
     tc, fb = ctypes.c_longlong(), ctypes.c_longlong()
     assert libstr.str_path_counts(None, ctypes.byref(tc), ctypes.byref(fb)) == -1
     # the schedule helper with layer kinds: unknown kinds and missing arrays are refused

@@ -90,6 +90,31 @@ def test_conv_split_and_gated_norm(ctx, dtype, Bz, T, H, p, n, G):
     assert max_rel_err(got, ref) <= TOL[dtype]
 
 
+@pytest.mark.parametrize("dtype,Bz,T,D,H,p,n,G", [("bf16", 1, 4224, 512, 8, 64, 128, 2), ("bf16", 3, 333, 256, 8, 32, 32, 1),
+                                                  ("bf16", 1, 100, 256, 8, 64, 128, 2), ("bf16", 4, 31, 128, 16, 64, 64, 1),
+                                                  ("bf16", 2, 1, 128, 8, 32, 32, 1), ("f32", 2, 70, 64, 8, 32, 16, 1),
+                                                  ("bf16", 1, 300, 256, 4, 16, 8, 1)])
+def test_in_projection_with_the_prescan_step_in_its_epilogue(ctx, dtype, Bz, T, D, H, p, n, G):
+    """str_mamba_in_proj_conv against the two calls it stands for (str_gemm, str_mamba_conv_split): every output equal
+    bit for bit, whether the conv ran in the projection's epilogue (the first five cases: sequences that start and end
+    inside a warp's 32 rows, fewer rows than one tile, one-token sequences) or the call composed the two kernels."""
+    d_inner, gn = H * p, G * n
+    N = 2 * d_inner + 2 * gn + H
+    g = inputs.rng(58, T + D)
+    u = dev(inputs.to_grid(g.standard_normal((Bz * T, D), dtype=np.float32), dtype), dtype)
+    w = dev(inputs.to_grid(g.standard_normal((N, D), dtype=np.float32) / np.sqrt(D), dtype), dtype)
+    cw = dev(g.uniform(-0.5, 0.5, size=(d_inner + 2 * gn, 4)).astype(np.float32))
+    cb = dev(g.uniform(-0.1, 0.1, size=(d_inner + 2 * gn,)).astype(np.float32))
+    dtb = dev(inputs.softplus_inverse(g.uniform(1e-3, 1e-1, size=H)).astype(np.float32))
+    zx = binding.str_gemm(ctx, u, w)
+    ref = binding.str_mamba_conv_split(ctx, zx, cw, cb, dtb, Bz, T, H, p, n, G)
+    got = binding.str_mamba_in_proj_conv(ctx, u, w, cw, cb, dtb, Bz, T, H, p, n, G)
+    ctx.check_status()
+    assert bool((got[0][:, :d_inner] == zx[:, :d_inner]).all())                 # the gate columns
+    for a, b, name in zip(got[1:], ref, "xBCd"):
+        assert bool((a == b).all()), name
+
+
 # the last case has more than 65535 rows (batch 4 of the 16512-token attention layers has 66048)
 @pytest.mark.parametrize("dtype,Bz,T,Hq,Hkv,d", [("bf16", 1, 200, 8, 2, 128), ("f32", 2, 50, 4, 4, 32),
                                                    ("bf16", 2, 35000, 2, 1, 16)])
