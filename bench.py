@@ -25,7 +25,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # Measured DRAM traffic / algorithmic bytes of one launch, from the ncu captures summarised under profiles/
 # (smaller cases of the same kernels; traffic grows in proportion to the algorithmic bytes).  A kernel that
 # has changed since its capture is left out (traffic is then reported as null).
-NCU_TRAFFIC_RATIO = {"gemm": 464.1 / 343.2, "ssd_scan": 115.1 / 157.9, "mamba_score": 86.7 / 84.0, "compact": 226.6 / 270.7}
+NCU_TRAFFIC_RATIO = {"gemm": 514.1 / 343.2, "ssd_scan": 115.1 / 157.9, "mamba_score": 86.7 / 84.0, "compact": 226.6 / 270.7}
 
 
 def peaks():

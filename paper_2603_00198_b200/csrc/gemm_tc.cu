@@ -1,6 +1,8 @@
 // bf16 GEMM on the 5th-generation tensor cores: out[M,N] = a[M,K] * w[N,K]^T (+ residual).
 //
-// Persistent, warp-specialised kernel, one CTA per SM:
+// Two persistent, warp-specialised kernels with the same roles and the same epilogue function.  gemm_tc_pair_kernel
+// (further down) runs one 256 x 256 tile per cluster of two CTAs and is the one used above 128 rows; gemm_tc_kernel
+// runs one 128 x 256 tile per CTA:
 //   warp 0     TMA producer: streams 128x64 A tiles and 256x64 W tiles (128-byte swizzle) through a
 //              4-stage shared-memory ring guarded by full/empty mbarriers.
 //   warp 1     MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16) into one of two
@@ -15,7 +17,8 @@
 // Tiles are walked in bands of 8 column tiles so that a band of W stays in L2 while A streams.
 // The epilogue can fuse the RMSNorm that surrounds the projections of a pre-norm block: it scales the accumulator
 // row by 1/rms of the A row (from partial sums of squares left by the kernel that wrote A), and it leaves the
-// partial sums of squares of its own output rows, one per 256-column tile, for the next projection.
+// partial sums of squares of its own output rows, one per 256-column tile, for the next projection.  For a Mamba
+// in-projection it can run the block's pre-scan step (conv, SiLU, split, softplus) instead of storing the projection.
 // Every mbarrier wait is bounded; on give-up the kernel records STR_ERR_TIMEOUT and tears down.
 #include <stdlib.h>
 
