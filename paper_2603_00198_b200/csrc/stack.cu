@@ -8,11 +8,11 @@
 
 #include "dispatch.cuh"
 
-// Debug switch: STR_CONV_FUSE=0 keeps the pre-scan step in its own kernel (A/B runs of the fused epilogue).
+// Debug switch: STR_CONV_FUSE=0 keeps the pre-scan step in its own kernel (A/B runs of the fused epilogue).  Read at
+// every call, so that one process can run both routes.
 static bool str_conv_fusion_on() {
-    static int v = -1;
-    if (v < 0) { const char *e = getenv("STR_CONV_FUSE"); v = (e && e[0] == '0') ? 0 : 1; }
-    return v == 1;
+    const char *e = getenv("STR_CONV_FUSE");
+    return !(e && e[0] == '0');
 }
 
 namespace {

@@ -152,6 +152,32 @@ def test_select_before_the_mixer_epilogue_leaves_survivors_bit_identical(ctx, pa
         assert bool((out2[b] == out[b][idx2[b].long()]).all())
 
 
+def test_stack_is_bit_identical_on_every_gemm_route(monkeypatch):
+    """The GEMM on CTA pairs against one CTA per tile, and the Mamba pre-scan step in the in-projection's epilogue
+    against its own kernel: four routes through the same arithmetic in the same order.  A reducing hybrid stack on
+    tensor-core shapes (several row tiles, a ragged last tile, two sequences) must come out bit for bit the same on
+    all of them, hidden states, positions, ids, scores and selections."""
+    n_vis, M, Bz = 700, 20, 2
+    layers = inputs.stack_params(71, "MAM", MS_TC, AS_TC, "bf16")
+    h0 = dev(inputs.hidden_inputs(71, n_vis + M, MS_TC["D"], "bf16", batch=Bz), "bf16")
+    results = []
+    for pair, fuse in (("1", "1"), ("0", "1"), ("1", "0"), ("0", "0")):
+        monkeypatch.setenv("STR_GEMM_PAIR", pair)
+        monkeypatch.setenv("STR_CONV_FUSE", fuse)
+        c = binding.Context(0)
+        st = binding.Stack(c, layers, "bf16", Bz, n_vis, M, [n_vis // 2, n_vis // 2, n_vis // 4], Q=MS_TC["Q"])
+        out, pos, idx, tr = binding.str_stack_prefill(st, h0, want_trace=True)
+        c.check_status()
+        assert c.path_counts()[1] == 0
+        results.append((out, pos, idx, tr))
+        c.close()
+    ref = results[0]
+    for got in results[1:]:
+        assert bool((got[0] == ref[0]).all()) and bool((got[1] == ref[1]).all()) and bool((got[2] == ref[2]).all())
+        for a, b in zip(got[3], ref[3]):
+            assert bool((a["scores"] == b["scores"]).all()) and bool((a["kept"] == b["kept"]).all())
+
+
 @pytest.mark.parametrize("dtype,shape", [("f32", MS), ("bf16", MS), ("bf16", MS_TC)])
 def test_single_mamba_layer_reduced_by_the_full_dynamic_score(ctx, dtype, shape):
     """The scoring ablation inside the stack: selection by |w| of Eq. 1 instead of Eq. 2.  The budget is set
